@@ -1,0 +1,301 @@
+"""Pins for the CPU oracle: everything here compares the oracle with something that is NOT the
+oracle -- the schedules printed in the paper, a brute-force broadcast simulation, closed forms,
+the paper's lemmas, and brute-force definitions on tiny inputs."""
+import numpy as np
+import pytest
+
+import oracle
+from tests import bcast_sim
+from tests.golden_tables import SECOND_P9, TABLES, load
+
+
+# ---------------------------------------------------------------- printed worked examples
+@pytest.mark.parametrize("name", TABLES)
+def test_printed_tables_match_both_forms(name):
+    g = load(name)
+    p, q = g["p"], g["q"]
+    assert oracle.q_of(p) == q
+    assert list(oracle.skips(p)) == g["skips"]                      # captions of Tables 1-4
+    bb = oracle.baseblock_list(p)
+    assert list(bb[1:]) == g["baseblock"][1:]                       # root cell ignored
+    assert [oracle.baseblock(p, r) for r in range(1, p)] == g["baseblock"][1:]   # Algorithm 2
+    recv_a, send_a = oracle.full_table(p)                           # array form
+    recv_r, send_r = oracle.build_range(p, 0, p)                    # per-rank form, Alg. 4/5
+    recv_u, send_u = oracle.build_range(p, 0, p, special=False)     # two-window rule everywhere
+    for recv, send in ((recv_a, send_a), (recv_r, send_r), (recv_u, send_u)):
+        assert np.array_equal(recv, g["recv"])
+        assert np.array_equal(send, g["send"])
+
+
+def test_second_p9_schedule_is_valid_but_not_ours():
+    """Table 5, right: also a correct schedule, differing in the four bold cells.  The simulation
+    accepts it, so the simulation alone does not pin the construction; the printed tables do."""
+    left, right = load(TABLES[-1]), load(SECOND_P9)
+    p, q = 9, 4
+    recv, send = oracle.full_table(p)
+    assert np.array_equal(recv, left["recv"]) and np.array_equal(send, left["send"])
+    diff = [(int(r), int(k)) for r, k in zip(*np.nonzero(recv != right["recv"]))]
+    assert diff == [(8, 1), (8, 2)]                                  # bold receive cells
+    diff = [(int(r), int(k)) for r, k in zip(*np.nonzero(send != right["send"]))]
+    assert sorted(diff) == [(5, 2), (6, 1)]                          # bold send cells
+    for n in (1, 2, 5, q + 3):
+        assert bcast_sim.simulate(p, n, oracle.expand(p, n, right["recv"], right["send"])) is None
+        assert bcast_sim.simulate(p, n, oracle.expand(p, n, left["recv"], left["send"])) is None
+
+
+# ---------------------------------------------------------------- Algorithm 1 and Lemma 1
+def test_skips_closed_form_and_lemma1():
+    for p in list(range(1, 3000)) + [2**20 + 1, 2**30 - 1, 2**31 - 1, 100003, 2**16, 2**16 + 1]:
+        s = [int(v) for v in oracle.skips(p)]
+        q = oracle.q_of(p)
+        assert q == bcast_sim.ceil_log2(p) and len(s) == q + 1
+        assert s == bcast_sim.closed_form_skips(p)                  # nested ceil-halving
+        assert s[0] == 1 and s[q] == p
+        if q >= 1:
+            assert s[1] == 2 or p < 2 or q == 1 and s[1] == p
+        for k in range(q):
+            assert s[k] < s[k + 1]
+            assert 2 * s[k] >= s[k + 1]                             # Lemma 1, first claim
+            assert sum(s[: k + 1]) >= s[k + 1] - 1                  # Lemma 1, second claim
+        assert sum(s[k + 1] - s[k] for k in range(q)) == p - 1      # Lemma 1, third claim
+        if p & (p - 1) == 0:
+            assert s == [1 << k for k in range(q + 1)]              # powers of two
+
+
+# ---------------------------------------------------------------- Algorithm 2
+def test_baseblock_two_ways_and_structure():
+    for p in list(range(2, 700)) + [1000, 1024, 1025, 4097]:
+        s = [int(v) for v in oracle.skips(p)]
+        bb = oracle.baseblock_list(p)
+        assert bb[0] == -1 and oracle.baseblock(p, 0) == -1
+        assert [oracle.baseblock(p, r) for r in range(1, p)] == list(bb[1:])
+        for k in range(oracle.q_of(p)):
+            assert bb[s[k]] == k                                     # "baseblock of skips[k] is k"
+            lo, hi = s[k], s[k + 1] - 1                              # homerange repeats [1, ...]
+            assert list(bb[lo + 1: hi + 1]) == list(bb[1: hi - lo + 1])
+        assert (bb[1:-1] != bb[2:]).all()                            # successive baseblocks differ
+
+
+def test_baseblock_power_of_two_is_ctz():
+    for q in range(1, 13):
+        p = 1 << q
+        bb = oracle.baseblock_list(p)
+        assert all(bb[r] == (r & -r).bit_length() - 1 for r in range(1, p))
+
+
+# ---------------------------------------------------------------- the range search
+def test_rangeblocks_equals_definition():
+    rng = np.random.default_rng(1)
+    for p in list(range(2, 80)) + [127, 128, 129, 255, 300, 513]:
+        bb = oracle.baseblock_list(p)
+        pairs = [(a, b) for a in range(-p - 2, p + 2) for b in range(a - 1, a + p + 1)]
+        if len(pairs) > 4000:
+            pairs = [pairs[i] for i in rng.choice(len(pairs), 4000, replace=False)]
+        for a, b in pairs:
+            want = 0
+            if b - a + 1 >= p:
+                want = (1 << oracle.q_of(p)) - 1
+            else:
+                for x in range(a, b + 1):
+                    if x % p:
+                        want |= 1 << int(bb[x % p])
+            assert oracle.rangeblocks(p, a, b) == want, (p, a, b)
+            assert oracle.rangeblocks_scan(p, a, b) == want, (p, a, b)
+
+
+def test_lemma2_window_counts():
+    """Lemma 2: a range of skips[k] processors holds >= k different baseblocks, a range of
+    1 + sum_{i<k} skips[i] processors holds >= k+1 (ranges of non-root processors)."""
+    for p in list(range(2, 260)) + [511, 512, 513, 1000]:
+        s = [int(v) for v in oracle.skips(p)]
+        q = oracle.q_of(p)
+        bb = oracle.baseblock_list(p).astype(np.int64)
+        onehot = np.zeros((p, q), dtype=np.int64)
+        onehot[np.arange(1, p), bb[1:]] = 1
+        pre = np.vstack([np.zeros((1, q), dtype=np.int64), np.cumsum(onehot, axis=0)])  # pre[x+1]
+        for k in range(q + 1):
+            for size, least in ((s[k], k), (1 + sum(s[:k]), k + 1)):
+                if size > p - 1:
+                    continue
+                a = np.arange(1, p - size + 1)
+                distinct = ((pre[a + size] - pre[a]) > 0).sum(axis=1)
+                assert (distinct >= min(least, q)).all(), (p, k, size)
+
+
+# ---------------------------------------------------------------- schedule invariants
+def _check_rows(p, recv, send):
+    q = oracle.q_of(p)
+    s = [int(v) for v in oracle.skips(p)]
+    bb = oracle.baseblock_list(p)
+    assert list(send[0]) == list(range(q))                           # root sends block k in round k
+    assert sorted(recv[0]) == list(range(-q, 0))                     # root row: all previous-phase
+    for r in range(1, p):
+        h = max(k for k in range(q) if s[k] <= r)
+        row = [int(v) for v in recv[r]]
+        assert row[h] == bb[r]                                       # baseblock in the home round
+        others = sorted(row[:h] + row[h + 1:])
+        assert others == sorted(b - q for b in range(q) if b != bb[r])   # q-1 different others
+        allowed = {bb[r] - q}
+        for i in range(q):                                           # a sent block was received before
+            v = int(send[r][i])
+            assert v in allowed or v == bb[r] and i > h, (p, r, i)
+            allowed.add(row[i])
+    t = (np.arange(p)[:, None] + np.array(s[:q])[None, :]) % p       # Algorithm 5 / Algorithm 9
+    assert np.array_equal(send, recv[t, np.arange(q)[None, :]])
+
+
+def test_row_invariants_small_p():
+    for p in list(range(2, 400)) + [1023, 1024, 1025]:
+        recv, send = oracle.full_table(p)
+        _check_rows(p, recv, send)
+
+
+def test_power_of_two_closed_form():
+    """For p = 2^q the schedule is the classical one: baseblock ctz(r); in a non-home round i the
+    window (r-2^(i+1), r-2^i] holds exactly one multiple of 2^i and its block i+ctz(.) is new."""
+    for q in range(1, 13):
+        p = 1 << q
+        recv, _ = oracle.full_table(p)
+        for r in range(p):
+            for i in range(q):
+                if r >> i == 1:
+                    want = (r & -r).bit_length() - 1
+                else:
+                    m = ((r >> i) - 1) % (1 << (q - i))
+                    ctz = (m & -m).bit_length() - 1 if m else q - i
+                    want = i + ctz - q
+                assert recv[r][i] == want, (p, r, i)
+
+
+def test_two_forms_agree_exhaustive_small_and_sampled_large():
+    for p in range(1, 1400):
+        if p == 1:
+            assert oracle.full_table(1)[0].shape == (1, 0)
+            continue
+        a, b = oracle.full_table(p), oracle.build_range(p, 0, p)
+        assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1]), p
+    rng = np.random.default_rng(7)
+    for p in (4097, 65535, 65537, 100003, 2**20 + 1):
+        ranks = np.unique(np.concatenate([rng.integers(0, p, 300), [0, 1, 2, p - 2, p - 1]]))
+        a = oracle.full_table(p)
+        b = oracle.build_ranks(p, ranks)
+        assert np.array_equal(a[0][ranks], b[0]) and np.array_equal(a[1][ranks], b[1]), p
+
+
+def test_special_rounds_equal_uniform_rule():
+    """Rounds 0 and q-1 as Algorithm 4 writes them (baseblock of r-1; the last missing block)
+    give what the two-window rule gives."""
+    for p in range(2, 500):
+        a = oracle.build_range(p, 0, p, special=True)
+        b = oracle.build_range(p, 0, p, special=False)
+        assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1]), p
+
+
+def test_root_cell_reading_is_immaterial():
+    """Whether the root adds nothing, block 0 or every block to a range containing it does not
+    change any schedule (the printed tables show 0 in four tables and -1 in one)."""
+    try:
+        for p in list(range(2, 300)) + [1000, 1024, 1025, 4099]:
+            oracle.set_root_mode(0)
+            base = oracle.build_range(p, 0, p)
+            for mode in (1, 2):
+                oracle.set_root_mode(mode)
+                alt = oracle.build_range(p, 0, p)
+                assert np.array_equal(base[0], alt[0]) and np.array_equal(base[1], alt[1]), (p, mode)
+    finally:
+        oracle.set_root_mode(0)
+
+
+def test_degenerate_p():
+    assert oracle.q_of(1) == 0 and list(oracle.skips(1)) == [1]
+    recv, send = oracle.full_table(2)
+    assert recv.tolist() == [[-1], [0]] and send.tolist() == [[0], [-1]]
+    recv, send = oracle.build_range(2, 0, 2)
+    assert recv.tolist() == [[-1], [0]] and send.tolist() == [[0], [-1]]
+    recv, send = oracle.full_table(3)
+    assert bcast_sim.simulate(3, 4, oracle.expand(3, 4, recv, send)) is None
+
+
+# ---------------------------------------------------------------- Algorithm 6 + brute force
+def test_expansion_closed_form():
+    """Round j uses entry k=(j+x) mod q and block sched[k] - x + q*floor((j+x)/q), x the number of
+    virtual rounds; below 0 -> -1, above n-1 -> n-1."""
+    for p in (2, 3, 9, 20, 33, 64, 100):
+        q = oracle.q_of(p)
+        s = [int(v) for v in oracle.skips(p)]
+        recv, send = oracle.full_table(p)
+        for n in (1, 2, 3, q, q + 1, 2 * q + 3, 40):
+            tab = oracle.expand(p, n, recv, send)
+            x = (q - (n - 1 + q) % q) % q
+            assert (x + n - 1 + q) % q == 0
+            for r in range(p):
+                for j in range(n - 1 + q):
+                    i = j + x
+                    k = i % q
+                    want = []
+                    for row in (send, recv):
+                        blk = int(row[r][k]) - x + q * (i // q)
+                        want.append(-1 if blk < 0 else min(blk, n - 1))
+                    want += [(r + s[k]) % p, (r - s[k]) % p]
+                    assert tab[r, j].tolist() == want, (p, n, r, j)
+
+
+def test_broadcast_simulation_every_p_up_to_1024():
+    for p in range(2, 1025):
+        q = oracle.q_of(p)
+        recv, send = oracle.full_table(p)
+        for n in (1, 2, 5, q + 3):
+            err = bcast_sim.simulate(p, n, oracle.expand(p, n, recv, send))
+            assert err is None, (p, n, err)
+
+
+def test_broadcast_simulation_rerooted():
+    rng = np.random.default_rng(3)
+    for p in (2, 3, 9, 20, 31, 32, 33, 100, 257, 1000):
+        q = oracle.q_of(p)
+        recv, send = oracle.full_table(p)
+        for n in (1, 5, q + 3):
+            tab = oracle.expand(p, n, recv, send)
+            for root in {0, 1, p - 1, int(rng.integers(0, p))}:
+                err = bcast_sim.simulate(p, n, bcast_sim.reroot(tab, root), root=root)
+                assert err is None, (p, n, root, err)
+
+
+def test_simulation_rejects_planted_mistakes():
+    """The simulation is only a pin if it fails for wrong schedules: plant typical mistakes in a
+    copy of the oracle's tables (on the CPU) and expect a violation."""
+    p, n = 33, 9
+    q = oracle.q_of(p)
+    recv, send = oracle.full_table(p)
+    assert bcast_sim.simulate(p, n, oracle.expand(p, n, recv, send)) is None
+    bad = recv.copy(); bad[7, 1], bad[7, 2] = recv[7, 2], recv[7, 1]         # swapped rounds
+    assert bcast_sim.simulate(p, n, oracle.expand(p, n, bad, send)) is not None
+    bad = send.copy(); bad[5, 0] = send[5, 0] + 1                             # wrong send block
+    assert bcast_sim.simulate(p, n, oracle.expand(p, n, recv, bad)) is not None
+    bad_r, bad_s = recv.copy(), send.copy()                                   # min instead of max
+    bad_r[:, :] = np.where(recv < 0, -q - 1 - recv, recv)
+    bad_s[:, :] = np.where(send < 0, -q - 1 - send, send)
+    assert bcast_sim.simulate(p, n, oracle.expand(p, n, bad_r, bad_s)) is not None
+    tab = oracle.expand(p, n, recv, send)                                     # wrong neighbour
+    tab2 = tab.copy(); tab2[:, 3, 2] = (tab[:, 3, 2] + 1) % p
+    assert bcast_sim.simulate(p, n, tab2) is not None
+    tab2 = tab.copy(); tab2[:, -1, :2] = -1                                   # one round short
+    assert bcast_sim.simulate(p, n, tab2) is not None
+
+
+# ---------------------------------------------------------------- checksum helper
+def test_checksum_definition_and_additivity():
+    rng = np.random.default_rng(5)
+    buf = rng.integers(-30, 30, 1000).astype(np.int8)
+    mask = (1 << 64) - 1
+
+    def mix(e):
+        z = (e + 0x9E3779B97F4A7C15) & mask
+        z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & mask
+        z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & mask
+        return z ^ (z >> 31)
+
+    assert mix(0) == 0xE220A8397B1DCDAF          # first output of splitmix64 seeded with 0
+    want = sum(int(np.uint8(v)) * mix(17 + e) for e, v in enumerate(buf)) & mask
+    assert oracle.checksum(buf, 17) == want
+    assert (oracle.checksum(buf[:400], 17) + oracle.checksum(buf[400:], 417)) & mask == want
