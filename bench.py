@@ -1,0 +1,345 @@
+#!/usr/bin/env python
+"""Benchmark of the schedule construction on one B200 (or N independent replicas).
+
+A step = one bcs_build call for every rank of p = 2^20 + 1 (q = 21): the receive and the send
+schedule, 2 * 21 int8 entries per rank.  The metric is schedule ranks built per second.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "schedule ranks built/sec (int8 recv+send, q entries)"
+UNIT = "ranks/s"
+
+# Integer work the receive schedule of one rank needs in the construction that is timed
+# (descent steps of the range search, measured by a CPU count of the same loop structure, times
+# the integer operations of one step) -- see DESIGN.md, "Roofline".
+ALU_LANES_PER_SM = 64          # INT32 lanes per SM per clock
+SM_COUNT = 148
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), float(d.get("sm_max_mhz", 1965.0)), "measured"
+    return 6650.0, 1965.0, "fallback"
+
+
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def run_reference(args) -> None:
+    """CPU oracle (per-rank form: Algorithms 4 and 5 for every rank) on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2205_10072_b200 import workloads
+    p = workloads.P_SINGLE
+    sample = 32768                       # ranks per step: a bounded slice of the same workload
+    lo = (p // 2) - sample // 2
+    for _ in range(args.warmup):
+        oracle.build_range(p, lo, lo + sample)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.build_range(p, lo, lo + sample)
+    dt = time.perf_counter() - t0
+    value = args.steps * sample / dt
+    cores = oracle.num_threads()
+    sample_txt = "ranks %d..%d of p=2^20+1 per step (per-rank form, Algorithms 4+5)" % (lo, lo + sample - 1)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8/int32",
+        "data": "synthetic",
+        "config": {"workload": "single p=2^20+1 (q=21), all ranks, recv+send int8", "p": p,
+                   "sample": sample_txt},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": sample_txt},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def _event_ms(torch, fn, flush, steps, warmup):
+    """Device time of `steps` calls of fn, each preceded by an (untimed) L2 flush."""
+    for _ in range(warmup):
+        flush()
+        fn()
+    torch.cuda.synchronize()
+    pairs = []
+    for _ in range(steps):
+        flush()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        pairs.append((a, b))
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in pairs]
+
+
+def run_ours(args) -> None:
+    import torch
+    import torch.distributed as dist
+
+    import paper_2205_10072_b200 as bcs
+    from paper_2205_10072_b200 import workloads
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    bcs.lib()
+
+    hbm_gbs, sm_max_mhz, peak_src = _peaks()
+    p = workloads.P_SINGLE
+    q = bcs.bcs_q(p)
+    nb = p * q
+    recv = torch.empty(nb, dtype=torch.int8, device="cuda")
+    send = torch.empty(nb, dtype=torch.int8, device="cuda")
+    flush_buf = torch.empty(256 << 20, dtype=torch.int8, device="cuda")   # > 126 MB L2
+
+    def flush():
+        flush_buf.fill_(1)
+
+    def step():
+        bcs.bcs_build(p, 0, p, recv, send)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- the timed region: K steps, device time per step by CUDA events, L2 flushed between
+    for _ in range(args.warmup):
+        flush()
+        step()
+    barrier()
+    with ClockSampler(local) as clk:
+        t_wall0 = time.perf_counter()
+        ms = _event_ms(torch, step, flush, args.steps, 0)
+        barrier()
+        t_wall = time.perf_counter() - t_wall0
+    total_ms = sum(ms)
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * p / (ms_per_step * 1e-3)
+
+    out = None
+    if rank == 0:
+        # ---- per-kernel times (same protocol): receive kernel alone, then the send kernel
+        recv_ms = statistics.mean(_event_ms(torch, lambda: bcs.bcs_build(p, 0, p, recv, None),
+                                            flush, max(20, args.steps // 4), 3))
+        send_ms = max(ms_per_step - recv_ms, 0.0)
+
+        # ---- end to end: host buffers, D2H copies inside the timed region
+        stage = torch.empty(2 * ((nb + 255) // 256 * 256), dtype=torch.int8, device="cuda")
+        h_recv = torch.empty(nb, dtype=torch.int8).pin_memory()
+        h_send = torch.empty(nb, dtype=torch.int8).pin_memory()
+        e2e_steps = max(5, min(args.steps, 50))
+        for _ in range(3):
+            bcs.bcs_build_to_host(p, 0, p, h_recv, h_send, stage)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            bcs.bcs_build_to_host(p, 0, p, h_recv, h_send, stage)
+            torch.cuda.synchronize()
+        e2e_dt = (time.perf_counter() - t0) / e2e_steps
+        del stage
+
+        # ---- other entry points of the path (reported, not part of the metric)
+        aux = {}
+        pe, ne = workloads.P_EXPAND, workloads.N_EXPAND
+        qe = bcs.bcs_q(pe)
+        er = torch.empty(pe * qe, dtype=torch.int8, device="cuda")
+        es = torch.empty(pe * qe, dtype=torch.int8, device="cuda")
+        bcs.bcs_build(pe, 0, pe, er, es)
+        rounds = ne - 1 + qe
+        table = torch.empty((pe, rounds, 4), dtype=torch.int32, device="cuda")
+        ex_ms = statistics.mean(_event_ms(
+            torch, lambda: bcs.bcs_expand(pe, ne, 0, pe, er, es, table), flush, 20, 3))
+        ex_bytes = pe * rounds * 16
+        aux["expand"] = {"workload": "p=100003, n=1000, all ranks, 1016 rounds", "ms": ex_ms,
+                         "bytes": ex_bytes, "gbs": ex_bytes / ex_ms / 1e6,
+                         "roofline": {"bound": "hbm", "achieved": ex_bytes / ex_ms / 1e6,
+                                      "peak": hbm_gbs, "unit": "GB/s",
+                                      "frac": ex_bytes / ex_ms / 1e6 / hbm_gbs, "traffic": None,
+                                      "peak_source": peak_src}}
+        sums = torch.zeros(1, dtype=torch.int64, device="cuda")
+        tb = table.view(torch.int8).view(-1)
+        ck_ms = statistics.mean(_event_ms(
+            torch, lambda: bcs.bcs_checksum(tb, 0, sums), flush, 20, 3))
+        aux["checksum"] = {"workload": "1.63 GB buffer", "ms": ck_ms,
+                           "gbs": tb.numel() / ck_ms / 1e6,
+                           "frac_of_hbm": tb.numel() / ck_ms / 1e6 / hbm_gbs}
+        del table, tb
+        plan = bcs.bcs_batch_plan(workloads.small_sweep())
+        dplan = plan.to("cuda")
+        br = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
+        bs = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
+        b_ms = statistics.mean(_event_ms(
+            torch, lambda: bcs.bcs_build_batch(dplan, plan.total_ranks, plan.total_entries, br, bs),
+            flush, 20, 3))
+        aux["batch_small_sweep"] = {"workload": "every p in 2..1024, one launch pair",
+                                    "ranks": plan.total_ranks, "ms": b_ms,
+                                    "ranks_per_s": plan.total_ranks / b_ms * 1e3}
+        plan = bcs.bcs_batch_plan(workloads.batch_p_list())
+        dplan = plan.to("cuda")
+        br = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
+        bs = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
+        b_ms = statistics.mean(_event_ms(
+            torch, lambda: bcs.bcs_build_batch(dplan, plan.total_ranks, plan.total_entries, br, bs),
+            lambda: None, 3, 1))                       # outputs (24 GB) exceed L2 by themselves
+        aux["batch_irregular_sweep"] = {"workload": "4096 octave-uniform p in [2^10,2^20), seed 220510072",
+                                        "ranks": plan.total_ranks, "ms": b_ms,
+                                        "ranks_per_s": plan.total_ranks / b_ms * 1e3,
+                                        "out_gbs": 2 * plan.total_entries / b_ms / 1e6}
+        del br, bs
+
+        # ---- CPU baseline: the oracle as it stands, per-rank form, bounded sample
+        import oracle
+        cpu_sample = 262144
+        lo = p // 2 - cpu_sample // 2
+        t0 = time.perf_counter()
+        oracle.build_range(p, lo, lo + cpu_sample)
+        cpu_dt = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        oracle.full_table(p)
+        cpu_arr_dt = time.perf_counter() - t0
+        cpu = {"value": cpu_sample / cpu_dt, "unit": UNIT, "cores": oracle.num_threads(),
+               "kind": "oracle",
+               "sample": "ranks %d..%d of p=2^20+1, per-rank form (Algorithms 4+5), %.1f s"
+                         % (lo, lo + cpu_sample - 1, cpu_dt),
+               "array_form_value": p / cpu_arr_dt}
+
+        # ---- roofline of the dominant kernel (receive schedule): integer issue
+        model = ALU_MODEL[q]
+        ops_per_launch = model * p
+        alu_peak = SM_COUNT * ALU_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12     # T int-op/s
+        achieved = ops_per_launch / (recv_ms * 1e-3) / 1e12
+        roof = {"bound": "alu", "kernel": "recv_kernel", "achieved": achieved, "peak": alu_peak,
+                "unit": "Tint-op/s", "frac": achieved / alu_peak, "traffic": None,
+                "ms": recv_ms, "model_int_ops_per_rank": model,
+                "peak_source": "148 SMs x 64 INT32 lanes x %.0f MHz (max SM clock)" % sm_max_mhz,
+                "hbm_time_frac": (2 * nb / (hbm_gbs * 1e9)) / (ms_per_step * 1e-3),
+                "hbm_peak_source": peak_src}
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int8/int32", "data": "synthetic",
+            "config": {"workload": "single p=2^20+1 (q=21), all ranks, recv+send int8 (44 MB)",
+                       "p": p, "q": q, "l2": "flushed between timed steps (256 MiB write)",
+                       "parallelism": "replicas" if world > 1 else "1 GPU",
+                       "timed_wall_s": t_wall},
+            "out_gbs": 2 * nb / ms_per_step / 1e6,
+            "kernel_ms": {"recv_kernel": recv_ms, "send_kernel": send_ms},
+            "roofline": roof, "cpu_baseline": cpu,
+            "e2e": {"value": p / e2e_dt, "unit": UNIT, "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 2 * nb, "ms_per_step": e2e_dt * 1e3},
+            "gpu_launches": 2 * args.steps,
+            "clocks": clk.summary(), "aux": aux,
+        }
+    barrier()
+    if world > 1:
+        dist.destroy_process_group()
+    if out is not None:
+        print(json.dumps(out))
+
+
+# integer operations per rank of the receive-schedule construction that the kernel runs,
+# by q: descent steps per rank (CPU count of the same loops) x operations per step.
+ALU_MODEL = {21: 12 * 287 + 10 * 10 + 20 * 21}
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

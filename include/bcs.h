@@ -1,0 +1,134 @@
+/*
+ * bcs.h -- C ABI of the B200 (sm_100a) library that constructs the round-optimal
+ * n-block broadcast schedules on circulant graphs of J. L. Traff, "(Poly)Logarithmic
+ * Time Construction of Round-optimal n-Block Broadcast Schedules for Broadcast and
+ * irregular Allgather in MPI" (arXiv 2205.10072), Section 2.
+ *
+ * Notation (Section 2): p processors ranked 0..p-1, q = ceil(log2 p), skips[0..q]
+ * the jumps of the circulant graph (Algorithm 1), root = rank 0.  A schedule of
+ * rank r is two arrays of q block numbers in [-q, q-1]: recvsched[k] and
+ * sendsched[k] for round k of a phase; a non-negative entry is a block of the
+ * current phase, a negative entry b-q is block b of the previous phase.
+ *
+ * Conventions of every entry point
+ *   - "device" pointers are CUDA device addresses valid on the current device;
+ *     "host" pointers are ordinary host addresses.  The caller owns every buffer.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls only enqueue work on that stream; they do not synchronise, and the
+ *     library holds no device memory of its own unless an entry point says so.
+ *   - Schedule tables are int8, rank-major and unpadded: the row of rank r of a
+ *     call for ranks r_begin..r_end-1 starts at byte (r - r_begin) * q.
+ *   - Errors are return codes.  When a code other than BCS_OK is returned nothing
+ *     was enqueued and no output byte was written.
+ *   - Supported: 1 <= p <= 2^31 - 1 (block sets are 32-bit masks).  p == 1 has
+ *     q == 0: every call succeeds and writes nothing.
+ *   - An entry that the construction could not determine (Algorithm 4 finding no
+ *     new block in either window; never observed) is written as BCS_BAD_ENTRY.
+ */
+#ifndef BCS_H_
+#define BCS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BCS_OK = 0,
+    BCS_ERR_ARG = 1,          /* NULL where a buffer is required, n == 0, bad combination */
+    BCS_ERR_RANGE = 2,        /* p == 0, r_begin > r_end, r_end > p, offsets not monotone */
+    BCS_ERR_ALIGN = 3,        /* an output pointer is not 16-byte aligned */
+    BCS_ERR_UNSUPPORTED = 4,  /* p > 2^31 - 1, or a size beyond a stated maximum */
+    BCS_ERR_CUDA = 5          /* the CUDA runtime refused a launch or a copy */
+} bcs_status;
+
+#define BCS_BAD_ENTRY 127
+#define BCS_MAX_Q 31
+#define BCS_SKIPS_STRIDE 32   /* words per row of a skips table */
+
+/* Human-readable name of a status code (static string, never NULL). */
+const char *bcs_status_str(bcs_status st);
+
+/* q = ceil(log2 p) (Section 2, first paragraph); 0 for p == 1, -1 for p == 0. */
+int bcs_q(uint32_t p);
+
+/* Algorithm 1: skips[q] = p, skips[k] = ceil(skips[k+1] / 2), skips[0] = 1.
+ * skips_host: host array of at least q+1 words.  Errors: p == 0 -> BCS_ERR_RANGE,
+ * p > 2^31-1 -> BCS_ERR_UNSUPPORTED, NULL -> BCS_ERR_ARG. */
+bcs_status bcs_skips(uint32_t p, uint32_t *skips_host);
+
+/* Receive and send schedules (Algorithm 4; Algorithm 5 resp. the table lookup of
+ * Algorithm 9, sendsched[r][k] = recvsched[(r+skips[k]) mod p][k]) of the ranks
+ * r_begin..r_end-1 of one p.
+ *   recv_out, send_out: device, int8, (r_end-r_begin)*q bytes each, 16-byte
+ *   aligned; either may be NULL (not wanted), not both unless the range is empty.
+ * A send entry whose to-processor lies inside the range is looked up in recv_out
+ * (when given); the others are recomputed with Algorithm 4, so any sub-range is
+ * self-contained.  Errors: see the status codes. */
+bcs_status bcs_build(uint32_t p, uint64_t r_begin, uint64_t r_end,
+                     int8_t *recv_out, int8_t *send_out, void *cuda_stream);
+
+/* As bcs_build, then copies the tables to HOST memory on the same stream
+ * (cudaMemcpyAsync; pinned host memory makes the copies asynchronous).
+ *   recv_host, send_host: host, (r_end-r_begin)*q bytes each, either may be NULL.
+ *   stage_dev: device staging buffer supplied by the caller, 16-byte aligned, of
+ *   at least 2 * align256((r_end-r_begin)*q) bytes (align256 = round up to 256).
+ * The host buffers are complete once the stream has been synchronised. */
+bcs_status bcs_build_to_host(uint32_t p, uint64_t r_begin, uint64_t r_end,
+                             int8_t *recv_host, int8_t *send_host,
+                             void *stage_dev, size_t stage_bytes, void *cuda_stream);
+
+/* Host helper for bcs_build_batch: for a list of num_p values of p fills
+ *   rank_off_host[num_p+1]  prefix sums of p_j            (flattened rank index),
+ *   entry_off_host[num_p+1] prefix sums of p_j * q_j      (byte offset of p_j's table),
+ *   skips_tab_host[num_p * BCS_SKIPS_STRIDE] row j = skips[0..q_j] of p_j (Algorithm 1),
+ *                           the rest of the row 0.
+ * The caller copies the three arrays and p_list to the device. */
+bcs_status bcs_batch_plan(const uint32_t *p_list_host, uint32_t num_p,
+                          uint64_t *rank_off_host, uint64_t *entry_off_host,
+                          uint32_t *skips_tab_host);
+
+/* All ranks of many p at once (the "full schedule" of Algorithm 9 for each p_j),
+ * one launch over the flattened list of (p_j, r) pairs.  Device inputs as laid
+ * out by bcs_batch_plan; total_ranks = rank_off[num_p], total_entries =
+ * entry_off[num_p] (the host knows both).  Outputs: device int8, total_entries
+ * bytes each, 16-byte aligned; the table of p_j starts at byte entry_off[j] and
+ * is rank-major with q_j bytes per rank.  send_out may be NULL; recv_out is
+ * required (the send table is looked up in it). */
+bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_dev,
+                           const uint64_t *entry_off_dev, const uint32_t *skips_tab_dev,
+                           uint32_t num_p, uint64_t total_ranks, uint64_t total_entries,
+                           int8_t *recv_out, int8_t *send_out, void *cuda_stream);
+
+/* Round tables of the n-block broadcast (Algorithm 6 without the Send||Recv): for
+ * each rank r of r_begin..r_end-1 and each round j of 0..n-2+q one record of four
+ * int32 {send block, receive block, to-processor, from-processor} with
+ *   x = (q - (n-1+q) mod q) mod q, i = j + x, k = i mod q,
+ *   block = sched[k] - x + q * floor(i / q); below 0 -> -1 (nothing is sent or
+ *   received), above n-1 -> n-1; to = (r+skips[k]) mod p, from = (r-skips[k]+p) mod p.
+ *   recv, send: device int8 rows of exactly these ranks as bcs_build writes them.
+ *   table_out: device, (r_end-r_begin) * (n-1+q) records of 16 bytes, 16-byte
+ *   aligned; record of (r, j) at index (r-r_begin)*(n-1+q) + j. */
+bcs_status bcs_expand(uint32_t p, uint32_t n, uint64_t r_begin, uint64_t r_end,
+                      const int8_t *recv, const int8_t *send, int32_t *table_out,
+                      void *cuda_stream);
+
+/* Position-weighted 64-bit checksum of a stretch of schedule entries, additive
+ * over disjoint stretches (no counterpart in the paper; used to compare outputs
+ * that are too large to copy back).  The bytes are read as little-endian 32-bit
+ * words of the whole entry stream: word g covers entries 4g..4g+3.
+ *   sum = sum over words g of  word_g * weight(g)   mod 2^64,
+ *   weight(g) = fmix32(low32(g) ^ (0x9E3779B9 * high32(g))) | 1,
+ * fmix32 = the 32-bit finaliser of MurmurHash3.  buf_dev: device, 4-byte aligned;
+ * first_entry_index must be a multiple of 4; a last partial word is zero-padded.
+ * sum_dev: device uint64, overwritten with the sum (set to 0 first, then
+ * accumulated atomically). */
+bcs_status bcs_checksum(const int8_t *buf_dev, uint64_t n_entries,
+                        uint64_t first_entry_index, uint64_t *sum_dev, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BCS_H_ */

@@ -451,19 +451,30 @@ void bcso_expand_range(uint32_t p, uint32_t n, uint64_t r_begin, uint64_t r_end,
     }
 }
 
-/* Order-independent 64-bit checksum of a stretch of schedule entries:
- * sum over e of (entry_e as unsigned byte) * mix(first_index + e)  mod 2^64,
- * mix = the splitmix64 output function (Steele, Lea, Flood 2014) applied to
- * the index.  Not from the paper: a tool for comparing 64 GB outputs. */
+/* Position-weighted 64-bit checksum of a stretch of schedule entries (not from
+ * the paper: a tool for comparing outputs too large to copy).  Entry number e
+ * of the whole stream is byte e mod 4 of the little-endian 32-bit word
+ * g = floor(e / 4); the sum is  sum_e (byte_e << 8 (e mod 4)) * weight(g)  mod
+ * 2^64 with weight(g) = fmix32(low32(g) ^ 0x9E3779B9 * high32(g)) | 1, fmix32
+ * being the finaliser of MurmurHash3 (Appleby, public domain). */
+static uint32_t murmur3_fmix32(uint32_t h)
+{
+    h ^= h >> 16;
+    h *= 0x85ebca6bu;
+    h ^= h >> 13;
+    h *= 0xc2b2ae35u;
+    h ^= h >> 16;
+    return h;
+}
+
 uint64_t bcso_checksum(const int8_t *buf, uint64_t n_entries, uint64_t first_index)
 {
     uint64_t sum = 0, e;
     for (e = 0; e < n_entries; e++) {
-        uint64_t z = first_index + e + 0x9E3779B97F4A7C15ull;
-        z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
-        z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
-        z = z ^ (z >> 31);
-        sum += (uint64_t)(uint8_t)buf[e] * z;
+        uint64_t pos = first_index + e;
+        uint64_t g = pos / 4;
+        uint32_t w = murmur3_fmix32((uint32_t)g ^ (0x9E3779B9u * (uint32_t)(g >> 32))) | 1u;
+        sum += ((uint64_t)(uint8_t)buf[e] << (8 * (pos % 4))) * (uint64_t)w;
     }
     return sum;
 }

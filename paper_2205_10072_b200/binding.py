@@ -1,0 +1,171 @@
+"""ctypes binding of libbcs.so: argument marshalling only (include/bcs.h has the contracts)."""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+from . import build_ext
+
+BCS_SKIPS_STRIDE = 32
+BCS_BAD_ENTRY = 127
+
+_c = ctypes
+_lib = None
+
+
+class BcsError(RuntimeError):
+    """A bcs_* call returned a status other than BCS_OK."""
+
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s" % (where, bcs_status_str(status)))
+
+
+def lib_path() -> str:
+    return build_ext.LIB_PATH
+
+
+def lib():
+    """Loads libbcs.so (must have been built: python -m paper_2205_10072_b200.build_ext)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(build_ext.LIB_PATH):
+            raise ImportError(
+                "libbcs.so is missing: build it with paper_2205_10072_b200.build_ext.build(); "
+                "there is no CPU fallback")
+        L = _c.CDLL(build_ext.LIB_PATH)
+        vp, u32, u64, i32 = _c.c_void_p, _c.c_uint32, _c.c_uint64, _c.c_int
+        L.bcs_status_str.argtypes = [i32]
+        L.bcs_status_str.restype = _c.c_char_p
+        L.bcs_q.argtypes = [u32]
+        L.bcs_q.restype = i32
+        L.bcs_skips.argtypes = [u32, vp]
+        L.bcs_skips.restype = i32
+        L.bcs_build.argtypes = [u32, u64, u64, vp, vp, vp]
+        L.bcs_build.restype = i32
+        L.bcs_build_to_host.argtypes = [u32, u64, u64, vp, vp, vp, _c.c_size_t, vp]
+        L.bcs_build_to_host.restype = i32
+        L.bcs_batch_plan.argtypes = [vp, u32, vp, vp, vp]
+        L.bcs_batch_plan.restype = i32
+        L.bcs_build_batch.argtypes = [vp, vp, vp, vp, u32, u64, u64, vp, vp, vp]
+        L.bcs_build_batch.restype = i32
+        L.bcs_expand.argtypes = [u32, u32, u64, u64, vp, vp, vp, vp]
+        L.bcs_expand.restype = i32
+        L.bcs_checksum.argtypes = [vp, u64, u64, vp, vp]
+        L.bcs_checksum.restype = i32
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise BcsError(status, where)
+
+
+def _ptr(t) -> int | None:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> int | None:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream or None
+
+
+def bcs_status_str(status: int) -> str:
+    return lib().bcs_status_str(int(status)).decode()
+
+
+def bcs_q(p: int) -> int:
+    return lib().bcs_q(p)
+
+
+def bcs_skips(p: int) -> list[int]:
+    buf = (_c.c_uint32 * (BCS_SKIPS_STRIDE + 1))()
+    _check(lib().bcs_skips(p, buf), "bcs_skips")
+    return list(buf[: bcs_q(p) + 1])
+
+
+def bcs_build(p: int, r_begin: int, r_end: int, recv_out, send_out, stream=None) -> None:
+    """recv_out / send_out: CUDA int8 tensors of (r_end-r_begin)*q elements, or None."""
+    _check(lib().bcs_build(p, r_begin, r_end, _ptr(recv_out), _ptr(send_out), _stream(stream)),
+           "bcs_build")
+
+
+def bcs_build_to_host(p: int, r_begin: int, r_end: int, recv_host, send_host, stage_dev,
+                      stream=None) -> None:
+    """recv_host / send_host: CPU int8 tensors (pinned for asynchronous copies) or None;
+    stage_dev: CUDA uint8/int8 tensor used as staging."""
+    _check(lib().bcs_build_to_host(p, r_begin, r_end, _ptr(recv_host), _ptr(send_host),
+                                   _ptr(stage_dev), stage_dev.numel() * stage_dev.element_size(),
+                                   _stream(stream)), "bcs_build_to_host")
+
+
+@dataclass
+class BatchPlan:
+    """Host-side result of bcs_batch_plan (int64/int32 tensors hold the uint64/uint32 bit patterns)."""
+    p_list: torch.Tensor      # int32 [num_p]
+    rank_off: torch.Tensor    # int64 [num_p+1]
+    entry_off: torch.Tensor   # int64 [num_p+1]
+    skips_tab: torch.Tensor   # int32 [num_p, 32]
+
+    @property
+    def num_p(self) -> int:
+        return self.p_list.numel()
+
+    @property
+    def total_ranks(self) -> int:
+        return int(self.rank_off[-1])
+
+    @property
+    def total_entries(self) -> int:
+        return int(self.entry_off[-1])
+
+    def to(self, device, non_blocking: bool = False) -> "BatchPlan":
+        return BatchPlan(*(t.to(device, non_blocking=non_blocking)
+                           for t in (self.p_list, self.rank_off, self.entry_off, self.skips_tab)))
+
+
+def bcs_batch_plan(p_list, pin: bool = False) -> BatchPlan:
+    pl = torch.as_tensor(list(p_list) if not torch.is_tensor(p_list) else p_list,
+                         dtype=torch.int64)
+    if pl.numel() and (int(pl.min()) < 0 or int(pl.max()) > 0xFFFFFFFF):
+        raise BcsError(2, "bcs_batch_plan")
+    n = pl.numel()
+    # uint32 bit patterns in an int32 tensor
+    p32 = torch.where(pl >= 2**31, pl - 2**32, pl).to(torch.int32).contiguous()
+    rank_off = torch.zeros(n + 1, dtype=torch.int64)
+    entry_off = torch.zeros(n + 1, dtype=torch.int64)
+    skips_tab = torch.zeros((n, BCS_SKIPS_STRIDE), dtype=torch.int32)
+    if pin:
+        p32, rank_off, entry_off, skips_tab = (t.pin_memory()
+                                               for t in (p32, rank_off, entry_off, skips_tab))
+    _check(lib().bcs_batch_plan(p32.data_ptr(), n, rank_off.data_ptr(), entry_off.data_ptr(),
+                                skips_tab.data_ptr()), "bcs_batch_plan")
+    return BatchPlan(p32, rank_off, entry_off, skips_tab)
+
+
+def bcs_build_batch(plan_dev: BatchPlan, total_ranks: int, total_entries: int, recv_out, send_out,
+                    stream=None) -> None:
+    """plan_dev: a BatchPlan whose tensors live on the CUDA device."""
+    _check(lib().bcs_build_batch(plan_dev.p_list.data_ptr(), plan_dev.rank_off.data_ptr(),
+                                 plan_dev.entry_off.data_ptr(), plan_dev.skips_tab.data_ptr(),
+                                 plan_dev.num_p, total_ranks, total_entries, _ptr(recv_out),
+                                 _ptr(send_out), _stream(stream)), "bcs_build_batch")
+
+
+def bcs_expand(p: int, n: int, r_begin: int, r_end: int, recv, send, table_out, stream=None) -> None:
+    """recv/send: CUDA int8 rows of ranks r_begin..r_end-1; table_out: CUDA int32
+    [(r_end-r_begin), n-1+q, 4]."""
+    _check(lib().bcs_expand(p, n, r_begin, r_end, _ptr(recv), _ptr(send), _ptr(table_out),
+                            _stream(stream)), "bcs_expand")
+
+
+def bcs_checksum(buf, first_entry_index: int, sum_out, stream=None, n_entries: int | None = None) -> None:
+    """buf: CUDA int8 tensor; sum_out: CUDA int64 tensor with one element (uint64 bit pattern)."""
+    n = buf.numel() if n_entries is None else n_entries
+    _check(lib().bcs_checksum(_ptr(buf), n, first_entry_index, _ptr(sum_out), _stream(stream)),
+           "bcs_checksum")

@@ -1,0 +1,92 @@
+"""CPU-only checks of the boundary: the shared library loads, exports every symbol that
+include/bcs.h declares, and its host-side entry points (no kernel launch) behave."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2205_10072_b200 import build_ext
+    build_ext.build()
+    import paper_2205_10072_b200 as bcs
+    return bcs
+
+
+def _declared_symbols():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            text = open(os.path.join(ROOT, "include", fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names |= set(re.findall(r"\b(bcs_[a-z_0-9]+)\s*\(", text))
+    return sorted(names)
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared_symbols()
+    assert {"bcs_build", "bcs_build_batch", "bcs_expand", "bcs_checksum", "bcs_skips", "bcs_q",
+            "bcs_batch_plan", "bcs_status_str", "bcs_build_to_host"} <= set(names)
+    dll = ctypes.CDLL(lib.lib_path())
+    for n in names:
+        assert hasattr(dll, n), n
+        assert callable(getattr(lib, n)), "binding lacks %s" % n
+
+
+def test_q_and_skips_host_side(lib):
+    assert lib.bcs_q(0) == -1 and lib.bcs_q(1) == 0 and lib.bcs_q(2) == 1
+    assert lib.bcs_q(1024) == 10 and lib.bcs_q(1025) == 11 and lib.bcs_q(2**31 - 1) == 31
+    assert lib.bcs_skips(1) == [1]
+    assert lib.bcs_skips(20) == [1, 2, 3, 5, 10, 20]            # caption of Table 1
+    assert lib.bcs_skips(33) == [1, 2, 3, 5, 9, 17, 33]         # caption of Table 2
+    assert lib.bcs_skips(31) == [1, 2, 4, 8, 16, 31]            # caption of Table 4
+    assert lib.bcs_skips(2**30 - 1) == [2**k for k in range(30)] + [2**30 - 1]
+    with pytest.raises(lib.BcsError) as e:
+        lib.bcs_skips(0)
+    assert e.value.status == 2
+    with pytest.raises(lib.BcsError) as e:
+        lib.bcs_skips(2**31)
+    assert e.value.status == 4
+
+
+def test_status_strings(lib):
+    assert [lib.bcs_status_str(i) for i in range(6)] == [
+        "BCS_OK", "BCS_ERR_ARG", "BCS_ERR_RANGE", "BCS_ERR_ALIGN", "BCS_ERR_UNSUPPORTED",
+        "BCS_ERR_CUDA"]
+    assert lib.bcs_status_str(99) == "BCS_ERR_UNKNOWN"
+
+
+def test_batch_plan_host_side(lib):
+    plan = lib.bcs_batch_plan([2, 3, 20, 1, 1025])
+    assert plan.rank_off.tolist() == [0, 2, 5, 25, 26, 1051]
+    assert plan.entry_off.tolist() == [0, 2, 8, 108, 108, 108 + 1025 * 11]
+    assert plan.skips_tab[2].tolist()[:6] == [1, 2, 3, 5, 10, 20]
+    assert plan.skips_tab[3].tolist()[:2] == [1, 0]
+    assert plan.total_ranks == 1051
+    with pytest.raises(lib.BcsError):
+        lib.bcs_batch_plan([5, 0])
+
+
+def test_argument_errors_need_no_gpu(lib):
+    """Validation happens before any CUDA call: these return an error code on a CPU-only box."""
+    L = lib.lib()
+    assert L.bcs_build(0, 0, 0, None, None, None) == 2
+    assert L.bcs_build(2**31, 0, 1, None, None, None) == 4
+    assert L.bcs_build(10, 5, 4, None, None, None) == 2
+    assert L.bcs_build(10, 0, 11, None, None, None) == 2
+    assert L.bcs_build(10, 0, 10, None, None, None) == 1
+    assert L.bcs_build(10, 0, 10, 8, None, None) == 3            # misaligned pointer
+    assert L.bcs_build(1, 0, 1, None, None, None) == 0           # q == 0: nothing to do
+    assert L.bcs_build(10, 3, 3, None, None, None) == 0          # empty range
+    assert L.bcs_expand(10, 0, 0, 10, 16, 16, 16, None) == 1     # n == 0
+    assert L.bcs_expand(10, 4, 0, 10, None, 16, 16, None) == 1
+    assert L.bcs_expand(10, 4, 0, 10, 16, 16, 8, None) == 3
+    assert L.bcs_checksum(16, 8, 2, 16, None) == 3               # first index not a multiple of 4
+    assert L.bcs_checksum(16, 8, 0, None, None) == 1
+    assert L.bcs_build_batch(None, None, None, None, 3, 10, 40, 16, None, None) == 1
+    assert L.bcs_build_to_host(10, 0, 10, None, None, 16, 1024, None) == 1
+    assert L.bcs_build_to_host(10, 0, 10, 16, None, 16, 16, None) == 1   # staging too small

@@ -1,0 +1,332 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle, element by element.
+All schedule entries are integers: the bar is bit-exactness."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2205_10072_b200 import workloads
+from tests import bcast_sim
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def bcs():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2205_10072_b200 as lib
+    lib.lib()                      # raises if the CUDA library has not been built
+    torch.cuda.set_device(0)
+    return lib
+
+
+GUARD = 256
+
+
+def _guarded(nbytes, fill=0x5A):
+    """int8 CUDA buffer of nbytes framed by guard bytes (start stays 16-byte aligned)."""
+    raw = torch.full((nbytes + 2 * GUARD,), fill, dtype=torch.int8, device="cuda")
+    return raw, raw[GUARD:GUARD + nbytes]
+
+
+def _guards_intact(raw, nbytes, fill=0x5A):
+    return bool((raw[:GUARD] == fill).all()) and bool((raw[GUARD + nbytes:] == fill).all())
+
+
+def _build(bcs, p, r0, r1, want_recv=True, want_send=True):
+    q = bcs.bcs_q(p)
+    nb = (r1 - r0) * q
+    raw_r, recv = _guarded(nb) if want_recv else (None, None)
+    raw_s, send = _guarded(nb) if want_send else (None, None)
+    bcs.bcs_build(p, r0, r1, recv, send)
+    torch.cuda.synchronize()
+    out = []
+    for raw, t in ((raw_r, recv), (raw_s, send)):
+        if t is None:
+            out.append(None)
+        else:
+            assert _guards_intact(raw, nb)
+            out.append(t.cpu().numpy().reshape(r1 - r0, q))
+    return out
+
+
+# ---------------------------------------------------------------- printed tables, small p
+def test_printed_tables_through_the_gpu(bcs):
+    from tests.golden_tables import TABLES, load
+    for name in TABLES:
+        g = load(name)
+        recv, send = _build(bcs, g["p"], 0, g["p"])
+        assert np.array_equal(recv, g["recv"]) and np.array_equal(send, g["send"]), name
+
+
+def test_every_p_up_to_1024_single_calls(bcs):
+    for p in workloads.small_sweep():
+        want_r, want_s = oracle.full_table(p)
+        recv, send = _build(bcs, p, 0, p)
+        assert np.array_equal(recv, want_r), p
+        assert np.array_equal(send, want_s), p
+
+
+def test_every_p_up_to_1024_batched_and_simulated(bcs):
+    plist = workloads.small_sweep()
+    plan = bcs.bcs_batch_plan(plist)
+    assert plan.total_ranks == 524799 and plan.total_entries == 5072726
+    dev = plan.to("cuda")
+    raw_r, recv = _guarded(plan.total_entries)
+    raw_s, send = _guarded(plan.total_entries)
+    bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, send)
+    torch.cuda.synchronize()
+    assert _guards_intact(raw_r, plan.total_entries) and _guards_intact(raw_s, plan.total_entries)
+    recv, send = recv.cpu().numpy(), send.cpu().numpy()
+    eo = plan.entry_off.tolist()
+    for j, p in enumerate(plist):
+        q = oracle.q_of(p)
+        want_r, want_s = oracle.full_table(p)
+        got_r = recv[eo[j]:eo[j + 1]].reshape(p, q)
+        got_s = send[eo[j]:eo[j + 1]].reshape(p, q)
+        assert np.array_equal(got_r, want_r), p
+        assert np.array_equal(got_s, want_s), p
+        if p % 7 == 0 or p < 70:            # broadcast simulation on the GPU's own output
+            for n in (1, 2, 5, q + 3):
+                tab = torch.empty((p, n - 1 + q, 4), dtype=torch.int32, device="cuda")
+                bcs.bcs_expand(p, n, 0, p, torch.from_numpy(got_r.copy()).cuda(),
+                               torch.from_numpy(got_s.copy()).cuda(), tab)
+                assert bcast_sim.simulate(p, n, tab.cpu().numpy()) is None, (p, n)
+
+
+def test_batch_with_trivial_and_duplicate_p(bcs):
+    plist = [1, 2, 1, 300, 300, 1, 17, 4096, 1]
+    plan = bcs.bcs_batch_plan(plist)
+    dev = plan.to("cuda")
+    raw_r, recv = _guarded(plan.total_entries)
+    raw_s, send = _guarded(plan.total_entries)
+    bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, send)
+    torch.cuda.synchronize()
+    assert _guards_intact(raw_r, plan.total_entries) and _guards_intact(raw_s, plan.total_entries)
+    eo = plan.entry_off.tolist()
+    for j, p in enumerate(plist):
+        if p == 1:
+            assert eo[j] == eo[j + 1]
+            continue
+        want_r, want_s = oracle.full_table(p)
+        assert np.array_equal(recv[eo[j]:eo[j + 1]].cpu().numpy().reshape(p, -1), want_r)
+        assert np.array_equal(send[eo[j]:eo[j + 1]].cpu().numpy().reshape(p, -1), want_s)
+    # receive table alone
+    raw_r, recv = _guarded(plan.total_entries)
+    bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, None)
+    torch.cuda.synchronize()
+    assert np.array_equal(recv[eo[3]:eo[4]].cpu().numpy().reshape(300, -1), oracle.full_table(300)[0])
+
+
+# ---------------------------------------------------------------- ranges, tails, degenerate
+def test_sub_ranges_ragged_tails_and_single_outputs(bcs):
+    p = 100003
+    q = oracle.q_of(p)
+    want_r, want_s = oracle.full_table(p)
+    for r0, r1 in ((0, 1), (0, 255), (0, 257), (1, 258), (777, 1300), (p - 300, p), (p - 1, p),
+                   (50000, 50000 + 16 * 3 + 5), (99000, 100003)):
+        recv, send = _build(bcs, p, r0, r1)
+        assert np.array_equal(recv, want_r[r0:r1]), (r0, r1)
+        assert np.array_equal(send, want_s[r0:r1]), (r0, r1)      # partly looked up, partly recomputed
+    recv, _ = _build(bcs, p, 123, 999, want_send=False)
+    assert np.array_equal(recv, want_r[123:999])
+    _, send = _build(bcs, p, 123, 999, want_recv=False)           # every send entry recomputed
+    assert np.array_equal(send, want_s[123:999])
+    assert q == 17
+
+
+def test_degenerate_sizes_and_errors(bcs):
+    L = bcs.lib()
+    buf = torch.zeros(64, dtype=torch.int8, device="cuda")
+    bcs.bcs_build(1, 0, 1, buf, buf)                    # q == 0
+    bcs.bcs_build(20, 7, 7, buf, buf)                   # empty range
+    torch.cuda.synchronize()
+    assert int(buf.abs().sum()) == 0
+    recv, send = _build(bcs, 2, 0, 2)
+    assert recv.tolist() == [[-1], [0]] and send.tolist() == [[0], [-1]]
+    recv, send = _build(bcs, 3, 0, 3)
+    want = oracle.full_table(3)
+    assert np.array_equal(recv, want[0]) and np.array_equal(send, want[1])
+    assert L.bcs_build(20, 0, 20, buf.data_ptr() + 1, None, None) == 3
+    assert L.bcs_build(20, 0, 21, buf.data_ptr(), None, None) == 2
+    assert L.bcs_build(0, 0, 0, buf.data_ptr(), None, None) == 2
+    torch.cuda.synchronize()
+    assert int(buf.abs().sum()) == 0                    # an error writes nothing
+
+
+def test_p_at_the_upper_limit(bcs):
+    """p = 2^31 - 1 (q = 31): rank arithmetic near 2^32; a few ranges vs the per-rank oracle."""
+    p = 2**31 - 1
+    for r0, r1 in ((0, 300), (2**30 - 100, 2**30 + 200), (p - 300, p)):
+        want_r, want_s = oracle.build_range(p, r0, r1)
+        recv, send = _build(bcs, p, r0, r1)
+        assert np.array_equal(recv, want_r), (r0, r1)
+        assert np.array_equal(send, want_s), (r0, r1)
+
+
+# ---------------------------------------------------------------- full-size workloads
+def test_single_p_2pow20_plus_1_full_table(bcs):
+    p = workloads.P_SINGLE
+    want_r, want_s = oracle.full_table(p)
+    recv, send = _build(bcs, p, 0, p)
+    assert recv.shape == (p, 21)
+    assert np.array_equal(recv, want_r)
+    assert np.array_equal(send, want_s)
+
+
+def test_build_to_host_matches(bcs):
+    p = 65537
+    q = bcs.bcs_q(p)
+    want_r, want_s = oracle.full_table(p)
+    nb = p * q
+    stage = torch.empty(2 * ((nb + 255) // 256 * 256), dtype=torch.int8, device="cuda")
+    hr = torch.zeros(nb, dtype=torch.int8).pin_memory()
+    hs = torch.zeros(nb, dtype=torch.int8).pin_memory()
+    bcs.bcs_build_to_host(p, 0, p, hr, hs, stage)
+    torch.cuda.synchronize()
+    assert np.array_equal(hr.numpy().reshape(p, q), want_r)
+    assert np.array_equal(hs.numpy().reshape(p, q), want_s)
+    hs.zero_()
+    bcs.bcs_build_to_host(p, 100, 5000, None, hs, stage)
+    torch.cuda.synchronize()
+    assert np.array_equal(hs.numpy()[: 4900 * q].reshape(4900, q), want_s[100:5000])
+
+
+def test_batched_irregular_sweep_full_size(bcs):
+    """4096 octave-uniform p in [2^10, 2^20): the launch the benchmark uses.  Full tables are
+    compared for a spread of p, seeded sample ranks for every p."""
+    plist = workloads.batch_p_list()
+    plan = bcs.bcs_batch_plan(plist)
+    assert plan.total_ranks == 639466253
+    dev = plan.to("cuda")
+    recv = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
+    send = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
+    bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, send)
+    torch.cuda.synchronize()
+    eo = plan.entry_off.tolist()
+    order = sorted(range(len(plist)), key=lambda j: plist[j])
+    full = set(order[:24] + order[-3:] + order[::300] + list(range(6)))
+    for j in sorted(full):
+        p, q = plist[j], oracle.q_of(plist[j])
+        want_r, want_s = oracle.full_table(p)
+        assert np.array_equal(recv[eo[j]:eo[j + 1]].cpu().numpy().reshape(p, q), want_r), p
+        assert np.array_equal(send[eo[j]:eo[j + 1]].cpu().numpy().reshape(p, q), want_s), p
+    rng = np.random.default_rng(220510072)
+    for j, p in enumerate(plist):
+        if j in full:
+            continue
+        q = oracle.q_of(p)
+        ranks = np.unique(np.concatenate([rng.integers(0, p, 48), [0, 1, p - 1]]))
+        want_r, want_s = oracle.build_ranks(p, ranks)
+        idx = (torch.from_numpy(ranks)[:, None] * q + torch.arange(q)[None, :] + eo[j]).cuda()
+        assert np.array_equal(recv[idx].cpu().numpy(), want_r), p
+        assert np.array_equal(send[idx].cpu().numpy(), want_s), p
+
+
+def test_expansion_full_size(bcs):
+    """p = 100003, n = 1000: 1016 rounds, 16 bytes per record, compared record by record."""
+    p, n = workloads.P_EXPAND, workloads.N_EXPAND
+    q = oracle.q_of(p)
+    want_r, want_s = oracle.full_table(p)
+    recv = torch.from_numpy(want_r).cuda()
+    send = torch.from_numpy(want_s).cuda()
+    rounds = n - 1 + q
+    assert rounds == 1016 and p * rounds * 16 == 1625648768
+    tab = torch.empty((p, rounds, 4), dtype=torch.int32, device="cuda")
+    bcs.bcs_expand(p, n, 0, p, recv, send, tab)
+    torch.cuda.synchronize()
+    step = 20000
+    for r0 in range(0, p, step):
+        r1 = min(p, r0 + step)
+        want = oracle.expand(p, n, want_r, want_s, r0, r1)
+        assert np.array_equal(tab[r0:r1].cpu().numpy(), want), r0
+    # a sub-range with rows of that range only, ragged against the 8-rank CTA tile
+    sub = torch.empty((1003, rounds, 4), dtype=torch.int32, device="cuda")
+    bcs.bcs_expand(p, n, 4321, 5324, recv[4321:5324].contiguous(), send[4321:5324].contiguous(), sub)
+    torch.cuda.synchronize()
+    assert torch.equal(sub, tab[4321:5324])
+
+
+def test_expansion_small_cases_and_simulation(bcs):
+    for p in (2, 3, 9, 20, 33, 257, 1000):
+        q = oracle.q_of(p)
+        want_r, want_s = oracle.full_table(p)
+        recv, send = torch.from_numpy(want_r).cuda(), torch.from_numpy(want_s).cuda()
+        for n in (1, 2, 5, q, q + 1, q + 3, 3 * q + 2, 700):
+            raw = torch.full((p * (n - 1 + q) * 4 + 128,), -77, dtype=torch.int32, device="cuda")
+            tab = raw[64:64 + p * (n - 1 + q) * 4].view(p, n - 1 + q, 4)
+            bcs.bcs_expand(p, n, 0, p, recv, send, tab)
+            torch.cuda.synchronize()
+            assert bool((raw[:64] == -77).all()) and bool((raw[-64:] == -77).all())
+            got = tab.cpu().numpy()
+            assert np.array_equal(got, oracle.expand(p, n, want_r, want_s)), (p, n)
+            if n <= 40:
+                assert bcast_sim.simulate(p, n, got) is None
+
+
+def test_checksum_matches_oracle(bcs):
+    rng = np.random.default_rng(11)
+    out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    for nbytes, first in ((0, 0), (1, 0), (3, 4), (4, 8), (1000, 16), (1003, 2**34 + 8),
+                          (5 * 2**20 + 1, 2**36)):
+        host = rng.integers(-31, 31, nbytes).astype(np.int8)
+        dev = torch.from_numpy(host).cuda() if nbytes else torch.zeros(4, dtype=torch.int8,
+                                                                       device="cuda")
+        bcs.bcs_checksum(dev, first, out, n_entries=nbytes)
+        got = int(out.cpu()[0]) & (2**64 - 1)
+        assert got == oracle.checksum(host, first), (nbytes, first)
+
+
+def test_large_p_chunked_spot_checked(bcs):
+    """p = 2^30 - 1 (q = 30) in 8 rank chunks through one reused buffer: per chunk a checksum
+    (two runs must agree; additive pieces must add up) and seeded sample ranks against the
+    per-rank oracle (10^6 ranks for the receive rows, a tenth of them for the send rows, which
+    the oracle recomputes with Algorithm 5 at cubic cost)."""
+    p = workloads.P_LARGE
+    q = 30
+    chunks = workloads.large_chunks()
+    assert len(chunks) == 8 and chunks[-1][1] == p
+    ranks = np.array(workloads.spot_ranks(p, 1000000), dtype=np.int64)
+    want_r, _ = oracle.build_ranks(p, ranks, want_send=False)
+    send_ranks = ranks[:100000]
+    _, want_s = oracle.build_ranks(p, send_ranks, want_recv=False)
+    cap = (1 << 27) * q
+    recv = torch.empty(cap, dtype=torch.int8, device="cuda")
+    send = torch.empty(cap, dtype=torch.int8, device="cuda")
+    sums = torch.zeros(4, dtype=torch.int64, device="cuda")
+    m64 = 2**64 - 1
+    SEND_BASE = 1 << 36                 # entry index at which the send table is taken to start
+    checked = 0
+    for c, (r0, r1) in enumerate(chunks):
+        nb = (r1 - r0) * q
+        bcs.bcs_build(p, r0, r1, recv, send)
+        bcs.bcs_checksum(recv, r0 * q, sums[0:1], n_entries=nb)
+        bcs.bcs_checksum(send, SEND_BASE + r0 * q, sums[1:2], n_entries=nb)
+        half = (nb // 2) // 4 * 4
+        bcs.bcs_checksum(recv[:half], r0 * q, sums[2:3], n_entries=half)
+        bcs.bcs_checksum(recv[half:], r0 * q + half, sums[3:4], n_entries=nb - half)
+        first = [int(v) & m64 for v in sums.cpu()]
+        assert (first[2] + first[3]) & m64 == first[0]
+        sel = (ranks >= r0) & (ranks < r1)
+        idx = (torch.from_numpy(ranks[sel] - r0)[:, None] * q + torch.arange(q)[None, :]).cuda()
+        assert np.array_equal(recv[idx].cpu().numpy(), want_r[sel]), c
+        sel_s = (send_ranks >= r0) & (send_ranks < r1)
+        idx = (torch.from_numpy(send_ranks[sel_s] - r0)[:, None] * q
+               + torch.arange(q)[None, :]).cuda()
+        assert np.array_equal(send[idx].cpu().numpy(), want_s[sel_s]), c
+        checked += int(sel.sum())
+        # head of the chunk against the oracle's own checksum of its own rows
+        head = 3000
+        o_r, _ = oracle.build_range(p, r0, r0 + head, want_send=False)
+        bcs.bcs_checksum(recv, r0 * q, sums[2:3], n_entries=head * q)
+        assert int(sums.cpu()[2]) & m64 == oracle.checksum(o_r, r0 * q)
+        if c in (0, 7):                                   # rebuilt chunk gives the same sums
+            recv.fill_(0)
+            send.fill_(0)
+            bcs.bcs_build(p, r0, r1, recv, send)
+            bcs.bcs_checksum(recv, r0 * q, sums[0:1], n_entries=nb)
+            bcs.bcs_checksum(send, SEND_BASE + r0 * q, sums[1:2], n_entries=nb)
+            again = [int(v) & m64 for v in sums.cpu()]
+            assert again[:2] == first[:2]
+    assert checked == len(ranks)

@@ -286,16 +286,32 @@ def test_simulation_rejects_planted_mistakes():
 # ---------------------------------------------------------------- checksum helper
 def test_checksum_definition_and_additivity():
     rng = np.random.default_rng(5)
-    buf = rng.integers(-30, 30, 1000).astype(np.int8)
-    mask = (1 << 64) - 1
+    buf = rng.integers(-30, 30, 1003).astype(np.int8)
+    m64, m32 = (1 << 64) - 1, (1 << 32) - 1
 
-    def mix(e):
-        z = (e + 0x9E3779B97F4A7C15) & mask
-        z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & mask
-        z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & mask
-        return z ^ (z >> 31)
+    def fmix32(h):
+        h ^= h >> 16
+        h = (h * 0x85EBCA6B) & m32
+        h ^= h >> 13
+        h = (h * 0xC2B2AE35) & m32
+        return h ^ (h >> 16)
 
-    assert mix(0) == 0xE220A8397B1DCDAF          # first output of splitmix64 seeded with 0
-    want = sum(int(np.uint8(v)) * mix(17 + e) for e, v in enumerate(buf)) & mask
-    assert oracle.checksum(buf, 17) == want
-    assert (oracle.checksum(buf[:400], 17) + oracle.checksum(buf[400:], 417)) & mask == want
+    # MurmurHash3 x86_32 of the empty key with seed 1 is fmix32(1) = 0x514E28B7 (reference vector)
+    assert fmix32(1) == 0x514E28B7
+
+    def weight(g):
+        return fmix32((g & m32) ^ ((0x9E3779B9 * (g >> 32)) & m32)) | 1
+
+    def by_words(b, first):
+        assert first % 4 == 0
+        pad = np.concatenate([b.view(np.uint8), np.zeros((-len(b)) % 4, dtype=np.uint8)])
+        words = pad.view("<u4")
+        return sum(int(w) * weight(first // 4 + i) for i, w in enumerate(words)) & m64
+
+    want = by_words(buf, 16)
+    assert oracle.checksum(buf, 16) == want
+    assert (oracle.checksum(buf[:400], 16) + oracle.checksum(buf[400:], 416)) & m64 == want
+    big = (1 << 34) + 8                                   # word index above 2^32
+    assert oracle.checksum(buf, big) == by_words(buf, big)
+    swapped = buf.copy(); swapped[[3, 700]] = swapped[[700, 3]]
+    assert buf[3] != buf[700] and oracle.checksum(swapped, 16) != want
