@@ -317,8 +317,9 @@ expand_kernel(SkipTable tab, uint32_t n, uint64_t r_begin, uint64_t r_end,
               const int8_t *__restrict__ recv, const int8_t *__restrict__ send,
               int4 *__restrict__ table_out)
 {
-    // per rank of the CTA and per round k of a phase: {send entry - x (+q), recv entry - x (+q),
-    // to, from}: the two arrays after the adjustment loop of Algorithm 6.
+    // per rank of the CTA and per round k of a phase: {send entry - x, recv entry - x, to, from}.
+    // Algorithm 6 adds q to an entry after each use and starts entries k < x at +q because
+    // their first use is in the second phase; both are covered by adding q * floor(i / q).
     __shared__ int4 base[kExpandRanks][32];
     const int q = tab.q;
     const uint32_t p = tab.p;
@@ -332,7 +333,7 @@ expand_kernel(SkipTable tab, uint32_t n, uint64_t r_begin, uint64_t r_end,
             const uint64_t row = (j0 + g) * (uint64_t)q;
             const uint32_t r = (uint32_t)(r_begin + j0 + g);
             const uint32_t sk = tab.s[k];
-            const int adj = k < x ? q - x : -x;
+            const int adj = -x;
             uint32_t to = r + sk;
             if (to >= p) to -= p;
             uint32_t from = r >= sk ? r - sk : r + p - sk;
