@@ -147,6 +147,64 @@ def _event_ms(torch, fn, flush, steps, warmup):
     return [a.elapsed_time(b) for a, b in pairs]
 
 
+def _bench_expand(torch, bcs, workloads, flush, hbm_gbs, peak_src, steps):
+    pe, ne = workloads.P_EXPAND, workloads.N_EXPAND
+    qe = bcs.bcs_q(pe)
+    er = torch.empty(pe * qe, dtype=torch.int8, device="cuda")
+    es = torch.empty(pe * qe, dtype=torch.int8, device="cuda")
+    bcs.bcs_build(pe, 0, pe, er, es)
+    rounds = ne - 1 + qe
+    table = torch.empty((pe, rounds, 4), dtype=torch.int32, device="cuda")
+    ms = statistics.mean(_event_ms(
+        torch, lambda: bcs.bcs_expand(pe, ne, 0, pe, er, es, table), flush, steps, 3))
+    nbytes = pe * rounds * 16
+    gbs = nbytes / ms / 1e6
+    res = {"workload": "p=100003, n=1000, all ranks, 1016 rounds, 16 B records", "ms": ms,
+           "bytes": nbytes, "gbs": gbs,
+           "roofline": {"bound": "hbm", "kernel": "expand_kernel", "achieved": gbs, "peak": hbm_gbs,
+                        "unit": "GB/s", "frac": gbs / hbm_gbs, "traffic": EXPAND_TRAFFIC_BYTES,
+                        "peak_source": peak_src}}
+    return res, table
+
+
+def _bench_checksum(torch, bcs, flush, hbm_gbs, peak_src, table, steps):
+    sums = torch.zeros(1, dtype=torch.int64, device="cuda")
+    tb = table.view(torch.int8).view(-1)
+    ms = statistics.mean(_event_ms(torch, lambda: bcs.bcs_checksum(tb, 0, sums), flush, steps, 3))
+    gbs = tb.numel() / ms / 1e6
+    return {"workload": "%.2f GB buffer" % (tb.numel() / 1e9), "ms": ms, "gbs": gbs,
+            "roofline": {"bound": "hbm", "kernel": "checksum_kernel", "achieved": gbs,
+                         "peak": hbm_gbs, "unit": "GB/s", "frac": gbs / hbm_gbs, "traffic": None,
+                         "peak_source": peak_src}}
+
+
+def _bench_batch(torch, bcs, workloads, flush, full):
+    out = {}
+    plan = bcs.bcs_batch_plan(workloads.small_sweep())
+    dplan = plan.to("cuda")
+    br = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
+    bs = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
+    ms = statistics.mean(_event_ms(
+        torch, lambda: bcs.bcs_build_batch(dplan, plan.total_ranks, plan.total_entries, br, bs),
+        flush, 20, 3))
+    out["batch_small_sweep"] = {"workload": "every p in 2..1024, one launch pair",
+                                "ranks": plan.total_ranks, "ms": ms,
+                                "ranks_per_s": plan.total_ranks / ms * 1e3}
+    plist = workloads.batch_p_list() if full else workloads.batch_p_list(count=256)
+    plan = bcs.bcs_batch_plan(plist)
+    dplan = plan.to("cuda")
+    br = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
+    bs = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
+    ms = statistics.mean(_event_ms(
+        torch, lambda: bcs.bcs_build_batch(dplan, plan.total_ranks, plan.total_entries, br, bs),
+        lambda: None, 3, 1))                       # the outputs exceed L2 by themselves
+    out["batch_irregular_sweep"] = {
+        "workload": "%d octave-uniform p in [2^10,2^20), seed %d" % (len(plist), workloads.SEED_BATCH),
+        "ranks": plan.total_ranks, "ms": ms, "ranks_per_s": plan.total_ranks / ms * 1e3,
+        "out_gbs": 2 * plan.total_entries / ms / 1e6}
+    return out
+
+
 def run_ours(args) -> None:
     import torch
     import torch.distributed as dist
@@ -165,15 +223,31 @@ def run_ours(args) -> None:
     bcs.lib()
 
     hbm_gbs, sm_max_mhz, peak_src = _peaks()
+    flush_buf = torch.empty(256 << 20, dtype=torch.int8, device="cuda")   # > 126 MB L2
+
+    def flush():
+        flush_buf.fill_(1)
+
+    if args.only in ("expand", "checksum", "batch"):       # small single-part runs (profiling)
+        if rank == 0:
+            res = {}
+            if args.only in ("expand", "checksum"):
+                ex, table = _bench_expand(torch, bcs, workloads, flush, hbm_gbs, peak_src,
+                                          args.steps)
+                res["expand"] = ex
+                if args.only == "checksum":
+                    res["checksum"] = _bench_checksum(torch, bcs, flush, hbm_gbs, peak_src, table,
+                                                      args.steps)
+            else:
+                res = _bench_batch(torch, bcs, workloads, flush, full=False)
+            print(json.dumps({"only": args.only, "steps": args.steps, "aux": res}))
+        return
+
     p = workloads.P_SINGLE
     q = bcs.bcs_q(p)
     nb = p * q
     recv = torch.empty(nb, dtype=torch.int8, device="cuda")
     send = torch.empty(nb, dtype=torch.int8, device="cuda")
-    flush_buf = torch.empty(256 << 20, dtype=torch.int8, device="cuda")   # > 126 MB L2
-
-    def flush():
-        flush_buf.fill_(1)
 
     def step():
         bcs.bcs_build(p, 0, p, recv, send)
@@ -204,98 +278,15 @@ def run_ours(args) -> None:
 
     out = None
     if rank == 0:
-        # ---- per-kernel times (same protocol): receive kernel alone, then the send kernel
+        # ---- per-kernel times (same protocol): receive kernel alone, the send kernel by difference
         recv_ms = statistics.mean(_event_ms(torch, lambda: bcs.bcs_build(p, 0, p, recv, None),
-                                            flush, max(20, args.steps // 4), 3))
+                                            flush, max(5, args.steps // 4), 3))
         send_ms = max(ms_per_step - recv_ms, 0.0)
-
-        # ---- end to end: host buffers, D2H copies inside the timed region
-        stage = torch.empty(2 * ((nb + 255) // 256 * 256), dtype=torch.int8, device="cuda")
-        h_recv = torch.empty(nb, dtype=torch.int8).pin_memory()
-        h_send = torch.empty(nb, dtype=torch.int8).pin_memory()
-        e2e_steps = max(5, min(args.steps, 50))
-        for _ in range(3):
-            bcs.bcs_build_to_host(p, 0, p, h_recv, h_send, stage)
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        for _ in range(e2e_steps):
-            bcs.bcs_build_to_host(p, 0, p, h_recv, h_send, stage)
-            torch.cuda.synchronize()
-        e2e_dt = (time.perf_counter() - t0) / e2e_steps
-        del stage
-
-        # ---- other entry points of the path (reported, not part of the metric)
-        aux = {}
-        pe, ne = workloads.P_EXPAND, workloads.N_EXPAND
-        qe = bcs.bcs_q(pe)
-        er = torch.empty(pe * qe, dtype=torch.int8, device="cuda")
-        es = torch.empty(pe * qe, dtype=torch.int8, device="cuda")
-        bcs.bcs_build(pe, 0, pe, er, es)
-        rounds = ne - 1 + qe
-        table = torch.empty((pe, rounds, 4), dtype=torch.int32, device="cuda")
-        ex_ms = statistics.mean(_event_ms(
-            torch, lambda: bcs.bcs_expand(pe, ne, 0, pe, er, es, table), flush, 20, 3))
-        ex_bytes = pe * rounds * 16
-        aux["expand"] = {"workload": "p=100003, n=1000, all ranks, 1016 rounds", "ms": ex_ms,
-                         "bytes": ex_bytes, "gbs": ex_bytes / ex_ms / 1e6,
-                         "roofline": {"bound": "hbm", "achieved": ex_bytes / ex_ms / 1e6,
-                                      "peak": hbm_gbs, "unit": "GB/s",
-                                      "frac": ex_bytes / ex_ms / 1e6 / hbm_gbs, "traffic": None,
-                                      "peak_source": peak_src}}
-        sums = torch.zeros(1, dtype=torch.int64, device="cuda")
-        tb = table.view(torch.int8).view(-1)
-        ck_ms = statistics.mean(_event_ms(
-            torch, lambda: bcs.bcs_checksum(tb, 0, sums), flush, 20, 3))
-        aux["checksum"] = {"workload": "1.63 GB buffer", "ms": ck_ms,
-                           "gbs": tb.numel() / ck_ms / 1e6,
-                           "frac_of_hbm": tb.numel() / ck_ms / 1e6 / hbm_gbs}
-        del table, tb
-        plan = bcs.bcs_batch_plan(workloads.small_sweep())
-        dplan = plan.to("cuda")
-        br = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
-        bs = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
-        b_ms = statistics.mean(_event_ms(
-            torch, lambda: bcs.bcs_build_batch(dplan, plan.total_ranks, plan.total_entries, br, bs),
-            flush, 20, 3))
-        aux["batch_small_sweep"] = {"workload": "every p in 2..1024, one launch pair",
-                                    "ranks": plan.total_ranks, "ms": b_ms,
-                                    "ranks_per_s": plan.total_ranks / b_ms * 1e3}
-        plan = bcs.bcs_batch_plan(workloads.batch_p_list())
-        dplan = plan.to("cuda")
-        br = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
-        bs = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
-        b_ms = statistics.mean(_event_ms(
-            torch, lambda: bcs.bcs_build_batch(dplan, plan.total_ranks, plan.total_entries, br, bs),
-            lambda: None, 3, 1))                       # outputs (24 GB) exceed L2 by themselves
-        aux["batch_irregular_sweep"] = {"workload": "4096 octave-uniform p in [2^10,2^20), seed 220510072",
-                                        "ranks": plan.total_ranks, "ms": b_ms,
-                                        "ranks_per_s": plan.total_ranks / b_ms * 1e3,
-                                        "out_gbs": 2 * plan.total_entries / b_ms / 1e6}
-        del br, bs
-
-        # ---- CPU baseline: the oracle as it stands, per-rank form, bounded sample
-        import oracle
-        cpu_sample = 262144
-        lo = p // 2 - cpu_sample // 2
-        t0 = time.perf_counter()
-        oracle.build_range(p, lo, lo + cpu_sample)
-        cpu_dt = time.perf_counter() - t0
-        t0 = time.perf_counter()
-        oracle.full_table(p)
-        cpu_arr_dt = time.perf_counter() - t0
-        cpu = {"value": cpu_sample / cpu_dt, "unit": UNIT, "cores": oracle.num_threads(),
-               "kind": "oracle",
-               "sample": "ranks %d..%d of p=2^20+1, per-rank form (Algorithms 4+5), %.1f s"
-                         % (lo, lo + cpu_sample - 1, cpu_dt),
-               "array_form_value": p / cpu_arr_dt}
-
-        # ---- roofline of the dominant kernel (receive schedule): integer issue
         model = ALU_MODEL[q]
-        ops_per_launch = model * p
         alu_peak = SM_COUNT * ALU_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12     # T int-op/s
-        achieved = ops_per_launch / (recv_ms * 1e-3) / 1e12
+        achieved = model * p / (recv_ms * 1e-3) / 1e12
         roof = {"bound": "alu", "kernel": "recv_kernel", "achieved": achieved, "peak": alu_peak,
-                "unit": "Tint-op/s", "frac": achieved / alu_peak, "traffic": None,
+                "unit": "Tint-op/s", "frac": achieved / alu_peak, "traffic": RECV_TRAFFIC_BYTES,
                 "ms": recv_ms, "model_int_ops_per_rank": model,
                 "peak_source": "148 SMs x 64 INT32 lanes x %.0f MHz (max SM clock)" % sm_max_mhz,
                 "hbm_time_frac": (2 * nb / (hbm_gbs * 1e9)) / (ms_per_step * 1e-3),
@@ -310,18 +301,61 @@ def run_ours(args) -> None:
                        "timed_wall_s": t_wall},
             "out_gbs": 2 * nb / ms_per_step / 1e6,
             "kernel_ms": {"recv_kernel": recv_ms, "send_kernel": send_ms},
-            "roofline": roof, "cpu_baseline": cpu,
-            "e2e": {"value": p / e2e_dt, "unit": UNIT, "h2d_bytes_per_step": 0,
-                    "d2h_bytes_per_step": 2 * nb, "ms_per_step": e2e_dt * 1e3},
-            "gpu_launches": 2 * args.steps,
-            "clocks": clk.summary(), "aux": aux,
+            "roofline": roof, "gpu_launches": 2 * args.steps, "clocks": clk.summary(),
         }
+        if args.only == "all":
+            # ---- end to end: host buffers, D2H copies inside the timed region
+            stage = torch.empty(2 * ((nb + 255) // 256 * 256), dtype=torch.int8, device="cuda")
+            h_recv = torch.empty(nb, dtype=torch.int8).pin_memory()
+            h_send = torch.empty(nb, dtype=torch.int8).pin_memory()
+            e2e_steps = max(5, min(args.steps, 50))
+            for _ in range(3):
+                bcs.bcs_build_to_host(p, 0, p, h_recv, h_send, stage)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for _ in range(e2e_steps):
+                bcs.bcs_build_to_host(p, 0, p, h_recv, h_send, stage)
+                torch.cuda.synchronize()
+            e2e_dt = (time.perf_counter() - t0) / e2e_steps
+            del stage
+            out["e2e"] = {"value": p / e2e_dt, "unit": UNIT, "h2d_bytes_per_step": 0,
+                          "d2h_bytes_per_step": 2 * nb, "ms_per_step": e2e_dt * 1e3}
+
+            # ---- other entry points of the path (reported, not part of the metric)
+            aux = {}
+            aux["expand"], table = _bench_expand(torch, bcs, workloads, flush, hbm_gbs, peak_src, 20)
+            aux["checksum"] = _bench_checksum(torch, bcs, flush, hbm_gbs, peak_src, table, 20)
+            del table
+            aux.update(_bench_batch(torch, bcs, workloads, flush, full=True))
+            out["aux"] = aux
+
+            # ---- CPU baseline: the oracle as it stands, per-rank form, bounded sample
+            import oracle
+            cpu_sample = 1 << 20
+            lo = 0
+            t0 = time.perf_counter()
+            oracle.build_range(p, lo, lo + cpu_sample)
+            cpu_dt = time.perf_counter() - t0
+            t0 = time.perf_counter()
+            oracle.full_table(p)
+            cpu_arr_dt = time.perf_counter() - t0
+            out["cpu_baseline"] = {
+                "value": cpu_sample / cpu_dt, "unit": UNIT, "cores": oracle.num_threads(),
+                "kind": "oracle",
+                "sample": "ranks %d..%d of p=2^20+1, per-rank form (Algorithms 4+5), %.1f s"
+                          % (lo, lo + cpu_sample - 1, cpu_dt),
+                "array_form_value": p / cpu_arr_dt}
     barrier()
     if world > 1:
         dist.destroy_process_group()
     if out is not None:
         print(json.dumps(out))
 
+
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of the
+# current kernels); None until counters have been taken for the kernel as it stands.
+RECV_TRAFFIC_BYTES = None
+EXPAND_TRAFFIC_BYTES = None
 
 # integer operations per rank of the receive-schedule construction that the kernel runs,
 # by q: descent steps per rank (CPU count of the same loops) x operations per step.
@@ -334,6 +368,8 @@ def main() -> None:
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--only", default="all", choices=["all", "build", "expand", "checksum", "batch"],
+                    help="run one part only (small, profiler-friendly runs); 'all' is the benchmark")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
