@@ -152,7 +152,8 @@ def _bench_expand(torch, bcs, workloads, flush, hbm_gbs, peak_src, steps):
     qe = bcs.bcs_q(pe)
     er = torch.empty(pe * qe, dtype=torch.int8, device="cuda")
     es = torch.empty(pe * qe, dtype=torch.int8, device="cuda")
-    bcs.bcs_build(pe, 0, pe, er, es)
+    ews = torch.empty(bcs.bcs_build_workspace_bytes(pe, 0, pe), dtype=torch.int8, device="cuda")
+    bcs.bcs_build(pe, 0, pe, er, es, ews)
     rounds = ne - 1 + qe
     table = torch.empty((pe, rounds, 4), dtype=torch.int32, device="cuda")
     ms = statistics.mean(_event_ms(
@@ -184,8 +185,10 @@ def _bench_batch(torch, bcs, workloads, flush, full):
     dplan = plan.to("cuda")
     br = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
     bs = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
+    bw = torch.empty(bcs.bcs_build_batch_workspace_bytes(plan.total_ranks, plan.total_entries),
+                     dtype=torch.int8, device="cuda")
     ms = statistics.mean(_event_ms(
-        torch, lambda: bcs.bcs_build_batch(dplan, plan.total_ranks, plan.total_entries, br, bs),
+        torch, lambda: bcs.bcs_build_batch(dplan, plan.total_ranks, plan.total_entries, br, bs, bw),
         flush, 20, 3))
     out["batch_small_sweep"] = {"workload": "every p in 2..1024, one launch pair",
                                 "ranks": plan.total_ranks, "ms": ms,
@@ -193,10 +196,13 @@ def _bench_batch(torch, bcs, workloads, flush, full):
     plist = workloads.batch_p_list() if full else workloads.batch_p_list(count=256)
     plan = bcs.bcs_batch_plan(plist)
     dplan = plan.to("cuda")
+    del br, bs, bw
     br = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
     bs = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
+    bw = torch.empty(bcs.bcs_build_batch_workspace_bytes(plan.total_ranks, plan.total_entries),
+                     dtype=torch.int8, device="cuda")
     ms = statistics.mean(_event_ms(
-        torch, lambda: bcs.bcs_build_batch(dplan, plan.total_ranks, plan.total_entries, br, bs),
+        torch, lambda: bcs.bcs_build_batch(dplan, plan.total_ranks, plan.total_entries, br, bs, bw),
         lambda: None, 3, 1))                       # the outputs exceed L2 by themselves
     out["batch_irregular_sweep"] = {
         "workload": "%d octave-uniform p in [2^10,2^20), seed %d" % (len(plist), workloads.SEED_BATCH),
@@ -248,9 +254,11 @@ def run_ours(args) -> None:
     nb = p * q
     recv = torch.empty(nb, dtype=torch.int8, device="cuda")
     send = torch.empty(nb, dtype=torch.int8, device="cuda")
+    ws_bytes = bcs.bcs_build_workspace_bytes(p, 0, p)
+    ws = torch.empty(ws_bytes, dtype=torch.int8, device="cuda")
 
     def step():
-        bcs.bcs_build(p, 0, p, recv, send)
+        bcs.bcs_build(p, 0, p, recv, send, ws)
 
     def barrier():
         torch.cuda.synchronize()
@@ -278,17 +286,21 @@ def run_ours(args) -> None:
 
     out = None
     if rank == 0:
-        # ---- per-kernel times (same protocol): receive kernel alone, the send kernel by difference
-        recv_ms = statistics.mean(_event_ms(torch, lambda: bcs.bcs_build(p, 0, p, recv, None),
+        # ---- per-kernel times (same protocol).  A receive-only call runs the codes kernel and the
+        # receive kernel (without the round-major copy); the send kernel is the difference.
+        recv_ms = statistics.mean(_event_ms(torch, lambda: bcs.bcs_build(p, 0, p, recv, None, ws),
                                             flush, max(5, args.steps // 4), 3))
         send_ms = max(ms_per_step - recv_ms, 0.0)
+        slow_ms = statistics.mean(_event_ms(torch, lambda: bcs.bcs_build(p, 0, p, recv, send, None),
+                                            flush, 10, 2))
         model = ALU_MODEL[q]
         alu_peak = SM_COUNT * ALU_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12     # T int-op/s
         achieved = model * p / (recv_ms * 1e-3) / 1e12
-        roof = {"bound": "alu", "kernel": "recv_kernel", "achieved": achieved, "peak": alu_peak,
-                "unit": "Tint-op/s", "frac": achieved / alu_peak, "traffic": RECV_TRAFFIC_BYTES,
-                "ms": recv_ms, "model_int_ops_per_rank": model,
+        roof = {"bound": "alu", "kernel": "codes_kernel+recv_codes_kernel", "achieved": achieved,
+                "peak": alu_peak, "unit": "Tint-op/s", "frac": achieved / alu_peak,
+                "traffic": RECV_TRAFFIC_BYTES, "ms": recv_ms, "model_int_ops_per_rank": model,
                 "peak_source": "148 SMs x 64 INT32 lanes x %.0f MHz (max SM clock)" % sm_max_mhz,
+                "hbm_bound_ms": 2 * nb / (hbm_gbs * 1e6),
                 "hbm_time_frac": (2 * nb / (hbm_gbs * 1e9)) / (ms_per_step * 1e-3),
                 "hbm_peak_source": peak_src}
         out = {
@@ -300,12 +312,15 @@ def run_ours(args) -> None:
                        "parallelism": "replicas" if world > 1 else "1 GPU",
                        "timed_wall_s": t_wall},
             "out_gbs": 2 * nb / ms_per_step / 1e6,
-            "kernel_ms": {"recv_kernel": recv_ms, "send_kernel": send_ms},
-            "roofline": roof, "gpu_launches": 2 * args.steps, "clocks": clk.summary(),
+            "kernel_ms": {"codes+recv_codes": recv_ms, "send_rm": send_ms,
+                          "self_contained_path_step": slow_ms},
+            "workspace_bytes": ws_bytes,
+            "roofline": roof, "gpu_launches": 3 * args.steps, "clocks": clk.summary(),
         }
         if args.only == "all":
             # ---- end to end: host buffers, D2H copies inside the timed region
-            stage = torch.empty(2 * ((nb + 255) // 256 * 256), dtype=torch.int8, device="cuda")
+            stage = torch.empty(2 * ((nb + 255) // 256 * 256) + ws_bytes, dtype=torch.int8,
+                                device="cuda")
             h_recv = torch.empty(nb, dtype=torch.int8).pin_memory()
             h_send = torch.empty(nb, dtype=torch.int8).pin_memory()
             e2e_steps = max(5, min(args.steps, 50))
@@ -357,9 +372,11 @@ def run_ours(args) -> None:
 RECV_TRAFFIC_BYTES = None
 EXPAND_TRAFFIC_BYTES = None
 
-# integer operations per rank of the receive-schedule construction that the kernel runs,
-# by q: descent steps per rank (CPU count of the same loops) x operations per step.
-ALU_MODEL = {21: 12 * 287 + 10 * 10 + 20 * 21}
+# integer operations per rank of the receive-schedule construction that the kernels run, by q:
+# skip code (3 per level + 5) + per round 22 (two address selects, code load, one step of the
+# head search, set update, entry, two stores, loop) + the measured extra 0.66 search steps and
+# 0.19 second windows per rank (CPU count of the same loops over sampled ranks of p = 2^20+1).
+ALU_MODEL = {21: (3 * 21 + 5) + 22 * 21 + 14}
 
 
 def main() -> None:

@@ -15,7 +15,8 @@
  *     "host" pointers are ordinary host addresses.  The caller owns every buffer.
  *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
  *     Calls only enqueue work on that stream; they do not synchronise, and the
- *     library holds no device memory of its own unless an entry point says so.
+ *     library holds no device memory of its own unless an entry point says so
+ *     (scratch memory is passed in by the caller as a `workspace`).
  *   - Schedule tables are int8, rank-major and unpadded: the row of rank r of a
  *     call for ranks r_begin..r_end-1 starts at byte (r - r_begin) * q.
  *   - Errors are return codes.  When a code other than BCS_OK is returned nothing
@@ -64,17 +65,30 @@ bcs_status bcs_skips(uint32_t p, uint32_t *skips_host);
  * r_begin..r_end-1 of one p.
  *   recv_out, send_out: device, int8, (r_end-r_begin)*q bytes each, 16-byte
  *   aligned; either may be NULL (not wanted), not both unless the range is empty.
- * A send entry whose to-processor lies inside the range is looked up in recv_out
- * (when given); the others are recomputed with Algorithm 4, so any sub-range is
- * self-contained.  Errors: see the status codes. */
+ *   workspace: device scratch owned by the caller, 16-byte aligned, or NULL.  With at
+ *   least bcs_build_workspace_bytes(p, r_begin, r_end) bytes the call runs its fast
+ *   construction: one pass writes a 32-bit "skip code" per rank of p (which skips add
+ *   up to the rank, the sums Algorithm 2 walks down), a second finds each round's
+ *   block from the codes of the two ranks bounding the window of Algorithm 4 and also
+ *   keeps a round-major copy of the receive rows, a third reads the send rows from
+ *   that copy.  With NULL (or too few bytes) a self-contained, several times slower
+ *   construction runs (homerange descent per window; send entries whose to-processor
+ *   lies outside the range are recomputed with Algorithm 4).  Both give identical
+ *   tables, and any sub-range is self-contained either way.  The workspace holds
+ *   nothing of value after the call; calls that share one must not overlap.
+ * Errors: see the status codes. */
+size_t bcs_build_workspace_bytes(uint32_t p, uint64_t r_begin, uint64_t r_end);
 bcs_status bcs_build(uint32_t p, uint64_t r_begin, uint64_t r_end,
-                     int8_t *recv_out, int8_t *send_out, void *cuda_stream);
+                     int8_t *recv_out, int8_t *send_out,
+                     void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /* As bcs_build, then copies the tables to HOST memory on the same stream
  * (cudaMemcpyAsync; pinned host memory makes the copies asynchronous).
  *   recv_host, send_host: host, (r_end-r_begin)*q bytes each, either may be NULL.
  *   stage_dev: device staging buffer supplied by the caller, 16-byte aligned, of
- *   at least 2 * align256((r_end-r_begin)*q) bytes (align256 = round up to 256).
+ *   at least 2 * align256((r_end-r_begin)*q) bytes (align256 = round up to 256);
+ *   what exceeds that is handed to bcs_build as its workspace, so adding
+ *   bcs_build_workspace_bytes(...) bytes selects the fast construction.
  * The host buffers are complete once the stream has been synchronised. */
 bcs_status bcs_build_to_host(uint32_t p, uint64_t r_begin, uint64_t r_end,
                              int8_t *recv_host, int8_t *send_host,
@@ -84,23 +98,30 @@ bcs_status bcs_build_to_host(uint32_t p, uint64_t r_begin, uint64_t r_end,
  *   rank_off_host[num_p+1]  prefix sums of p_j            (flattened rank index),
  *   entry_off_host[num_p+1] prefix sums of p_j * q_j      (byte offset of p_j's table),
  *   skips_tab_host[num_p * BCS_SKIPS_STRIDE] row j = skips[0..q_j] of p_j (Algorithm 1),
- *                           the rest of the row 0.
- * The caller copies the three arrays and p_list to the device. */
+ *                           the rest of the row 0,
+ *   full_tab_host[num_p * BCS_SKIPS_STRIDE]  row j, word d = skip code of rank
+ *                           skips[d]-1 of p_j, d = 0..q_j.
+ * The caller copies the four arrays and p_list to the device. */
 bcs_status bcs_batch_plan(const uint32_t *p_list_host, uint32_t num_p,
                           uint64_t *rank_off_host, uint64_t *entry_off_host,
-                          uint32_t *skips_tab_host);
+                          uint32_t *skips_tab_host, uint32_t *full_tab_host);
 
 /* All ranks of many p at once (the "full schedule" of Algorithm 9 for each p_j),
- * one launch over the flattened list of (p_j, r) pairs.  Device inputs as laid
- * out by bcs_batch_plan; total_ranks = rank_off[num_p], total_entries =
+ * one launch sequence over the flattened list of (p_j, r) pairs.  Device inputs as
+ * laid out by bcs_batch_plan; total_ranks = rank_off[num_p], total_entries =
  * entry_off[num_p] (the host knows both).  Outputs: device int8, total_entries
  * bytes each, 16-byte aligned; the table of p_j starts at byte entry_off[j] and
  * is rank-major with q_j bytes per rank.  send_out may be NULL; recv_out is
- * required (the send table is looked up in it). */
+ * required.  workspace as for bcs_build, of
+ * bcs_build_batch_workspace_bytes(total_ranks, total_entries) bytes for the fast
+ * construction, or NULL. */
+size_t bcs_build_batch_workspace_bytes(uint64_t total_ranks, uint64_t total_entries);
 bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_dev,
                            const uint64_t *entry_off_dev, const uint32_t *skips_tab_dev,
+                           const uint32_t *full_tab_dev,
                            uint32_t num_p, uint64_t total_ranks, uint64_t total_entries,
-                           int8_t *recv_out, int8_t *send_out, void *cuda_stream);
+                           int8_t *recv_out, int8_t *send_out,
+                           void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /* Round tables of the n-block broadcast (Algorithm 6 without the Send||Recv): for
  * each rank r of r_begin..r_end-1 and each round j of 0..n-2+q one record of four

@@ -12,6 +12,8 @@ from .binding import (  # noqa: F401
     bcs_batch_plan,
     bcs_build,
     bcs_build_batch,
+    bcs_build_batch_workspace_bytes,
+    bcs_build_workspace_bytes,
     bcs_build_to_host,
     bcs_checksum,
     bcs_expand,

@@ -44,13 +44,17 @@ def lib():
         L.bcs_q.restype = i32
         L.bcs_skips.argtypes = [u32, vp]
         L.bcs_skips.restype = i32
-        L.bcs_build.argtypes = [u32, u64, u64, vp, vp, vp]
+        L.bcs_build_workspace_bytes.argtypes = [u32, u64, u64]
+        L.bcs_build_workspace_bytes.restype = _c.c_size_t
+        L.bcs_build.argtypes = [u32, u64, u64, vp, vp, vp, _c.c_size_t, vp]
         L.bcs_build.restype = i32
         L.bcs_build_to_host.argtypes = [u32, u64, u64, vp, vp, vp, _c.c_size_t, vp]
         L.bcs_build_to_host.restype = i32
-        L.bcs_batch_plan.argtypes = [vp, u32, vp, vp, vp]
+        L.bcs_batch_plan.argtypes = [vp, u32, vp, vp, vp, vp]
         L.bcs_batch_plan.restype = i32
-        L.bcs_build_batch.argtypes = [vp, vp, vp, vp, u32, u64, u64, vp, vp, vp]
+        L.bcs_build_batch_workspace_bytes.argtypes = [u64, u64]
+        L.bcs_build_batch_workspace_bytes.restype = _c.c_size_t
+        L.bcs_build_batch.argtypes = [vp, vp, vp, vp, vp, u32, u64, u64, vp, vp, vp, _c.c_size_t, vp]
         L.bcs_build_batch.restype = i32
         L.bcs_expand.argtypes = [u32, u32, u64, u64, vp, vp, vp, vp]
         L.bcs_expand.restype = i32
@@ -89,10 +93,20 @@ def bcs_skips(p: int) -> list[int]:
     return list(buf[: bcs_q(p) + 1])
 
 
-def bcs_build(p: int, r_begin: int, r_end: int, recv_out, send_out, stream=None) -> None:
-    """recv_out / send_out: CUDA int8 tensors of (r_end-r_begin)*q elements, or None."""
-    _check(lib().bcs_build(p, r_begin, r_end, _ptr(recv_out), _ptr(send_out), _stream(stream)),
-           "bcs_build")
+def _nbytes(t) -> int:
+    return 0 if t is None else t.numel() * t.element_size()
+
+
+def bcs_build_workspace_bytes(p: int, r_begin: int, r_end: int) -> int:
+    return lib().bcs_build_workspace_bytes(p, r_begin, r_end)
+
+
+def bcs_build(p: int, r_begin: int, r_end: int, recv_out, send_out, workspace=None,
+              stream=None) -> None:
+    """recv_out / send_out: CUDA int8 tensors of (r_end-r_begin)*q elements, or None;
+    workspace: CUDA tensor of bcs_build_workspace_bytes(...) bytes (fast path) or None."""
+    _check(lib().bcs_build(p, r_begin, r_end, _ptr(recv_out), _ptr(send_out), _ptr(workspace),
+                           _nbytes(workspace), _stream(stream)), "bcs_build")
 
 
 def bcs_build_to_host(p: int, r_begin: int, r_end: int, recv_host, send_host, stage_dev,
@@ -111,6 +125,7 @@ class BatchPlan:
     rank_off: torch.Tensor    # int64 [num_p+1]
     entry_off: torch.Tensor   # int64 [num_p+1]
     skips_tab: torch.Tensor   # int32 [num_p, 32]
+    full_tab: torch.Tensor    # int32 [num_p, 32]
 
     @property
     def num_p(self) -> int:
@@ -126,7 +141,8 @@ class BatchPlan:
 
     def to(self, device, non_blocking: bool = False) -> "BatchPlan":
         return BatchPlan(*(t.to(device, non_blocking=non_blocking)
-                           for t in (self.p_list, self.rank_off, self.entry_off, self.skips_tab)))
+                           for t in (self.p_list, self.rank_off, self.entry_off, self.skips_tab,
+                                     self.full_tab)))
 
 
 def bcs_batch_plan(p_list, pin: bool = False) -> BatchPlan:
@@ -140,21 +156,28 @@ def bcs_batch_plan(p_list, pin: bool = False) -> BatchPlan:
     rank_off = torch.zeros(n + 1, dtype=torch.int64)
     entry_off = torch.zeros(n + 1, dtype=torch.int64)
     skips_tab = torch.zeros((n, BCS_SKIPS_STRIDE), dtype=torch.int32)
+    full_tab = torch.zeros((n, BCS_SKIPS_STRIDE), dtype=torch.int32)
     if pin:
-        p32, rank_off, entry_off, skips_tab = (t.pin_memory()
-                                               for t in (p32, rank_off, entry_off, skips_tab))
+        p32, rank_off, entry_off, skips_tab, full_tab = (
+            t.pin_memory() for t in (p32, rank_off, entry_off, skips_tab, full_tab))
     _check(lib().bcs_batch_plan(p32.data_ptr(), n, rank_off.data_ptr(), entry_off.data_ptr(),
-                                skips_tab.data_ptr()), "bcs_batch_plan")
-    return BatchPlan(p32, rank_off, entry_off, skips_tab)
+                                skips_tab.data_ptr(), full_tab.data_ptr()), "bcs_batch_plan")
+    return BatchPlan(p32, rank_off, entry_off, skips_tab, full_tab)
+
+
+def bcs_build_batch_workspace_bytes(total_ranks: int, total_entries: int) -> int:
+    return lib().bcs_build_batch_workspace_bytes(total_ranks, total_entries)
 
 
 def bcs_build_batch(plan_dev: BatchPlan, total_ranks: int, total_entries: int, recv_out, send_out,
-                    stream=None) -> None:
-    """plan_dev: a BatchPlan whose tensors live on the CUDA device."""
+                    workspace=None, stream=None) -> None:
+    """plan_dev: a BatchPlan whose tensors live on the CUDA device; workspace: CUDA tensor of
+    bcs_build_batch_workspace_bytes(...) bytes (fast path) or None."""
     _check(lib().bcs_build_batch(plan_dev.p_list.data_ptr(), plan_dev.rank_off.data_ptr(),
                                  plan_dev.entry_off.data_ptr(), plan_dev.skips_tab.data_ptr(),
-                                 plan_dev.num_p, total_ranks, total_entries, _ptr(recv_out),
-                                 _ptr(send_out), _stream(stream)), "bcs_build_batch")
+                                 plan_dev.full_tab.data_ptr(), plan_dev.num_p, total_ranks,
+                                 total_entries, _ptr(recv_out), _ptr(send_out), _ptr(workspace),
+                                 _nbytes(workspace), _stream(stream)), "bcs_build_batch")
 
 
 def bcs_expand(p: int, n: int, r_begin: int, r_end: int, recv, send, table_out, stream=None) -> None:

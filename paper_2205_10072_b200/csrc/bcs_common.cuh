@@ -1,0 +1,216 @@
+// Shared pieces of the schedule, round-table and checksum translation units: per-p tables,
+// the Section 2 primitives of arXiv 2205.10072 as device functions, and the tile bookkeeping
+// that turns per-rank rows into contiguous, 16-byte vectorised output spans.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "bcs.h"
+
+namespace bcs {
+
+constexpr int kTile = 256;                    // ranks (= threads) per CTA of the schedule kernels
+constexpr int kStageBytes = kTile * 32 + 16;  // kTile rows of <= 31 bytes + alignment shift
+constexpr int kCachedRows = 4;                // per-p table rows a batch CTA keeps in shared memory
+constexpr int kRow = BCS_SKIPS_STRIDE;        // words per table row
+
+// Per-p constants (kernel parameter of the single-p kernels).
+//   s[k]    = skips[k] of Algorithm 1, k = 0..q (q <= 31)
+//   full[d] = skip code of rank skips[d]-1, d = 0..q (see skip_code below)
+struct PTable {
+    uint32_t s[kRow];
+    uint32_t full[kRow];
+    uint32_t p;
+    int q;
+};
+
+struct BatchArgs {
+    const uint32_t *p_list;
+    const uint64_t *rank_off;
+    const uint64_t *entry_off;
+    const uint32_t *skips_tab;   // [num_p][kRow]
+    const uint32_t *full_tab;    // [num_p][kRow]
+    uint32_t num_p;
+    uint64_t total_ranks;
+};
+
+__host__ __device__ inline int ceil_log2_u32(uint32_t p)
+{
+    int q = 0;
+    while (q < 32 && (uint64_t(1) << q) < p) ++q;
+    return q;
+}
+
+__device__ __forceinline__ int ceil_log2_fast(uint32_t p) { return p > 1u ? 32 - __clz(p - 1u) : 0; }
+
+// ---------------------------------------------------------------- Section 2 primitives
+// Largest k with skips[k] <= x (the homerange of x), 1 <= x < p.  Algorithm 1 gives
+// 2^(k-1) < skips[k] <= 2^k, so k is floor(log2 x) or one more.
+__device__ __forceinline__ int home_of(const uint32_t *s, uint32_t x)
+{
+    int m = 31 - __clz(x);
+    return m + (s[m + 1] <= x ? 1 : 0);
+}
+
+// Skip code of rank x (0 <= x < p): bit k set iff skips[k] is a term of the greedy
+// decomposition x = skips[k1] + skips[k2] + ... that Algorithm 2 walks down (largest skip
+// not above the remainder first; the remainder after taking skips[k] is below skips[k], so a
+// downward scan over the levels finds the same terms).  The baseblock of x is the lowest set
+// bit, its homerange the highest.  Codes order like ranks.
+__host__ __device__ inline uint32_t skip_code(const uint32_t *s, int q, uint32_t x)
+{
+    uint32_t code = 0;
+    for (int k = q - 1; k >= 0; --k) {
+        if (x >= s[k]) {
+            x -= s[k];
+            code |= 1u << k;
+        }
+    }
+    return code;
+}
+
+// ---------------------------------------------------------------- tile bookkeeping
+struct RankCtx {
+    const uint32_t *s;      // skips of this rank's p (shared or global memory)
+    const uint32_t *full;   // full[] of this rank's p
+    uint32_t p;
+    int q;
+    uint32_t r;
+    uint32_t pj;            // index of p in the batch (0 for the single-p kernels)
+    uint64_t rank0;         // flattened index of rank 0 of this p (0 for single p)
+    uint64_t entry;         // byte offset of the rank's row in the output
+    bool valid;
+};
+
+struct TileShared {
+    uint32_t skips[kCachedRows][kRow];
+    uint32_t full[kCachedRows][kRow];
+    uint64_t span_begin, span_end;
+    uint32_t j_first, j_last;
+    __align__(16) uint8_t stage[kStageBytes];
+};
+
+// Copies stage[shift, shift+len) to out[byte0, byte0+len); (byte0 & 15) == shift and `out`
+// is 16-byte aligned, so all but the ragged ends go out as 16-byte vectors.
+__device__ __forceinline__ void flush_span(const uint8_t *stage, uint32_t shift, uint32_t len,
+                                           int8_t *out, uint64_t byte0)
+{
+    uint8_t *dst = reinterpret_cast<uint8_t *>(out) + (byte0 - shift);
+    const uint32_t end = shift + len;
+    const uint32_t nvec = (end + 15u) >> 4;
+    for (uint32_t v = threadIdx.x; v < nvec; v += blockDim.x) {
+        uint32_t lo = v << 4, hi = lo + 16u;
+        if (lo >= shift && hi <= end) {
+            *reinterpret_cast<uint4 *>(dst + lo) = *reinterpret_cast<const uint4 *>(stage + lo);
+        } else {
+            uint32_t from = lo < shift ? shift : lo, to = hi > end ? end : hi;
+            for (uint32_t e = from; e < to; ++e) dst[e] = stage[e];
+        }
+    }
+}
+
+// Largest j with off[j] <= g, searched in [lo, hi].
+__device__ __forceinline__ uint32_t find_segment(const uint64_t *off, uint32_t lo, uint32_t hi,
+                                                 uint64_t g)
+{
+    while (lo < hi) {
+        uint32_t mid = (lo + hi + 1) >> 1;
+        if (off[mid] <= g) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+// Resolves the rank this thread works on.  Single p: consecutive ranks from r_begin.
+// Batch: flattened index g over all (p_j, r); the CTA looks up the first and last p it
+// touches once, keeps the first few table rows in shared memory, and each thread finds
+// its own p between the two.
+template <bool kBatch>
+__device__ __forceinline__ RankCtx resolve_rank(TileShared &sh, const PTable &tab,
+                                                uint64_t r_begin, uint64_t r_end,
+                                                const BatchArgs &ba)
+{
+    RankCtx c;
+    const uint64_t g0 = (uint64_t)blockIdx.x * kTile;
+    if (!kBatch) {
+        if (threadIdx.x < kRow) {
+            sh.skips[0][threadIdx.x] = tab.s[threadIdx.x];
+            sh.full[0][threadIdx.x] = tab.full[threadIdx.x];
+        }
+        const uint64_t count = r_end - r_begin;
+        const uint64_t g1 = g0 + kTile < count ? g0 + kTile : count;
+        if (threadIdx.x == 0) {
+            sh.span_begin = g0 * (uint64_t)tab.q;
+            sh.span_end = g1 * (uint64_t)tab.q;
+        }
+        __syncthreads();
+        const uint64_t g = g0 + threadIdx.x;
+        c.s = sh.skips[0];
+        c.full = sh.full[0];
+        c.p = tab.p;
+        c.q = tab.q;
+        c.pj = 0;
+        c.rank0 = 0;
+        c.valid = g < count;
+        c.r = (uint32_t)(r_begin + g);
+        c.entry = g * (uint64_t)tab.q;
+        return c;
+    }
+    const uint64_t g1 = g0 + kTile < ba.total_ranks ? g0 + kTile : ba.total_ranks;
+    if (threadIdx.x == 0) {
+        uint32_t jf = find_segment(ba.rank_off, 0, ba.num_p - 1, g0);
+        uint32_t jl = find_segment(ba.rank_off, jf, ba.num_p - 1, g1 - 1);
+        sh.j_first = jf;
+        sh.j_last = jl;
+        int qf = ceil_log2_fast(ba.p_list[jf]);
+        int ql = ceil_log2_fast(ba.p_list[jl]);
+        sh.span_begin = ba.entry_off[jf] + (g0 - ba.rank_off[jf]) * (uint64_t)qf;
+        sh.span_end = ba.entry_off[jl] + (g1 - ba.rank_off[jl]) * (uint64_t)ql;
+    }
+    __syncthreads();
+    const uint32_t jf = sh.j_first, jl = sh.j_last;
+    {
+        const uint32_t row = threadIdx.x / (2 * kRow), col = threadIdx.x % (2 * kRow);
+        if (row < kCachedRows && jf + row <= jl) {
+            if (col < kRow)
+                sh.skips[row][col] = ba.skips_tab[(size_t)(jf + row) * kRow + col];
+            else
+                sh.full[row][col - kRow] = ba.full_tab[(size_t)(jf + row) * kRow + col - kRow];
+        }
+    }
+    __syncthreads();
+    const uint64_t g = g0 + threadIdx.x;
+    c.valid = g < g1;
+    const uint32_t j = c.valid ? find_segment(ba.rank_off, jf, jl, g) : jf;
+    const bool cached = j - jf < (uint32_t)kCachedRows;
+    c.s = cached ? sh.skips[j - jf] : ba.skips_tab + (size_t)j * kRow;
+    c.full = cached ? sh.full[j - jf] : ba.full_tab + (size_t)j * kRow;
+    c.pj = j;
+    c.p = ba.p_list[j];
+    c.q = ceil_log2_fast(c.p);
+    c.rank0 = ba.rank_off[j];
+    c.r = (uint32_t)(g - c.rank0);
+    c.entry = ba.entry_off[j] + (uint64_t)c.r * (uint64_t)c.q;
+    return c;
+}
+
+// ---------------------------------------------------------------- host helpers
+bcs_status make_table(uint32_t p, PTable *tab);
+
+inline bool aligned16(const void *ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
+
+inline bcs_status launch_status()
+{
+    return cudaGetLastError() == cudaSuccess ? BCS_OK : BCS_ERR_CUDA;
+}
+
+inline bcs_status check_range(uint32_t p, uint64_t r_begin, uint64_t r_end)
+{
+    if (p == 0) return BCS_ERR_RANGE;
+    if (p > 0x7fffffffu) return BCS_ERR_UNSUPPORTED;
+    if (r_begin > r_end || r_end > p) return BCS_ERR_RANGE;
+    return BCS_OK;
+}
+
+inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace bcs

@@ -30,7 +30,8 @@ def _declared_symbols():
 def test_every_declared_symbol_is_exported(lib):
     names = _declared_symbols()
     assert {"bcs_build", "bcs_build_batch", "bcs_expand", "bcs_checksum", "bcs_skips", "bcs_q",
-            "bcs_batch_plan", "bcs_status_str", "bcs_build_to_host"} <= set(names)
+            "bcs_batch_plan", "bcs_status_str", "bcs_build_to_host", "bcs_build_workspace_bytes",
+            "bcs_build_batch_workspace_bytes"} <= set(names)
     dll = ctypes.CDLL(lib.lib_path())
     for n in names:
         assert hasattr(dll, n), n
@@ -66,6 +67,9 @@ def test_batch_plan_host_side(lib):
     assert plan.entry_off.tolist() == [0, 2, 8, 108, 108, 108 + 1025 * 11]
     assert plan.skips_tab[2].tolist()[:6] == [1, 2, 3, 5, 10, 20]
     assert plan.skips_tab[3].tolist()[:2] == [1, 0]
+    # full_tab[d] = skip code of rank skips[d]-1: p = 20, skips 1 2 3 5 10 20:
+    # 0 -> {}, 1 -> {0}, 2 -> {1}, 4 = 3+1 -> {2,0}, 9 = 5+3+1 -> {3,2,0}, 19 = 10+5+3+1
+    assert plan.full_tab[2].tolist()[:6] == [0, 1, 2, 5, 13, 29]
     assert plan.total_ranks == 1051
     with pytest.raises(lib.BcsError):
         lib.bcs_batch_plan([5, 0])
@@ -74,19 +78,22 @@ def test_batch_plan_host_side(lib):
 def test_argument_errors_need_no_gpu(lib):
     """Validation happens before any CUDA call: these return an error code on a CPU-only box."""
     L = lib.lib()
-    assert L.bcs_build(0, 0, 0, None, None, None) == 2
-    assert L.bcs_build(2**31, 0, 1, None, None, None) == 4
-    assert L.bcs_build(10, 5, 4, None, None, None) == 2
-    assert L.bcs_build(10, 0, 11, None, None, None) == 2
-    assert L.bcs_build(10, 0, 10, None, None, None) == 1
-    assert L.bcs_build(10, 0, 10, 8, None, None) == 3            # misaligned pointer
-    assert L.bcs_build(1, 0, 1, None, None, None) == 0           # q == 0: nothing to do
-    assert L.bcs_build(10, 3, 3, None, None, None) == 0          # empty range
+    assert L.bcs_build(0, 0, 0, None, None, None, 0, None) == 2
+    assert L.bcs_build(2**31, 0, 1, None, None, None, 0, None) == 4
+    assert L.bcs_build(10, 5, 4, None, None, None, 0, None) == 2
+    assert L.bcs_build(10, 0, 11, None, None, None, 0, None) == 2
+    assert L.bcs_build(10, 0, 10, None, None, None, 0, None) == 1
+    assert L.bcs_build(10, 0, 10, 8, None, None, 0, None) == 3   # misaligned pointer
+    assert L.bcs_build(1, 0, 1, None, None, None, 0, None) == 0  # q == 0: nothing to do
+    assert L.bcs_build(10, 3, 3, None, None, None, 0, None) == 0 # empty range
+    assert L.bcs_build_workspace_bytes(2**20 + 1, 0, 2**20 + 1) == 4194560 + 21 * 1048592
+    assert L.bcs_build_workspace_bytes(0, 0, 0) == 0
+    assert L.bcs_build_batch_workspace_bytes(1000, 9000) == 4096 + 9000
     assert L.bcs_expand(10, 0, 0, 10, 16, 16, 16, None) == 1     # n == 0
     assert L.bcs_expand(10, 4, 0, 10, None, 16, 16, None) == 1
     assert L.bcs_expand(10, 4, 0, 10, 16, 16, 8, None) == 3
     assert L.bcs_checksum(16, 8, 2, 16, None) == 3               # first index not a multiple of 4
     assert L.bcs_checksum(16, 8, 0, None, None) == 1
-    assert L.bcs_build_batch(None, None, None, None, 3, 10, 40, 16, None, None) == 1
+    assert L.bcs_build_batch(None, None, None, None, None, 3, 10, 40, 16, None, None, 0, None) == 1
     assert L.bcs_build_to_host(10, 0, 10, None, None, 16, 1024, None) == 1
     assert L.bcs_build_to_host(10, 0, 10, 16, None, 16, 16, None) == 1   # staging too small

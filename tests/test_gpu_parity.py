@@ -34,13 +34,20 @@ def _guards_intact(raw, nbytes, fill=0x5A):
     return bool((raw[:GUARD] == fill).all()) and bool((raw[GUARD + nbytes:] == fill).all())
 
 
-def _build(bcs, p, r0, r1, want_recv=True, want_send=True):
+def _build(bcs, p, r0, r1, want_recv=True, want_send=True, fast=True):
+    """fast=True: with a workspace (skip-code construction); False: self-contained construction."""
     q = bcs.bcs_q(p)
     nb = (r1 - r0) * q
     raw_r, recv = _guarded(nb) if want_recv else (None, None)
     raw_s, send = _guarded(nb) if want_send else (None, None)
-    bcs.bcs_build(p, r0, r1, recv, send)
+    ws = raw_w = None
+    if fast:
+        need = bcs.bcs_build_workspace_bytes(p, r0, r1)
+        raw_w, ws = _guarded(need)
+    bcs.bcs_build(p, r0, r1, recv, send, ws)
     torch.cuda.synchronize()
+    if raw_w is not None:
+        assert _guards_intact(raw_w, ws.numel())
     out = []
     for raw, t in ((raw_r, recv), (raw_s, send)):
         if t is None:
@@ -60,23 +67,33 @@ def test_printed_tables_through_the_gpu(bcs):
         assert np.array_equal(recv, g["recv"]) and np.array_equal(send, g["send"]), name
 
 
-def test_every_p_up_to_1024_single_calls(bcs):
+@pytest.mark.parametrize("fast", [True, False])
+def test_every_p_up_to_1024_single_calls(bcs, fast):
     for p in workloads.small_sweep():
         want_r, want_s = oracle.full_table(p)
-        recv, send = _build(bcs, p, 0, p)
+        recv, send = _build(bcs, p, 0, p, fast=fast)
         assert np.array_equal(recv, want_r), p
         assert np.array_equal(send, want_s), p
 
 
-def test_every_p_up_to_1024_batched_and_simulated(bcs):
+def _batch_ws(bcs, plan, fast):
+    if not fast:
+        return None, None
+    return _guarded(bcs.bcs_build_batch_workspace_bytes(plan.total_ranks, plan.total_entries))
+
+
+@pytest.mark.parametrize("fast", [True, False])
+def test_every_p_up_to_1024_batched_and_simulated(bcs, fast):
     plist = workloads.small_sweep()
     plan = bcs.bcs_batch_plan(plist)
     assert plan.total_ranks == 524799 and plan.total_entries == 5072726
     dev = plan.to("cuda")
     raw_r, recv = _guarded(plan.total_entries)
     raw_s, send = _guarded(plan.total_entries)
-    bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, send)
+    raw_w, ws = _batch_ws(bcs, plan, fast)
+    bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, send, ws)
     torch.cuda.synchronize()
+    assert raw_w is None or _guards_intact(raw_w, ws.numel())
     assert _guards_intact(raw_r, plan.total_entries) and _guards_intact(raw_s, plan.total_entries)
     recv, send = recv.cpu().numpy(), send.cpu().numpy()
     eo = plan.entry_off.tolist()
@@ -95,14 +112,17 @@ def test_every_p_up_to_1024_batched_and_simulated(bcs):
                 assert bcast_sim.simulate(p, n, tab.cpu().numpy()) is None, (p, n)
 
 
-def test_batch_with_trivial_and_duplicate_p(bcs):
+@pytest.mark.parametrize("fast", [True, False])
+def test_batch_with_trivial_and_duplicate_p(bcs, fast):
     plist = [1, 2, 1, 300, 300, 1, 17, 4096, 1]
     plan = bcs.bcs_batch_plan(plist)
     dev = plan.to("cuda")
     raw_r, recv = _guarded(plan.total_entries)
     raw_s, send = _guarded(plan.total_entries)
-    bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, send)
+    raw_w, ws = _batch_ws(bcs, plan, fast)
+    bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, send, ws)
     torch.cuda.synchronize()
+    assert raw_w is None or _guards_intact(raw_w, ws.numel())
     assert _guards_intact(raw_r, plan.total_entries) and _guards_intact(raw_s, plan.total_entries)
     eo = plan.entry_off.tolist()
     for j, p in enumerate(plist):
@@ -114,24 +134,25 @@ def test_batch_with_trivial_and_duplicate_p(bcs):
         assert np.array_equal(send[eo[j]:eo[j + 1]].cpu().numpy().reshape(p, -1), want_s)
     # receive table alone
     raw_r, recv = _guarded(plan.total_entries)
-    bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, None)
+    bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, None, ws)
     torch.cuda.synchronize()
     assert np.array_equal(recv[eo[3]:eo[4]].cpu().numpy().reshape(300, -1), oracle.full_table(300)[0])
 
 
 # ---------------------------------------------------------------- ranges, tails, degenerate
-def test_sub_ranges_ragged_tails_and_single_outputs(bcs):
+@pytest.mark.parametrize("fast", [True, False])
+def test_sub_ranges_ragged_tails_and_single_outputs(bcs, fast):
     p = 100003
     q = oracle.q_of(p)
     want_r, want_s = oracle.full_table(p)
     for r0, r1 in ((0, 1), (0, 255), (0, 257), (1, 258), (777, 1300), (p - 300, p), (p - 1, p),
                    (50000, 50000 + 16 * 3 + 5), (99000, 100003)):
-        recv, send = _build(bcs, p, r0, r1)
+        recv, send = _build(bcs, p, r0, r1, fast=fast)
         assert np.array_equal(recv, want_r[r0:r1]), (r0, r1)
         assert np.array_equal(send, want_s[r0:r1]), (r0, r1)      # partly looked up, partly recomputed
-    recv, _ = _build(bcs, p, 123, 999, want_send=False)
+    recv, _ = _build(bcs, p, 123, 999, want_send=False, fast=fast)
     assert np.array_equal(recv, want_r[123:999])
-    _, send = _build(bcs, p, 123, 999, want_recv=False)           # every send entry recomputed
+    _, send = _build(bcs, p, 123, 999, want_recv=False, fast=fast)
     assert np.array_equal(send, want_s[123:999])
     assert q == 17
 
@@ -139,37 +160,50 @@ def test_sub_ranges_ragged_tails_and_single_outputs(bcs):
 def test_degenerate_sizes_and_errors(bcs):
     L = bcs.lib()
     buf = torch.zeros(64, dtype=torch.int8, device="cuda")
-    bcs.bcs_build(1, 0, 1, buf, buf)                    # q == 0
-    bcs.bcs_build(20, 7, 7, buf, buf)                   # empty range
+    bcs.bcs_build(1, 0, 1, buf, buf, buf)               # q == 0
+    bcs.bcs_build(20, 7, 7, buf, buf, buf)              # empty range
     torch.cuda.synchronize()
     assert int(buf.abs().sum()) == 0
-    recv, send = _build(bcs, 2, 0, 2)
-    assert recv.tolist() == [[-1], [0]] and send.tolist() == [[0], [-1]]
-    recv, send = _build(bcs, 3, 0, 3)
-    want = oracle.full_table(3)
-    assert np.array_equal(recv, want[0]) and np.array_equal(send, want[1])
-    assert L.bcs_build(20, 0, 20, buf.data_ptr() + 1, None, None) == 3
-    assert L.bcs_build(20, 0, 21, buf.data_ptr(), None, None) == 2
-    assert L.bcs_build(0, 0, 0, buf.data_ptr(), None, None) == 2
+    assert bcs.bcs_build_workspace_bytes(1, 0, 1) == 0 and bcs.bcs_build_workspace_bytes(20, 7, 7) == 0
+    assert bcs.bcs_build_workspace_bytes(20, 0, 20) == 256 + 5 * 32
+    for fast in (True, False):
+        recv, send = _build(bcs, 2, 0, 2, fast=fast)
+        assert recv.tolist() == [[-1], [0]] and send.tolist() == [[0], [-1]]
+        recv, send = _build(bcs, 3, 0, 3, fast=fast)
+        want = oracle.full_table(3)
+        assert np.array_equal(recv, want[0]) and np.array_equal(send, want[1])
+    small = torch.zeros(64, dtype=torch.int8, device="cuda")         # too small a workspace:
+    out = torch.zeros(100003 * 17, dtype=torch.int8, device="cuda")  # the slow path must run
+    bcs.bcs_build(100003, 0, 100003, out, None, small)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy().reshape(100003, 17), oracle.full_table(100003)[0])
+    assert int(small.abs().sum()) == 0
+    assert L.bcs_build(20, 0, 20, buf.data_ptr() + 1, None, None, 0, None) == 3
+    assert L.bcs_build(20, 0, 20, buf.data_ptr(), None, buf.data_ptr() + 4, 64, None) == 3
+    assert L.bcs_build(20, 0, 21, buf.data_ptr(), None, None, 0, None) == 2
+    assert L.bcs_build(0, 0, 0, buf.data_ptr(), None, None, 0, None) == 2
     torch.cuda.synchronize()
     assert int(buf.abs().sum()) == 0                    # an error writes nothing
 
 
 def test_p_at_the_upper_limit(bcs):
-    """p = 2^31 - 1 (q = 31): rank arithmetic near 2^32; a few ranges vs the per-rank oracle."""
+    """p = 2^31 - 1 (q = 31): rank arithmetic near 2^32; a few ranges vs the per-rank oracle.
+    (Self-contained construction: the workspace of this p would be 8.6 GB; the skip-code
+    construction at large q is covered by the chunked p = 2^30 - 1 test.)"""
     p = 2**31 - 1
     for r0, r1 in ((0, 300), (2**30 - 100, 2**30 + 200), (p - 300, p)):
         want_r, want_s = oracle.build_range(p, r0, r1)
-        recv, send = _build(bcs, p, r0, r1)
+        recv, send = _build(bcs, p, r0, r1, fast=False)
         assert np.array_equal(recv, want_r), (r0, r1)
         assert np.array_equal(send, want_s), (r0, r1)
 
 
 # ---------------------------------------------------------------- full-size workloads
-def test_single_p_2pow20_plus_1_full_table(bcs):
+@pytest.mark.parametrize("fast", [True, False])
+def test_single_p_2pow20_plus_1_full_table(bcs, fast):
     p = workloads.P_SINGLE
     want_r, want_s = oracle.full_table(p)
-    recv, send = _build(bcs, p, 0, p)
+    recv, send = _build(bcs, p, 0, p, fast=fast)
     assert recv.shape == (p, 21)
     assert np.array_equal(recv, want_r)
     assert np.array_equal(send, want_s)
@@ -180,7 +214,8 @@ def test_build_to_host_matches(bcs):
     q = bcs.bcs_q(p)
     want_r, want_s = oracle.full_table(p)
     nb = p * q
-    stage = torch.empty(2 * ((nb + 255) // 256 * 256), dtype=torch.int8, device="cuda")
+    stage = torch.empty(2 * ((nb + 255) // 256 * 256) + bcs.bcs_build_workspace_bytes(p, 0, p),
+                        dtype=torch.int8, device="cuda")
     hr = torch.zeros(nb, dtype=torch.int8).pin_memory()
     hs = torch.zeros(nb, dtype=torch.int8).pin_memory()
     bcs.bcs_build_to_host(p, 0, p, hr, hs, stage)
@@ -190,6 +225,10 @@ def test_build_to_host_matches(bcs):
     hs.zero_()
     bcs.bcs_build_to_host(p, 100, 5000, None, hs, stage)
     torch.cuda.synchronize()
+    assert np.array_equal(hs.numpy()[: 4900 * q].reshape(4900, q), want_s[100:5000])
+    hs.zero_()
+    bcs.bcs_build_to_host(p, 100, 5000, None, hs, stage[: 2 * ((4900 * q + 255) // 256 * 256)])
+    torch.cuda.synchronize()                                  # no room for a workspace: slow path
     assert np.array_equal(hs.numpy()[: 4900 * q].reshape(4900, q), want_s[100:5000])
 
 
@@ -202,8 +241,11 @@ def test_batched_irregular_sweep_full_size(bcs):
     dev = plan.to("cuda")
     recv = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
     send = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
-    bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, send)
+    ws = torch.empty(bcs.bcs_build_batch_workspace_bytes(plan.total_ranks, plan.total_entries),
+                     dtype=torch.int8, device="cuda")
+    bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, send, ws)
     torch.cuda.synchronize()
+    del ws
     eo = plan.entry_off.tolist()
     order = sorted(range(len(plist)), key=lambda j: plist[j])
     full = set(order[:24] + order[-3:] + order[::300] + list(range(6)))
@@ -294,13 +336,14 @@ def test_large_p_chunked_spot_checked(bcs):
     cap = (1 << 27) * q
     recv = torch.empty(cap, dtype=torch.int8, device="cuda")
     send = torch.empty(cap, dtype=torch.int8, device="cuda")
+    ws = torch.empty(bcs.bcs_build_workspace_bytes(p, 0, 1 << 27), dtype=torch.int8, device="cuda")
     sums = torch.zeros(4, dtype=torch.int64, device="cuda")
     m64 = 2**64 - 1
     SEND_BASE = 1 << 36                 # entry index at which the send table is taken to start
     checked = 0
     for c, (r0, r1) in enumerate(chunks):
         nb = (r1 - r0) * q
-        bcs.bcs_build(p, r0, r1, recv, send)
+        bcs.bcs_build(p, r0, r1, recv, send, ws)
         bcs.bcs_checksum(recv, r0 * q, sums[0:1], n_entries=nb)
         bcs.bcs_checksum(send, SEND_BASE + r0 * q, sums[1:2], n_entries=nb)
         half = (nb // 2) // 4 * 4
@@ -321,10 +364,10 @@ def test_large_p_chunked_spot_checked(bcs):
         o_r, _ = oracle.build_range(p, r0, r0 + head, want_send=False)
         bcs.bcs_checksum(recv, r0 * q, sums[2:3], n_entries=head * q)
         assert int(sums.cpu()[2]) & m64 == oracle.checksum(o_r, r0 * q)
-        if c in (0, 7):                                   # rebuilt chunk gives the same sums
+        if c in (0, 7):     # rebuilt with the other (self-contained) construction: same sums
             recv.fill_(0)
             send.fill_(0)
-            bcs.bcs_build(p, r0, r1, recv, send)
+            bcs.bcs_build(p, r0, r1, recv, send, None)
             bcs.bcs_checksum(recv, r0 * q, sums[0:1], n_entries=nb)
             bcs.bcs_checksum(send, SEND_BASE + r0 * q, sums[1:2], n_entries=nb)
             again = [int(v) & m64 for v in sums.cpu()]
