@@ -48,6 +48,7 @@ typedef enum {
 #define BCS_BAD_ENTRY 127
 #define BCS_MAX_Q 31
 #define BCS_SKIPS_STRIDE 32   /* words per row of a skips table */
+#define BCS_STATIC_WORKSPACE_BYTES (8u << 20)   /* scratch built into the library, see bcs_build_static */
 
 /* Human-readable name of a status code (static string, never NULL). */
 const char *bcs_status_str(bcs_status st);
@@ -81,6 +82,30 @@ size_t bcs_build_workspace_bytes(uint32_t p, uint64_t r_begin, uint64_t r_end);
 bcs_status bcs_build(uint32_t p, uint64_t r_begin, uint64_t r_end,
                      int8_t *recv_out, int8_t *send_out,
                      void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* bcs_build for callers that have no device memory to offer as a workspace and may not
+ * allocate any (the paper has no counterpart; this is a convenience of the library).  Think of
+ * code that runs after a framework has claimed the whole GPU for its own memory pool, or of a
+ * latency-critical loop in which a cudaMalloc -- which can stall the whole device -- is not
+ * acceptable.  The fast construction of bcs_build runs with its scratch taken from an array of
+ * BCS_STATIC_WORKSPACE_BYTES (8 MiB) that is part of the library's device image: every GPU on
+ * which the library is loaded gives up that much memory until the process exits, whether or
+ * not this function is ever called.  The call itself allocates and frees nothing.
+ *   Limit: bcs_build_workspace_bytes(p, r_begin, r_end) must not exceed
+ *   BCS_STATIC_WORKSPACE_BYTES (all ranks of p up to about 300 000; of a larger p a
+ *   correspondingly shorter range, and none once 4*p alone exceeds the array);
+ *   otherwise BCS_ERR_UNSUPPORTED is returned and nothing is written.  Use bcs_build with
+ *   your own workspace, or with NULL, beyond that.
+ *   First use: the first call on each device asks the CUDA runtime for the array's device
+ *   address (with that device current) and remembers it.  Make that first call outside any
+ *   stream capture.
+ *   Sharing: all calls on a device use the same array.  Two calls whose kernels can overlap
+ *   on the GPU (different streams, or several host threads) race on it and produce garbage;
+ *   order them on one stream or with events.  The array keeps whatever the last call left
+ *   in it; this function needs none of it to be zero and reads only what it has written.
+ * Outputs, range and error codes otherwise as for bcs_build. */
+bcs_status bcs_build_static(uint32_t p, uint64_t r_begin, uint64_t r_end,
+                            int8_t *recv_out, int8_t *send_out, void *cuda_stream);
 
 /* As bcs_build, then copies the tables to HOST memory on the same stream
  * (cudaMemcpyAsync; pinned host memory makes the copies asynchronous).

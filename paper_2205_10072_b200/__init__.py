@@ -13,6 +13,7 @@ from .binding import (  # noqa: F401
     bcs_build,
     bcs_build_batch,
     bcs_build_batch_workspace_bytes,
+    bcs_build_static,
     bcs_build_workspace_bytes,
     bcs_build_to_host,
     bcs_checksum,

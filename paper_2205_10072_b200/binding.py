@@ -48,6 +48,8 @@ def lib():
         L.bcs_build_workspace_bytes.restype = _c.c_size_t
         L.bcs_build.argtypes = [u32, u64, u64, vp, vp, vp, _c.c_size_t, vp]
         L.bcs_build.restype = i32
+        L.bcs_build_static.argtypes = [u32, u64, u64, vp, vp, vp]
+        L.bcs_build_static.restype = i32
         L.bcs_build_to_host.argtypes = [u32, u64, u64, vp, vp, vp, _c.c_size_t, vp]
         L.bcs_build_to_host.restype = i32
         L.bcs_batch_plan.argtypes = [vp, u32, vp, vp, vp, vp]
@@ -107,6 +109,13 @@ def bcs_build(p: int, r_begin: int, r_end: int, recv_out, send_out, workspace=No
     workspace: CUDA tensor of bcs_build_workspace_bytes(...) bytes (fast path) or None."""
     _check(lib().bcs_build(p, r_begin, r_end, _ptr(recv_out), _ptr(send_out), _ptr(workspace),
                            _nbytes(workspace), _stream(stream)), "bcs_build")
+
+
+def bcs_build_static(p: int, r_begin: int, r_end: int, recv_out, send_out, stream=None) -> None:
+    """bcs_build with the library's built-in 8 MiB scratch: for callers that cannot allocate or
+    pass a workspace.  Raises BcsError (BCS_ERR_UNSUPPORTED) when the range needs more."""
+    _check(lib().bcs_build_static(p, r_begin, r_end, _ptr(recv_out), _ptr(send_out),
+                                  _stream(stream)), "bcs_build_static")
 
 
 def bcs_build_to_host(p: int, r_begin: int, r_end: int, recv_host, send_host, stage_dev,

@@ -16,10 +16,17 @@
 //    search done by descending the homeranges; the send schedule is looked up in the rank-major
 //    receive table where the to-processor is inside the call's range and recomputed
 //    (Algorithm 5) where it is not.
+#include <mutex>
+
 #include "bcs_common.cuh"
 
 namespace bcs {
 namespace {
+
+// Scratch of bcs_build_static: lives in the library's device image, so every GPU that loads
+// the library sets these bytes aside until the process ends.  In host code this name is only a
+// handle for cudaGetSymbolAddress, never an address a kernel may be given.
+static __device__ __align__(256) unsigned char g_static_scratch[BCS_STATIC_WORKSPACE_BYTES];
 
 // ================================================================ self-contained path
 // Algorithm 2: peel off the head of the homerange until r is a skip itself.
@@ -509,6 +516,44 @@ bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_
         if ((st = launch_status()) != BCS_OK) return st;
     }
     return BCS_OK;
+}
+
+// Device address of g_static_scratch on the current device, looked up once per device (with that
+// device current) and remembered; nullptr if the runtime refuses.
+static void *static_scratch_address()
+{
+    constexpr int kMaxDevices = 64;
+    static std::mutex lock;
+    static void *known[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return nullptr;
+    std::lock_guard<std::mutex> guard(lock);
+    if (dev < kMaxDevices && known[dev] != nullptr) return known[dev];
+    void *ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return nullptr;
+    }
+    if (dev < kMaxDevices) known[dev] = ptr;
+    return ptr;
+}
+
+bcs_status bcs_build_static(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_out,
+                            int8_t *send_out, void *cuda_stream)
+{
+    bcs_status st = check_range(p, r_begin, r_end);
+    if (st != BCS_OK) return st;
+    if (bcs_build_workspace_bytes(p, r_begin, r_end) > (size_t)BCS_STATIC_WORKSPACE_BYTES)
+        return BCS_ERR_UNSUPPORTED;          // needs more scratch than the library carries
+    const uint64_t count = r_end - r_begin;
+    if (count == 0 || ceil_log2_u32(p) == 0) return BCS_OK;
+    void *scratch = static_scratch_address();
+    if (scratch == nullptr) return BCS_ERR_CUDA;
+    // Nothing in the scratch has to start at zero: the codes of all p ranks and the round-major
+    // rows of the range are written by this call before anything reads them, so whatever an
+    // earlier call left behind is simply overwritten or never looked at.
+    return bcs_build(p, r_begin, r_end, recv_out, send_out, scratch, BCS_STATIC_WORKSPACE_BYTES,
+                     cuda_stream);
 }
 
 }  // extern "C"
