@@ -176,11 +176,27 @@ send_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, BatchArgs ba,
 }
 
 // ================================================================ workspace path
-// Skip code of every rank: codes[g] for the flattened rank g (single p: g = x).
+// Skip code of every rank: codes[g] for the flattened rank g (single p: g = x).  For a single
+// p the scan over the levels is unrolled, so every skip is an immediate operand from the
+// kernel parameters; levels at and above q never match (a rank is below skips[q] = p).
 template <bool kBatch>
 __global__ void __launch_bounds__(kTile)
 codes_kernel(PTable tab, BatchArgs ba, uint32_t *__restrict__ codes)
 {
+    if (!kBatch) {
+        const uint64_t g = (uint64_t)blockIdx.x * kTile + threadIdx.x;
+        if (g >= tab.p) return;
+        uint32_t x = (uint32_t)g, code = 0;
+#pragma unroll
+        for (int k = BCS_MAX_Q - 1; k >= 0; --k) {
+            if (k < tab.q && x >= tab.s[k]) {
+                x -= tab.s[k];
+                code |= 1u << k;
+            }
+        }
+        codes[g] = code;
+        return;
+    }
     __shared__ TileShared sh;
     RankCtx c = resolve_rank<kBatch>(sh, tab, 0, tab.p, ba);
     if (c.valid) codes[c.rank0 + c.r] = skip_code(c.s, c.q, c.r);
@@ -216,35 +232,75 @@ __device__ __forceinline__ int pick_block(uint32_t X, uint32_t F, uint32_t B,
     return U ? 31 - __clz(U) : -1;
 }
 
-// Second window of Algorithm 4, ranks r - sum_{j<=i} skips[j] .. r - skips[i+1] (cyclic, the
-// root contributes nothing): largest block not in B, or -1.
-__device__ __noinline__ int pick_second_window(const uint32_t *codes, const uint32_t *full,
-                                               uint32_t p, int q, uint32_t r,
-                                               unsigned long long sum, uint32_t hi_skip,
-                                               uint32_t B)
+// Second window of Algorithm 4: the ranks r - sum_{j<=i} skips[j] .. r - skips[i+1] (cyclic, the
+// root contributes nothing), i.e. the `len` ranks that end at rank `below` = r - skips[i+1]
+// mod p, whose code is `lower`.  len = sum_{j<=i} skips[j] - skips[i+1] + 1 is at most q + 1
+// (Lemma 1), so apart from the ranks next to the root the window does not wrap and one more
+// code, that of the rank just before the window, decides it.  Largest block not in B, or -1.
+__device__ __forceinline__ int pick_second_window(const uint32_t *codes, const uint32_t *full,
+                                                  uint32_t p, int q, uint32_t below,
+                                                  uint32_t lower, uint32_t len, uint32_t B)
 {
-    const long long lo = (long long)r - (long long)sum, hi = (long long)r - (long long)hi_skip;
-    const long long len = hi - lo + 1;
-    if (len <= 0) return -1;
-    if (len >= (long long)p) {
+    if (len == 0) return -1;
+    if (len >= p) {
         const uint32_t U = (q >= 32 ? 0xffffffffu : (1u << q) - 1u) & ~B;
         return U ? 31 - __clz(U) : -1;
     }
-    long long a = lo % (long long)p;
-    if (a < 0) a += p;
-    long long e = a + len - 1;
-    if (a == 0) a = 1;
-    if (e < (long long)p)
-        return a <= e ? pick_block(codes[a - 1], codes[e], B, full) : -1;
-    const int b1 = pick_block(codes[a - 1], full[q], B, full);     // a .. p-1 (code of p-1)
-    e -= p;
-    const int b2 = e >= 1 ? pick_block(0u, codes[e], B, full) : -1;  // 1 .. e
+    if (below >= len)                      // ranks below-len+1 .. below, all >= 1
+        return pick_block(codes[below - len], lower, B, full);
+    // the window reaches the root: ranks p-(len-below)+1 .. p-1 (if any), then 1 .. below
+    const uint32_t over = len - below;     // >= 1 ranks at or before the root
+    const int b1 = over >= 2 ? pick_block(codes[p - over], full[q], B, full) : -1;
+    const int b2 = below >= 1 ? pick_block(0u, lower, B, full) : -1;
     return b1 > b2 ? b1 : b2;
 }
 
+// What a round does when its first head is already in B (or its window is empty): the full
+// search of the first window, then the second window.  Kept out of line: a few percent of the
+// rounds come here.
+__device__ __noinline__ int pick_rest(const uint32_t *codes, const uint32_t *full, uint32_t p,
+                                      int q, uint32_t below, uint32_t lower, uint32_t upper,
+                                      uint32_t len, uint32_t B)
+{
+    int blk = pick_block(lower, upper, B, full);
+    if (blk < 0) blk = pick_second_window(codes, full, p, q, below, lower, len, B);
+    return blk;
+}
+
+// One round of Algorithm 4 on skip codes.  The window of round i is bounded by the ranks
+// r - skips[i+1] and r - skips[i] (mod p; both wrapped when i is past the home round, neither
+// before it), and the first head of pick_block -- the highest level at which their codes
+// differ -- is new in all but a few percent of the rounds, so that case is decided here.
+struct RoundState {
+    uint32_t B, upper, sum, lo_skip;
+};
+
+__device__ __forceinline__ int recv_round(const uint32_t *__restrict__ codes, const uint32_t *full,
+                                          uint32_t p, int q, uint32_t r, int i, int h, int bb,
+                                          uint32_t hi_skip, RoundState &st)
+{
+    st.sum += st.lo_skip;                                    // sum_{j<=i} skips[j] < p + q
+    const uint32_t below = r - hi_skip + (r >= hi_skip ? 0u : p);   // r - skips[i+1] mod p
+    const uint32_t lower = codes[below];
+    const uint32_t diff = lower ^ st.upper;
+    int blk = 31 - __clz(diff);                              // first head; -1 for an empty window
+    const bool taken = diff == 0 || ((st.B >> blk) & 1u);
+    const uint32_t upper = st.upper;
+    st.upper = lower;
+    st.lo_skip = hi_skip;
+    if (i == h) return bb;
+    if (taken) {
+        blk = pick_rest(codes, full, p, q, below, lower, upper, st.sum - hi_skip + 1u, st.B);
+        if (blk < 0) return BCS_BAD_ENTRY;
+    }
+    st.B |= 1u << blk;
+    return blk - q;
+}
+
 // Algorithm 4 on skip codes: rounds 0..last of rank r of a p whose codes start at `codes`.
-// row (shared memory, q bytes) and col (round-major copy, element k at col[k * col_stride])
-// receive the entries when not null; the entry of round `last` is returned.
+// kRowOut: entries go to row[0..last] (shared memory); kColOut: entry k also goes to
+// col[k * col_stride] (round-major copy).  The entry of round `last` is returned.
+template <bool kRowOut, bool kColOut>
 __device__ __forceinline__ int recv_rounds_codes(const uint32_t *__restrict__ codes,
                                                  const uint32_t *s, const uint32_t *full,
                                                  uint32_t p, int q, uint32_t r, int last,
@@ -252,42 +308,31 @@ __device__ __forceinline__ int recv_rounds_codes(const uint32_t *__restrict__ co
 {
     const uint32_t own = codes[r];
     int h = -1, bb = 0;
-    uint32_t B = 0;
+    RoundState st;
+    st.B = 0;
     if (r > 0) {
         h = 31 - __clz(own);          // homerange: highest term
         bb = __ffs(own) - 1;          // baseblock: lowest term (Algorithm 2)
-        B = 1u << bb;
+        st.B = 1u << bb;
     }
-    unsigned long long sum = 0;
+    st.sum = 0;
+    st.lo_skip = 1u;                                        // skips[0]
+    st.upper = codes[r >= 1u ? r - 1u : p - 1u];          // code of r - skips[0]
     int entry = 0;
-    uint32_t upper = codes[r >= 1u ? r - 1u : p - 1u];      // code of r - skips[0]
     for (int i = 0; i <= last; ++i) {
-        const uint32_t lo_skip = s[i], hi_skip = s[i + 1];
-        sum += lo_skip;
-        const uint32_t below = r >= hi_skip ? r - hi_skip : r + p - hi_skip;
-        const uint32_t lower = codes[below];                 // code of r - skips[i+1] (mod p)
-        if (i == h) {
-            entry = bb;
-        } else {
-            int blk = pick_block(lower, upper, B, full);
-            if (blk < 0) blk = pick_second_window(codes, full, p, q, r, sum, hi_skip, B);
-            if (blk < 0) {
-                entry = BCS_BAD_ENTRY;
-            } else {
-                B |= 1u << blk;
-                entry = blk - q;
-            }
+        entry = recv_round(codes, full, p, q, r, i, h, bb, s[i + 1], st);
+        if (kRowOut) row[i] = (uint8_t)entry;
+        if (kColOut) {
+            *col = (int8_t)entry;
+            col += col_stride;
         }
-        upper = lower;
-        if (row) row[i] = (uint8_t)entry;
-        if (col) col[(uint64_t)i * col_stride] = (int8_t)entry;
     }
     return entry;
 }
 
 // recv_t: round-major copy.  Single p: recv_t[k * t_stride + (r - r_begin)].
 // Batch: recv_t[entry_off[j] + k * p_j + r].
-template <bool kBatch>
+template <bool kBatch, bool kRowOut, bool kColOut>
 __global__ void __launch_bounds__(kTile)
 recv_codes_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, BatchArgs ba,
                   const uint32_t *__restrict__ codes, int8_t *recv_out, int8_t *recv_t,
@@ -299,23 +344,136 @@ recv_codes_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, BatchArgs ba,
     if (c.valid && c.q > 0) {
         int8_t *col = nullptr;
         uint64_t stride = 0;
-        if (recv_t != nullptr) {
+        if (kColOut) {
             col = kBatch ? recv_t + ba.entry_off[c.pj] + c.r : recv_t + (c.r - r_begin);
             stride = kBatch ? (uint64_t)c.p : t_stride;
         }
-        uint8_t *row = recv_out ? sh.stage + shift + (c.entry - sh.span_begin) : nullptr;
-        recv_rounds_codes(codes + c.rank0, c.s, c.full, c.p, c.q, c.r, c.q - 1, row, col, stride);
+        uint8_t *row = kRowOut ? sh.stage + shift + (c.entry - sh.span_begin) : nullptr;
+        recv_rounds_codes<kRowOut, kColOut>(codes + c.rank0, c.s, c.full, c.p, c.q, c.r, c.q - 1,
+                                            row, col, stride);
     }
-    if (recv_out != nullptr) {
+    if (kRowOut) {
         __syncthreads();
         flush_span(sh.stage, shift, (uint32_t)(sh.span_end - sh.span_begin), recv_out,
                    sh.span_begin);
     }
 }
 
-// Send rows from the round-major receive copy; to-processors outside the call's range
-// (single p, sub-range) are recomputed from the codes (Algorithm 5).
-template <bool kBatch>
+// Single p, p >= 64: the same rows with the first rounds done by the whole warp.  A warp holds 32
+// consecutive ranks, and the windows of the rounds with skips[i+1] <= 33 reach at most 32
+// ranks back, so every baseblock they can contain is the lowest code bit of a rank held by
+// this warp's lanes (rank r of each lane) or by the 32 ranks before them (one more load per
+// lane): the window sets of those rounds -- and of their second windows while
+// sum_{j<=i} skips[j] <= 32 -- are OR-ed together from warp shuffles, one per distance, the
+// same for all lanes.  These are the rounds in which neighbouring ranks disagree about which
+// path of the code search they take; the later rounds run the code search per lane.
+template <bool kRowOut, bool kColOut>
+__global__ void __launch_bounds__(kTile)
+recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uint64_t r_end,
+                       const uint32_t *__restrict__ codes, int8_t *recv_out, int8_t *recv_t,
+                       uint64_t t_stride)
+{
+    __shared__ __align__(16) uint8_t stage[kTile * 32];
+    __shared__ uint32_t full_sh[kRow];
+    constexpr unsigned kAll = 0xffffffffu;
+    const uint32_t p = tab.p;
+    const int q = tab.q;
+    if (threadIdx.x < kRow) full_sh[threadIdx.x] = tab.full[threadIdx.x];
+    __syncthreads();
+    const uint64_t count = r_end - r_begin;
+    const uint64_t g0 = (uint64_t)blockIdx.x * kTile;
+    const uint64_t g = g0 + threadIdx.x;
+    const bool valid = g < count;
+    const uint32_t lane = threadIdx.x & 31u;
+    // ranks of this lane and of the lane 32 ranks before it, mod p (defined for every lane of the
+    // warp, also past the end of the range: only lower lanes and `before` are read by others)
+    uint64_t wrapped = r_begin + g;
+    while (wrapped >= p) wrapped -= p;
+    const uint32_t r = (uint32_t)wrapped;
+    const uint32_t r_before = r >= 32u ? r - 32u : r + p - 32u;
+    const uint32_t own = codes[r];
+    const uint32_t before = codes[r_before];
+    const uint32_t own_bit = own & (0u - own);            // baseblock of r as a bit, 0 for the root
+    const uint32_t before_bit = before & (0u - before);
+    int h = -1, bb = 0;
+    RoundState st;
+    st.B = 0;
+    if (r > 0) {
+        h = 31 - __clz(own);
+        bb = __ffs(own) - 1;
+        st.B = own_bit;
+    }
+    st.sum = 0;
+    uint8_t *row = stage + threadIdx.x * q;
+    int8_t *col = kColOut ? recv_t + g : nullptr;
+    int i = 0;
+#pragma unroll 1
+    for (; i < q && tab.s[i + 1] <= 33u; ++i) {            // uniform over the grid
+        const uint32_t lo = tab.s[i], hi = tab.s[i + 1];
+        st.sum += lo;
+        uint32_t acc = 0;
+        for (uint32_t d = lo; d < hi; ++d) {                // ranks r - d, d = skips[i]..skips[i+1]-1
+            const uint32_t a = __shfl_up_sync(kAll, own_bit, d);
+            const uint32_t b = __shfl_down_sync(kAll, before_bit, 32u - d);
+            acc |= lane >= d ? a : b;
+        }
+        uint32_t U = acc & ~st.B;
+        const bool second = U == 0 && i != h;
+        if (__any_sync(kAll, second)) {
+            if (st.sum <= 32u) {                             // ranks r - d, d = skips[i+1]..sum
+                uint32_t acc2 = 0;
+                for (uint32_t d = hi; d <= st.sum; ++d) {
+                    const uint32_t a = __shfl_up_sync(kAll, own_bit, d);
+                    const uint32_t b = __shfl_down_sync(kAll, before_bit, 32u - d);
+                    acc2 |= lane >= d ? a : b;
+                }
+                if (second) U = acc2 & ~st.B;
+            } else if (second) {
+                const uint32_t below = r - hi + (r >= hi ? 0u : p);
+                const int b2 = pick_second_window(codes, full_sh, p, q, below, codes[below],
+                                                  st.sum - hi + 1u, st.B);
+                U = b2 >= 0 ? 1u << b2 : 0u;
+            }
+        }
+        int entry;
+        if (i == h) {
+            entry = bb;
+        } else if (U == 0) {
+            entry = BCS_BAD_ENTRY;
+        } else {
+            const int blk = 31 - __clz(U);
+            st.B |= 1u << blk;
+            entry = blk - q;
+        }
+        if (kRowOut) row[i] = (uint8_t)entry;
+        if (kColOut && valid) *col = (int8_t)entry;
+        if (kColOut) col += t_stride;
+    }
+    if (valid && i < q) {
+        const uint32_t edge = tab.s[i];
+        st.lo_skip = edge;
+        st.upper = codes[r - edge + (r >= edge ? 0u : p)];  // code of r - skips[i]
+#pragma unroll 1
+        for (; i < q; ++i) {
+            const int entry = recv_round(codes, full_sh, p, q, r, i, h, bb, tab.s[i + 1], st);
+            if (kRowOut) row[i] = (uint8_t)entry;
+            if (kColOut) {
+                *col = (int8_t)entry;
+                col += t_stride;
+            }
+        }
+    }
+    if (kRowOut) {
+        __syncthreads();
+        const uint64_t g1 = g0 + kTile < count ? g0 + kTile : count;
+        flush_span(stage, 0, (uint32_t)((g1 - g0) * (uint64_t)q), recv_out, g0 * (uint64_t)q);
+    }
+}
+
+// Send rows from the round-major receive copy.  kAllInside: every to-processor's row is in
+// the copy (all ranks of the p).  Otherwise (single p, sub-range) to-processors outside the
+// range are recomputed from the codes (Algorithm 5).
+template <bool kBatch, bool kAllInside>
 __global__ void __launch_bounds__(kTile)
 send_rm_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, BatchArgs ba,
                const uint32_t *__restrict__ codes, const int8_t *__restrict__ recv_t,
@@ -328,22 +486,109 @@ send_rm_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, BatchArgs ba,
         uint8_t *row = sh.stage + shift + (c.entry - sh.span_begin);
         const int8_t *tbl = kBatch ? recv_t + ba.entry_off[c.pj] : recv_t;
         const uint64_t stride = kBatch ? (uint64_t)c.p : t_stride;
-        for (int k = 0; k < c.q; ++k) {
-            uint32_t t = c.r + c.s[k];
-            if (t >= c.p) t -= c.p;
-            int v;
-            if (kBatch) {
-                v = tbl[(uint64_t)k * stride + t];
-            } else if (t >= r_begin && t < r_end) {
-                v = tbl[(uint64_t)k * stride + (t - r_begin)];
-            } else {
-                v = recv_rounds_codes(codes, c.s, c.full, c.p, c.q, t, k, nullptr, nullptr, 0);
+        if (kAllInside) {
+            for (int k0 = 0; k0 < c.q; k0 += 8) {
+                int v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int k = k0 + j < c.q ? k0 + j : c.q - 1;
+                    uint32_t t = c.r + c.s[k];
+                    if (t >= c.p) t -= c.p;
+                    v[j] = tbl[(uint64_t)k * stride + t];
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (k0 + j < c.q) row[k0 + j] = (uint8_t)v[j];
             }
-            row[k] = (uint8_t)v;
+        } else {
+            const uint32_t first = (uint32_t)r_begin, width = (uint32_t)(r_end - r_begin);
+            for (int k = 0; k < c.q; ++k) {
+                uint32_t t = c.r + c.s[k];
+                if (t >= c.p) t -= c.p;
+                const uint32_t rel = t - first;          // index into the round-major row
+                int v;
+                if (rel < width) {
+                    v = tbl[rel];
+                } else {
+                    v = recv_rounds_codes<false, false>(codes, c.s, c.full, c.p, c.q, t, k, nullptr,
+                                                        nullptr, 0);
+                }
+                row[k] = (uint8_t)v;
+                tbl += stride;
+            }
         }
     }
     __syncthreads();
     flush_span(sh.stage, shift, (uint32_t)(sh.span_end - sh.span_begin), send_out, sh.span_begin);
+}
+
+// All ranks of a single p: row k of the round-major send table is row k of the round-major
+// receive copy rotated by skips[k] (sendsched[r][k] = recvsched[(r+skips[k]) mod p][k]), so
+// the send table is a transposition with one rotation per row.  A CTA takes 256 consecutive
+// ranks: for every round it copies the 256 (rotated, possibly wrapping) bytes it needs with
+// 16-byte loads into shared memory, then every thread gathers its column into the rank-major
+// staging rows, which leave as one vectorised span.
+constexpr int kTrPitch = kTile + 32;      // bytes per round in shared memory: 256 + alignment slack
+
+__global__ void __launch_bounds__(kTile)
+send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restrict__ recv_t,
+                      uint64_t t_stride, int8_t *send_out)
+{
+    __shared__ __align__(16) uint8_t rounds[BCS_MAX_Q * kTrPitch];
+    __shared__ __align__(16) uint8_t stage[kTile * 32];
+    __shared__ uint32_t lead[BCS_MAX_Q];   // offset of the tile's first byte inside its pitch row
+    __shared__ uint32_t wraps;             // rounds whose 256 bytes pass the end of the row
+    const uint32_t p = tab.p;
+    const int q = tab.q;
+    const uint32_t r0 = blockIdx.x * kTile;
+    const uint32_t n = p - r0 < (uint32_t)kTile ? p - r0 : (uint32_t)kTile;   // ranks of this tile
+    if (threadIdx.x == 0) wraps = 0;
+    __syncthreads();
+    // one 16-byte piece per (round, vector): kTrPitch / 16 = 18 vectors cover 256 bytes at any
+    // misalignment.  The tile's bytes of round k are recv_t[k][(r0 + skips[k] + j) mod p], j < n:
+    // one run, or two when it passes the end of the row.
+    const int vecs = kTrPitch / 16;
+    for (int w = threadIdx.x; w < q * vecs; w += kTile) {
+        const int k = w / vecs, v = w - k * vecs;
+        const uint8_t *src_row = reinterpret_cast<const uint8_t *>(recv_t) + (uint64_t)k * t_stride;
+        uint32_t start = r0 + tab.s[k];
+        if (start >= p) start -= p;
+        const uint32_t mis = start & 15u;                 // rows start 16-byte aligned (t_stride % 16 == 0)
+        const uint32_t run = p - start < n ? p - start : n;      // bytes before the wrap
+        if (v == 0) {
+            lead[k] = mis;
+            if (run < n) atomicOr(&wraps, 1u << k);
+        }
+        uint8_t *dst = rounds + k * kTrPitch + v * 16;
+        const uint32_t at = start - mis + (uint32_t)v * 16u;      // aligned position in the row
+        if (at < start + run)                                     // at + 16 <= t_stride follows
+            *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src_row + at);
+    }
+    __syncthreads();
+    for (uint32_t left = wraps; left != 0; left &= left - 1u) {  // the part after the wrap, by bytes
+        const int k = __ffs(left) - 1;
+        uint32_t start = r0 + tab.s[k];
+        if (start >= p) start -= p;
+        const uint32_t run = p - start;                           // < n for these rounds
+        const uint8_t *src_row = reinterpret_cast<const uint8_t *>(recv_t) + (uint64_t)k * t_stride;
+        const uint32_t j = threadIdx.x;
+        if (j >= run && j < n) rounds[k * kTrPitch + (start & 15u) + j] = src_row[j - run];
+    }
+    if (wraps) __syncthreads();
+    {
+        // lane l of warp w takes rank 128 * (w / 4) + 4 * l + (w % 4): the rows written by one
+        // warp start q * 4 bytes = q words apart, which is a different bank for every lane when q
+        // is odd, and the bytes it reads lie in 32 consecutive words.
+        const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+        const uint32_t mine = 128u * (warp >> 2) + 4u * lane + (warp & 3u);
+        if (mine < n) {
+            uint8_t *row = stage + mine * q;
+            const uint8_t *column = rounds + mine;
+            for (int k = 0; k < q; ++k) row[k] = column[k * kTrPitch + lead[k]];
+        }
+    }
+    __syncthreads();
+    flush_span(stage, 0, n * (uint32_t)q, send_out, (uint64_t)r0 * (uint64_t)q);
 }
 
 struct Workspace {
@@ -409,13 +654,37 @@ bcs_status bcs_build(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_
         codes_kernel<false><<<(unsigned)((p + kTile - 1) / kTile), kTile, 0, stream>>>(tab, none,
                                                                                       ws.codes);
         if ((st = launch_status()) != BCS_OK) return st;
-        recv_codes_kernel<false><<<blocks, kTile, 0, stream>>>(
-            tab, r_begin, r_end, none, ws.codes, recv_out, send_out ? ws.recv_t : nullptr,
-            ws.t_stride);
+        const bool warp_rounds = p >= 64;      // the warp-cooperative kernel needs 32 ranks back
+        if (recv_out != nullptr && send_out != nullptr) {
+            if (warp_rounds)
+                recv_codes_warp_kernel<true, true><<<blocks, kTile, 0, stream>>>(
+                    tab, r_begin, r_end, ws.codes, recv_out, ws.recv_t, ws.t_stride);
+            else
+                recv_codes_kernel<false, true, true><<<blocks, kTile, 0, stream>>>(
+                    tab, r_begin, r_end, none, ws.codes, recv_out, ws.recv_t, ws.t_stride);
+        } else if (recv_out != nullptr) {
+            if (warp_rounds)
+                recv_codes_warp_kernel<true, false><<<blocks, kTile, 0, stream>>>(
+                    tab, r_begin, r_end, ws.codes, recv_out, nullptr, 0);
+            else
+                recv_codes_kernel<false, true, false><<<blocks, kTile, 0, stream>>>(
+                    tab, r_begin, r_end, none, ws.codes, recv_out, nullptr, 0);
+        } else {
+            if (warp_rounds)
+                recv_codes_warp_kernel<false, true><<<blocks, kTile, 0, stream>>>(
+                    tab, r_begin, r_end, ws.codes, nullptr, ws.recv_t, ws.t_stride);
+            else
+                recv_codes_kernel<false, false, true><<<blocks, kTile, 0, stream>>>(
+                    tab, r_begin, r_end, none, ws.codes, nullptr, ws.recv_t, ws.t_stride);
+        }
         if ((st = launch_status()) != BCS_OK) return st;
         if (send_out != nullptr) {
-            send_rm_kernel<false><<<blocks, kTile, 0, stream>>>(tab, r_begin, r_end, none, ws.codes,
-                                                                ws.recv_t, ws.t_stride, send_out);
+            if (count == p)
+                send_transpose_kernel<<<blocks, kTile, 0, stream>>>(tab, ws.recv_t, ws.t_stride,
+                                                                    send_out);
+            else
+                send_rm_kernel<false, false><<<blocks, kTile, 0, stream>>>(
+                    tab, r_begin, r_end, none, ws.codes, ws.recv_t, ws.t_stride, send_out);
             if ((st = launch_status()) != BCS_OK) return st;
         }
         return BCS_OK;
@@ -499,12 +768,16 @@ bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_
         int8_t *recv_t = static_cast<int8_t *>(workspace) + align_up(4ull * total_ranks, 256);
         codes_kernel<true><<<blocks, kTile, 0, stream>>>(none, ba, codes);
         if ((st = launch_status()) != BCS_OK) return st;
-        recv_codes_kernel<true><<<blocks, kTile, 0, stream>>>(none, 0, 0, ba, codes, recv_out,
-                                                              send_out ? recv_t : nullptr, 0);
+        if (send_out != nullptr)
+            recv_codes_kernel<true, true, true><<<blocks, kTile, 0, stream>>>(none, 0, 0, ba, codes,
+                                                                              recv_out, recv_t, 0);
+        else
+            recv_codes_kernel<true, true, false><<<blocks, kTile, 0, stream>>>(none, 0, 0, ba, codes,
+                                                                               recv_out, nullptr, 0);
         if ((st = launch_status()) != BCS_OK) return st;
         if (send_out != nullptr) {
-            send_rm_kernel<true><<<blocks, kTile, 0, stream>>>(none, 0, 0, ba, codes, recv_t, 0,
-                                                               send_out);
+            send_rm_kernel<true, true><<<blocks, kTile, 0, stream>>>(none, 0, 0, ba, codes, recv_t,
+                                                                     0, send_out);
             if ((st = launch_status()) != BCS_OK) return st;
         }
         return BCS_OK;
