@@ -369,13 +369,13 @@ def run_ours(args) -> None:
 
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of the
 # current kernels); None until counters have been taken for the kernel as it stands.
-RECV_TRAFFIC_BYTES = None
-EXPAND_TRAFFIC_BYTES = None
+RECV_TRAFFIC_BYTES = 4212224 + 185088        # recv_codes_warp_kernel<true,true>, p = 2^20+1
+EXPAND_TRAFFIC_BYTES = 1567312000 + 3457280   # expand_kernel, p = 100003, n = 1000
 
 # integer operations per rank of the receive-schedule construction that the kernels run, by q:
-# skip code (3 per level + 5) + per round 22 (two address selects, code load, one step of the
-# head search, set update, entry, two stores, loop) + the measured extra 0.66 search steps and
-# 0.19 second windows per rank (CPU count of the same loops over sampled ranks of p = 2^20+1).
+# skip code (3 per level + 5) + per round 22 (address select, code load, one step of the head
+# search, set update, entry, two stores, loop) + the measured extra 0.66 search steps and 0.19
+# second windows per rank (CPU count of the same loops over sampled ranks of p = 2^20+1).
 ALU_MODEL = {21: (3 * 21 + 5) + 22 * 21 + 14}
 
 
