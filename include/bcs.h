@@ -161,6 +161,27 @@ bcs_status bcs_expand(uint32_t p, uint32_t n, uint64_t r_begin, uint64_t r_end,
                       const int8_t *recv, const int8_t *send, int32_t *table_out,
                       void *cuda_stream);
 
+/* Counts the ranks of r_begin..r_end-1 whose rows break a property that every schedule of the
+ * construction has (text after Theorem 1; Algorithms 4, 5 and 9) -- a check that scales to
+ * tables far too large to compare entry by entry:
+ *   violations_dev[0]  receive row: the home round (skips[h] <= r < skips[h+1]) must hold the
+ *                      baseblock of r (Algorithm 2), every other round a negative entry b-q,
+ *                      the q-1 blocks b different from each other and from the baseblock; for
+ *                      the root q different negative entries;
+ *   violations_dev[1]  send row: the root sends block k in round k; any other rank sends a
+ *                      previous-phase block that it received in an earlier round of the row,
+ *                      or its own baseblock of the previous phase, or -- in the rounds after
+ *                      its home round -- its baseblock (without recv only "some previous-phase
+ *                      block" can be checked for the first two);
+ *   violations_dev[2]  pairing: send[r][k] == recv[(r+skips[k]) mod p][k] wherever the
+ *                      to-processor lies inside the range (needs both tables).
+ * recv, send: device int8 rows of the ranks of the range as bcs_build writes them, 16-byte
+ * aligned, either may be NULL (its checks are skipped).  violations_dev: device, three uint64,
+ * overwritten.  Baseblocks are recomputed with Algorithm 2, independently of bcs_build. */
+bcs_status bcs_validate(uint32_t p, uint64_t r_begin, uint64_t r_end,
+                        const int8_t *recv, const int8_t *send,
+                        uint64_t *violations_dev, void *cuda_stream);
+
 /* Position-weighted 64-bit checksum of a stretch of schedule entries, additive
  * over disjoint stretches (no counterpart in the paper; used to compare outputs
  * that are too large to copy back).  The bytes are read as little-endian 32-bit

@@ -66,6 +66,9 @@ def _load():
         lib.bcso_expand_range.restype = None
         lib.bcso_checksum.argtypes = [i8p, c.c_uint64, c.c_uint64]
         lib.bcso_checksum.restype = c.c_uint64
+        lib.bcso_validate.argtypes = [c.c_uint32, c.c_uint64, c.c_uint64, i8p, i8p,
+                                      c.POINTER(c.c_uint64)]
+        lib.bcso_validate.restype = None
         lib.bcso_set_root_mode.argtypes = [c.c_int]
         lib.bcso_set_root_mode.restype = None
         lib.bcso_num_threads.argtypes = []
@@ -193,6 +196,20 @@ def checksum(buf: np.ndarray, first_index: int = 0) -> int:
     """Order-independent 64-bit checksum of int8 entries (not from the paper)."""
     buf = np.ascontiguousarray(buf, dtype=np.int8).reshape(-1)
     return int(_load().bcso_checksum(_i8(buf), buf.shape[0], first_index))
+
+
+def validate(p: int, r_begin: int, r_end: int, recv, send):
+    """Ranks of the range whose rows break the promised properties -> (bad receive rows,
+    bad send rows, send/receive mismatches); recv/send are [r_end-r_begin][q] or None."""
+    q = q_of(p)
+    n = r_end - r_begin
+    if recv is not None:
+        recv = np.ascontiguousarray(recv, dtype=np.int8).reshape(n, q)
+    if send is not None:
+        send = np.ascontiguousarray(send, dtype=np.int8).reshape(n, q)
+    out = (ctypes.c_uint64 * 3)()
+    _load().bcso_validate(p, r_begin, r_end, _i8(recv), _i8(send), out)
+    return tuple(int(v) for v in out)
 
 
 def set_root_mode(mode: int) -> None:

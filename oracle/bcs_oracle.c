@@ -479,6 +479,72 @@ uint64_t bcso_checksum(const int8_t *buf, uint64_t n_entries, uint64_t first_ind
     return sum;
 }
 
+/* Counts the ranks r_begin..r_end-1 whose rows break what the text after
+ * Theorem 1 and Algorithms 5 / 9 promise (the same three counts the library's
+ * checker reports; recv / send hold the rows of the range, either may be NULL):
+ *   counts[0] receive row: baseblock (Algorithm 2) exactly in the home round,
+ *             all other entries negative, their blocks b = entry + q different
+ *             from each other and from the baseblock;
+ *   counts[1] send row: root sends k in round k; others send a previous-phase
+ *             block received in an earlier round of the row, or the own
+ *             baseblock of the previous phase, or -- after the home round -- the
+ *             baseblock of the current phase;
+ *   counts[2] send[r][k] != recv[(r + skips[k]) mod p][k] for a to-processor
+ *             inside the range. */
+void bcso_validate(uint32_t p, uint64_t r_begin, uint64_t r_end, const int8_t *recv,
+                   const int8_t *send, uint64_t *counts)
+{
+    uint32_t s[BCSO_MAXQ + 1];
+    int q = bcso_skips(p, s);
+    uint64_t j, n = r_end - r_begin;
+    counts[0] = counts[1] = counts[2] = 0;
+    for (j = 0; j < n; j++) {
+        uint32_t r = (uint32_t)(r_begin + j);
+        const int8_t *rr = recv ? recv + j * q : NULL, *sr = send ? send + j * q : NULL;
+        int bb = bcso_baseblock(p, r), h = -1, k, bad;
+        for (k = 0; k < q; k++)
+            if (s[k] <= r && r < s[k + 1]) h = k;
+        if (rr) {
+            int used[BCSO_MAXQ + 1] = {0};
+            bad = 0;
+            if (bb >= 0) used[bb] = 1;
+            for (k = 0; k < q; k++) {
+                if (k == h) {
+                    if (rr[k] != bb) bad = 1;
+                } else {
+                    int b = rr[k] + q;
+                    if (rr[k] >= 0 || b < 0 || used[b]) bad = 1;
+                    else used[b] = 1;
+                }
+            }
+            counts[0] += bad;
+        }
+        if (sr) {
+            int have[BCSO_MAXQ + 1] = {0};
+            bad = 0;
+            if (bb >= 0) have[bb] = 1;
+            for (k = 0; k < q; k++) {
+                if (r == 0) {
+                    if (sr[k] != k) bad = 1;
+                } else if (!(k > h && sr[k] == bb)) {
+                    int b = sr[k] + q;
+                    if (sr[k] >= 0 || b < 0 || (rr && !have[b])) bad = 1;
+                }
+                if (rr && k != h && rr[k] < 0 && rr[k] + q >= 0) have[rr[k] + q] = 1;
+            }
+            counts[1] += bad;
+        }
+        if (rr && sr) {
+            bad = 0;
+            for (k = 0; k < q; k++) {
+                uint64_t t = ((uint64_t)r + s[k]) % p;
+                if (t >= r_begin && t < r_end && recv[(t - r_begin) * q + k] != sr[k]) bad = 1;
+            }
+            counts[2] += bad;
+        }
+    }
+}
+
 int bcso_num_threads(void)
 {
 #ifdef _OPENMP

@@ -21,6 +21,7 @@ from .binding import (  # noqa: F401
     bcs_q,
     bcs_skips,
     bcs_status_str,
+    bcs_validate,
     lib,
     lib_path,
 )

@@ -60,6 +60,8 @@ def lib():
         L.bcs_build_batch.restype = i32
         L.bcs_expand.argtypes = [u32, u32, u64, u64, vp, vp, vp, vp]
         L.bcs_expand.restype = i32
+        L.bcs_validate.argtypes = [u32, u64, u64, vp, vp, vp, vp]
+        L.bcs_validate.restype = i32
         L.bcs_checksum.argtypes = [vp, u64, u64, vp, vp]
         L.bcs_checksum.restype = i32
         _lib = L
@@ -194,6 +196,13 @@ def bcs_expand(p: int, n: int, r_begin: int, r_end: int, recv, send, table_out, 
     [(r_end-r_begin), n-1+q, 4]."""
     _check(lib().bcs_expand(p, n, r_begin, r_end, _ptr(recv), _ptr(send), _ptr(table_out),
                             _stream(stream)), "bcs_expand")
+
+
+def bcs_validate(p: int, r_begin: int, r_end: int, recv, send, violations_out, stream=None) -> None:
+    """recv/send: CUDA int8 rows of the range (or None); violations_out: CUDA int64 tensor with
+    three elements: ranks with a bad receive row, a bad send row, a send/receive mismatch."""
+    _check(lib().bcs_validate(p, r_begin, r_end, _ptr(recv), _ptr(send), _ptr(violations_out),
+                              _stream(stream)), "bcs_validate")
 
 
 def bcs_checksum(buf, first_entry_index: int, sum_out, stream=None, n_entries: int | None = None) -> None:

@@ -406,16 +406,40 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uin
     st.sum = 0;
     uint8_t *row = stage + threadIdx.x * q;
     int8_t *col = kColOut ? recv_t + g : nullptr;
+    // run[j] / run_before[j]: baseblock bits OR-ed over the 2^j ranks ending at this lane's rank,
+    // resp. at the rank 32 below it (doubling; a lane's run may start in the 32 ranks before the
+    // warp).  A window of L ranks is the union of two runs of 2^floor(log2 L) ranks.
+    uint32_t run[5], run_before[5];
+    run[0] = own_bit;
+    run_before[0] = before_bit;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const unsigned w = 1u << j;
+        const uint32_t up = __shfl_up_sync(kAll, run[j], w);
+        const uint32_t wrap = __shfl_down_sync(kAll, run_before[j], 32u - w);
+        const uint32_t up_before = __shfl_up_sync(kAll, run_before[j], w);
+        run[j + 1] = run[j] | (lane >= w ? up : wrap);
+        run_before[j + 1] = run_before[j] | up_before;   // complete for lanes >= 2w - 1, all that is read
+    }
+    // OR over the 2^j ranks ending d ranks below this lane's rank (1 <= d <= 32)
+    auto run_below = [&](int j, uint32_t d) {
+        const uint32_t a = __shfl_up_sync(kAll, run[j], d);
+        const uint32_t b = __shfl_down_sync(kAll, run_before[j], 32u - d);
+        return lane >= d ? a : b;
+    };
     int i = 0;
 #pragma unroll 1
     for (; i < q && tab.s[i + 1] <= 33u; ++i) {            // uniform over the grid
         const uint32_t lo = tab.s[i], hi = tab.s[i + 1];
         st.sum += lo;
-        uint32_t acc = 0;
-        for (uint32_t d = lo; d < hi; ++d) {                // ranks r - d, d = skips[i]..skips[i+1]-1
-            const uint32_t a = __shfl_up_sync(kAll, own_bit, d);
-            const uint32_t b = __shfl_down_sync(kAll, before_bit, 32u - d);
-            acc |= lane >= d ? a : b;
+        // ranks r - d, d = lo..hi-1: runs of 2^j ranks ending at r - lo and at r - (hi - 2^j)
+        uint32_t acc;
+        switch (31 - __clz(hi - lo)) {                      // uniform
+            case 0: acc = run_below(0, lo); break;
+            case 1: acc = run_below(1, lo) | run_below(1, hi - 2u); break;
+            case 2: acc = run_below(2, lo) | run_below(2, hi - 4u); break;
+            case 3: acc = run_below(3, lo) | run_below(3, hi - 8u); break;
+            default: acc = run_below(4, lo) | run_below(4, hi - 16u); break;
         }
         uint32_t U = acc & ~st.B;
         const bool second = U == 0 && i != h;
@@ -450,18 +474,53 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uin
         if (kColOut) col += t_stride;
     }
     if (valid && i < q) {
+        // Per-lane rounds.  Before the home round h both window bounds are r - skip, after it
+        // both are r + p - skip: two loops with the wrap decided once, the home round between.
         const uint32_t edge = tab.s[i];
         st.lo_skip = edge;
         st.upper = codes[r - edge + (r >= edge ? 0u : p)];  // code of r - skips[i]
-#pragma unroll 1
-        for (; i < q; ++i) {
-            const int entry = recv_round(codes, full_sh, p, q, r, i, h, bb, tab.s[i + 1], st);
-            if (kRowOut) row[i] = (uint8_t)entry;
+        uint8_t *out = row + i;
+        auto round = [&](int ii, uint32_t from) {           // from = r or r + p
+            const uint32_t hi = tab.s[ii + 1];
+            st.sum += st.lo_skip;
+            st.lo_skip = hi;
+            const uint32_t below = from - hi;
+            const uint32_t lower = codes[below];
+            const uint32_t diff = lower ^ st.upper;
+            int blk = 31 - __clz(diff);                      // first head; -1 for an empty window
+            int entry;
+            if (diff == 0 || ((st.B >> blk) & 1u)) {
+                blk = pick_rest(codes, full_sh, p, q, below, lower, st.upper, st.sum - hi + 1u, st.B);
+                entry = blk < 0 ? BCS_BAD_ENTRY : blk - q;
+                if (blk >= 0) st.B |= 1u << blk;
+            } else {
+                st.B |= 1u << blk;
+                entry = blk - q;
+            }
+            st.upper = lower;
+            if (kRowOut) *out++ = (uint8_t)entry;
             if (kColOut) {
                 *col = (int8_t)entry;
                 col += t_stride;
             }
+        };
+#pragma unroll 1
+        for (; i < h; ++i) round(i, r);
+        if (i == h) {                                        // home round: the baseblock itself
+            const uint32_t hi = tab.s[i + 1];
+            st.sum += st.lo_skip;
+            st.lo_skip = hi;
+            st.upper = codes[r + p - hi];
+            if (kRowOut) *out++ = (uint8_t)bb;
+            if (kColOut) {
+                *col = (int8_t)bb;
+                col += t_stride;
+            }
+            ++i;
         }
+        const uint32_t rp = r + p;
+#pragma unroll 1
+        for (; i < q; ++i) round(i, rp);
     }
     if (kRowOut) {
         __syncthreads();
@@ -582,9 +641,11 @@ send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restri
         const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
         const uint32_t mine = 128u * (warp >> 2) + 4u * lane + (warp & 3u);
         if (mine < n) {
-            uint8_t *row = stage + mine * q;
-            const uint8_t *column = rounds + mine;
-            for (int k = 0; k < q; ++k) row[k] = column[k * kTrPitch + lead[k]];
+            uint8_t *__restrict__ row = stage + mine * q;
+            const uint8_t *__restrict__ column = rounds + mine;
+            const uint32_t *__restrict__ lead_k = lead;
+#pragma unroll 4
+            for (int k = 0; k < q; ++k) row[k] = column[k * kTrPitch + lead_k[k]];
         }
     }
     __syncthreads();

@@ -1,0 +1,148 @@
+// Checker of the properties that every schedule of the construction has (arXiv 2205.10072,
+// text after Theorem 1 and Algorithm 5), run over tables already on the device.  It uses
+// Algorithm 2 (homerange descent) for the baseblocks, not the skip codes of the fast
+// construction, so that it does not share its arithmetic with what it checks.
+#include "bcs_common.cuh"
+
+namespace bcs {
+namespace {
+
+// Algorithm 2: peel off the head of the homerange until r is a skip itself.
+__device__ __forceinline__ int base_block_of(const uint32_t *s, uint32_t r)
+{
+    for (;;) {
+        const int k = home_of(s, r);
+        const uint32_t v = s[k];
+        if (r == v) return k;
+        r -= v;
+    }
+}
+
+// Copies in[byte0, byte0+len) to stage[shift, shift+len), (byte0 & 15) == shift, `in` 16-byte
+// aligned: the mirror image of flush_span.
+__device__ __forceinline__ void load_span(uint8_t *stage, uint32_t shift, uint32_t len,
+                                          const int8_t *in, uint64_t byte0)
+{
+    const uint8_t *src = reinterpret_cast<const uint8_t *>(in) + (byte0 - shift);
+    const uint32_t end = shift + len;
+    const uint32_t nvec = (end + 15u) >> 4;
+    for (uint32_t v = threadIdx.x; v < nvec; v += blockDim.x) {
+        const uint32_t lo = v << 4, hi = lo + 16u;
+        if (lo >= shift && hi <= end) {
+            *reinterpret_cast<uint4 *>(stage + lo) = *reinterpret_cast<const uint4 *>(src + lo);
+        } else {
+            const uint32_t from = lo < shift ? shift : lo, to = hi > end ? end : hi;
+            for (uint32_t e = from; e < to; ++e) stage[e] = src[e];
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kTile)
+validate_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, const int8_t *__restrict__ recv,
+                const int8_t *__restrict__ send, unsigned long long *violations)
+{
+    __shared__ uint32_t s[kRow];
+    __shared__ __align__(16) uint8_t recv_rows[kTile * 32];
+    __shared__ __align__(16) uint8_t send_rows[kTile * 32];
+    const int q = tab.q;
+    const uint32_t p = tab.p;
+    if (threadIdx.x < kRow) s[threadIdx.x] = tab.s[threadIdx.x];
+    const uint64_t count = r_end - r_begin;
+    const uint64_t g0 = (uint64_t)blockIdx.x * kTile;
+    const uint32_t n = (uint32_t)(count - g0 < (uint64_t)kTile ? count - g0 : (uint64_t)kTile);
+    if (recv) load_span(recv_rows, 0, n * (uint32_t)q, recv, g0 * (uint64_t)q);
+    if (send) load_span(send_rows, 0, n * (uint32_t)q, send, g0 * (uint64_t)q);
+    __syncthreads();
+    unsigned bad_recv = 0, bad_send = 0, bad_pair = 0;
+    if (threadIdx.x < n) {
+        const uint32_t r = (uint32_t)(r_begin + g0 + threadIdx.x);
+        const int8_t *rrow = reinterpret_cast<const int8_t *>(recv_rows) + threadIdx.x * q;
+        const int8_t *srow = reinterpret_cast<const int8_t *>(send_rows) + threadIdx.x * q;
+        int h = -1, bb = -1;
+        if (r > 0) {
+            h = home_of(s, r);
+            bb = base_block_of(s, r);
+        }
+        if (recv) {
+            // the baseblock once, in the home round; q-1 different blocks of the previous phase
+            uint32_t seen = bb >= 0 ? 1u << bb : 0u;
+            for (int i = 0; i < q; ++i) {
+                const int v = rrow[i];
+                if (i == h) {
+                    if (v != bb) bad_recv = 1;
+                } else {
+                    const int b = v + q;
+                    if (v >= 0 || b < 0 || ((seen >> b) & 1u)) bad_recv = 1;
+                    else seen |= 1u << b;
+                }
+            }
+        }
+        if (send) {
+            // the root sends block k in round k; everybody else sends a previous-phase block that it
+            // received in an earlier round of the row, or its baseblock of the previous phase,
+            // or -- after the home round -- its baseblock of the current phase
+            uint32_t have = bb >= 0 ? 1u << bb : 0u;     // previous-phase blocks that may be sent
+            for (int k = 0; k < q; ++k) {
+                const int v = srow[k];
+                if (r == 0) {
+                    if (v != k) bad_send = 1;
+                } else if (!(k > h && v == bb)) {
+                    const int b = v + q;
+                    if (v >= 0 || b < 0 || (recv && !((have >> b) & 1u))) bad_send = 1;
+                }
+                if (recv && k != h) {
+                    const int b = rrow[k] + q;
+                    if (b >= 0 && b < q) have |= 1u << b;
+                }
+            }
+        }
+        if (recv && send) {
+            // Algorithm 5 / Algorithm 9: what r sends in round k is what r + skips[k] receives
+            for (int k = 0; k < q; ++k) {
+                uint32_t t = r + s[k];
+                if (t >= p) t -= p;
+                if (t >= r_begin && t < r_end &&
+                    recv[(t - r_begin) * (uint64_t)q + k] != srow[k])
+                    bad_pair = 1;
+            }
+        }
+    }
+    const unsigned n_recv = __syncthreads_count(bad_recv);
+    const unsigned n_send = __syncthreads_count(bad_send);
+    const unsigned n_pair = __syncthreads_count(bad_pair);
+    if (threadIdx.x == 0) {
+        if (n_recv) atomicAdd(violations + 0, (unsigned long long)n_recv);
+        if (n_send) atomicAdd(violations + 1, (unsigned long long)n_send);
+        if (n_pair) atomicAdd(violations + 2, (unsigned long long)n_pair);
+    }
+}
+
+}  // namespace
+}  // namespace bcs
+
+using namespace bcs;
+
+extern "C" {
+
+bcs_status bcs_validate(uint32_t p, uint64_t r_begin, uint64_t r_end, const int8_t *recv,
+                        const int8_t *send, uint64_t *violations_dev, void *cuda_stream)
+{
+    bcs_status st = check_range(p, r_begin, r_end);
+    if (st != BCS_OK) return st;
+    if (violations_dev == nullptr) return BCS_ERR_ARG;
+    if (recv == nullptr && send == nullptr) return BCS_ERR_ARG;
+    if (!aligned16(recv) || !aligned16(send)) return BCS_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(violations_dev, 0, 3 * sizeof(uint64_t), stream) != cudaSuccess)
+        return BCS_ERR_CUDA;
+    PTable tab;
+    make_table(p, &tab);
+    const uint64_t count = r_end - r_begin;
+    if (count == 0 || tab.q == 0) return BCS_OK;
+    const unsigned blocks = (unsigned)((count + kTile - 1) / kTile);
+    validate_kernel<<<blocks, kTile, 0, stream>>>(
+        tab, r_begin, r_end, recv, send, reinterpret_cast<unsigned long long *>(violations_dev));
+    return launch_status();
+}
+
+}  // extern "C"

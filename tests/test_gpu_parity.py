@@ -320,9 +320,41 @@ def test_checksum_matches_oracle(bcs):
         assert got == oracle.checksum(host, first), (nbytes, first)
 
 
+def test_validate_counts_match_oracle(bcs):
+    """bcs_validate on valid and on deliberately corrupted tables (corrupted on the CPU, in a copy
+    of the oracle's tables): the three violation counts equal the oracle's."""
+    rng = np.random.default_rng(17)
+    out = torch.zeros(3, dtype=torch.int64, device="cuda")
+    for p, r0, r1 in ((2, 0, 2), (33, 0, 33), (1000, 0, 1000), (100003, 0, 100003),
+                      (100003, 777, 60001), (65537, 65000, 65537)):
+        q = oracle.q_of(p)
+        recv, send = oracle.full_table(p)
+        recv, send = recv[r0:r1].copy(), send[r0:r1].copy()
+        for corrupt in (0, 1, 40):
+            for _ in range(corrupt):
+                tbl = recv if rng.integers(2) else send
+                j, k = rng.integers(r1 - r0), rng.integers(q)
+                tbl[j, k] = rng.integers(-q, q)
+            want = oracle.validate(p, r0, r1, recv, send)
+            d_recv, d_send = torch.from_numpy(recv).cuda(), torch.from_numpy(send).cuda()
+            bcs.bcs_validate(p, r0, r1, d_recv, d_send, out)
+            assert tuple(out.cpu().tolist()) == want, (p, r0, r1, corrupt)
+            if corrupt == 0:
+                assert want == (0, 0, 0)
+            bcs.bcs_validate(p, r0, r1, d_recv, None, out)
+            assert tuple(out.cpu().tolist()) == oracle.validate(p, r0, r1, recv, None)
+            bcs.bcs_validate(p, r0, r1, None, d_send, out)
+            assert tuple(out.cpu().tolist()) == oracle.validate(p, r0, r1, None, send)
+    L = bcs.lib()
+    assert L.bcs_validate(10, 0, 10, None, None, out.data_ptr(), None) == 1
+    assert L.bcs_validate(10, 0, 10, out.data_ptr(), None, None, None) == 1
+    assert L.bcs_validate(10, 0, 11, out.data_ptr(), None, out.data_ptr(), None) == 2
+
+
 def test_large_p_chunked_spot_checked(bcs):
     """p = 2^30 - 1 (q = 30) in 8 rank chunks through one reused buffer: per chunk a checksum
-    (two runs must agree; additive pieces must add up) and seeded sample ranks against the
+    (two runs must agree; additive pieces must add up), the property checker over every rank of
+    the chunk, and seeded sample ranks against the
     per-rank oracle (10^6 ranks for the receive rows, a tenth of them for the send rows, which
     the oracle recomputes with Algorithm 5 at cubic cost)."""
     p = workloads.P_LARGE
@@ -338,6 +370,7 @@ def test_large_p_chunked_spot_checked(bcs):
     send = torch.empty(cap, dtype=torch.int8, device="cuda")
     ws = torch.empty(bcs.bcs_build_workspace_bytes(p, 0, 1 << 27), dtype=torch.int8, device="cuda")
     sums = torch.zeros(4, dtype=torch.int64, device="cuda")
+    viol = torch.zeros(3, dtype=torch.int64, device="cuda")
     m64 = 2**64 - 1
     SEND_BASE = 1 << 36                 # entry index at which the send table is taken to start
     checked = 0
@@ -346,6 +379,8 @@ def test_large_p_chunked_spot_checked(bcs):
         bcs.bcs_build(p, r0, r1, recv, send, ws)
         bcs.bcs_checksum(recv, r0 * q, sums[0:1], n_entries=nb)
         bcs.bcs_checksum(send, SEND_BASE + r0 * q, sums[1:2], n_entries=nb)
+        bcs.bcs_validate(p, r0, r1, recv, send, viol)     # every rank of the chunk: row properties
+        assert viol.cpu().tolist() == [0, 0, 0], c        # and pairing inside the chunk
         half = (nb // 2) // 4 * 4
         bcs.bcs_checksum(recv[:half], r0 * q, sums[2:3], n_entries=half)
         bcs.bcs_checksum(recv[half:], r0 * q + half, sums[3:4], n_entries=nb - half)

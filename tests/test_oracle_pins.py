@@ -283,6 +283,34 @@ def test_simulation_rejects_planted_mistakes():
     assert bcast_sim.simulate(p, n, tab2) is not None
 
 
+# ---------------------------------------------------------------- property checker
+def test_validator_accepts_valid_and_counts_planted_mistakes():
+    """oracle.validate counts ranks whose rows break the promised properties.  Valid schedules
+    (every small p; both printed p = 9 schedules) give zero; mistakes planted by hand give the
+    counts that follow from where they were planted."""
+    for p in list(range(2, 300)) + [1000, 1024, 1025]:
+        recv, send = oracle.full_table(p)
+        assert oracle.validate(p, 0, p, recv, send) == (0, 0, 0), p
+        assert oracle.validate(p, p // 3, p, recv[p // 3:], send[p // 3:]) == (0, 0, 0), p
+        assert oracle.validate(p, 0, p, recv, None) == (0, 0, 0)
+        assert oracle.validate(p, 0, p, None, send) == (0, 0, 0)
+    right = load(SECOND_P9)
+    assert oracle.validate(9, 0, 9, right["recv"], right["send"]) == (0, 0, 0)
+    p = 33                                   # skips 1 2 3 5 9 17 33 (Table 2)
+    recv, send = oracle.full_table(p)
+    bad = recv.copy(); bad[5, 3] = -1        # rank 5 = skips[3]: home round 3 must hold block 3;
+    assert oracle.validate(p, 0, p, bad, send) == (1, 0, 1)      # its sender there is the root
+    bad = recv.copy(); bad[10, 0] = bad[10, 1]                   # a block twice in a receive row
+    c = oracle.validate(p, 0, p, bad, send)
+    assert c[0] == 1 and c[2] == 1           # rank 10's row; rank 9 sends it something else
+    bad = send.copy(); bad[0, 3] = 2         # the root must send block 3 in round 3
+    assert oracle.validate(p, 0, p, recv, bad) == (0, 1, 1)
+    bad = send.copy(); bad[20, 5] = 4        # rank 20 (home round 5, baseblock 2) sends a block
+    assert oracle.validate(p, 0, p, recv, bad) == (0, 1, 1)      # of the current phase it lacks
+    assert oracle.validate(p, 0, 20, recv[:20], bad[:20]) == (0, 0, 0)   # outside the range
+    assert oracle.validate(p, 20, 21, recv[20:21], bad[20:21]) == (0, 1, 0)  # to-processor outside
+
+
 # ---------------------------------------------------------------- checksum helper
 def test_checksum_definition_and_additivity():
     rng = np.random.default_rng(5)
