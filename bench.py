@@ -179,6 +179,44 @@ def _bench_checksum(torch, bcs, flush, hbm_gbs, peak_src, table, steps):
                          "peak_source": peak_src}}
 
 
+def _bench_large(torch, bcs, workloads, hbm_gbs):
+    """p = 2^30 - 1 in 8 rank chunks through one buffer: build, checksum and property check of
+    every chunk on one stream (64 GB of tables in total, never resident together)."""
+    p = workloads.P_LARGE
+    q = bcs.bcs_q(p)
+    chunks = workloads.large_chunks()
+    cap = max(r1 - r0 for r0, r1 in chunks)
+    recv = torch.empty(cap * q, dtype=torch.int8, device="cuda")
+    send = torch.empty(cap * q, dtype=torch.int8, device="cuda")
+    ws = torch.empty(max(bcs.bcs_build_workspace_bytes(p, r0, r1) for r0, r1 in chunks),
+                     dtype=torch.int8, device="cuda")
+    sums = torch.zeros(2, dtype=torch.int64, device="cuda")
+    viol = torch.zeros(3, dtype=torch.int64, device="cuda")
+    total_viol = torch.zeros(3, dtype=torch.int64, device="cuda")
+    res = {}
+    for what in ("build", "build+checksum+validate"):
+        bcs.bcs_build(p, chunks[0][0], chunks[0][1], recv, send, ws)      # warm-up
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for r0, r1 in chunks:
+            bcs.bcs_build(p, r0, r1, recv, send, ws)
+            if what != "build":
+                nb = (r1 - r0) * q
+                bcs.bcs_checksum(recv, r0 * q, sums[0:1], n_entries=nb)
+                bcs.bcs_checksum(send, (1 << 36) + r0 * q, sums[1:2], n_entries=nb)
+                bcs.bcs_validate(p, r0, r1, recv, send, viol)
+                total_viol += viol
+        b.record()
+        torch.cuda.synchronize()
+        res[what] = a.elapsed_time(b)
+    ms = res["build"]
+    return {"workload": "p=2^30-1 (q=30), 8 chunks of 2^27 ranks, recv+send, one reused buffer",
+            "ranks": p, "ms": ms, "ranks_per_s": p / ms * 1e3, "out_gbs": 2 * p * q / ms / 1e6,
+            "ms_with_checksum_and_validate": res["build+checksum+validate"],
+            "violations": total_viol.cpu().tolist()}
+
+
 def _bench_batch(torch, bcs, workloads, flush, full):
     out = {}
     plan = bcs.bcs_batch_plan(workloads.small_sweep())
@@ -340,8 +378,14 @@ def run_ours(args) -> None:
             aux = {}
             aux["expand"], table = _bench_expand(torch, bcs, workloads, flush, hbm_gbs, peak_src, 20)
             aux["checksum"] = _bench_checksum(torch, bcs, flush, hbm_gbs, peak_src, table, 20)
+            viol = torch.zeros(3, dtype=torch.int64, device="cuda")
+            v_ms = statistics.mean(_event_ms(
+                torch, lambda: bcs.bcs_validate(p, 0, p, recv, send, viol), flush, 20, 3))
+            aux["validate"] = {"workload": "p=2^20+1, both tables, all ranks", "ms": v_ms,
+                               "ranks_per_s": p / v_ms * 1e3, "violations": viol.cpu().tolist()}
             del table
             aux.update(_bench_batch(torch, bcs, workloads, flush, full=True))
+            aux["large_p_chunked"] = _bench_large(torch, bcs, workloads, hbm_gbs)
             out["aux"] = aux
 
             # ---- CPU baseline: the oracle as it stands, per-rank form, bounded sample
