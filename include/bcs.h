@@ -83,6 +83,23 @@ bcs_status bcs_build(uint32_t p, uint64_t r_begin, uint64_t r_end,
                      int8_t *recv_out, int8_t *send_out,
                      void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* The same tables in two steps, for building one p in several rank chunks (or both
+ * tables of the same ranks at different times) without repeating the construction:
+ *   bcs_prepare runs the construction once for ALL ranks of p and leaves, in the caller's
+ *   workspace of at least bcs_prepare_workspace_bytes(p) bytes (4 bytes of skip code plus q
+ *   bytes per rank: 36.5 GB for p = 2^30-1), the receive schedule in round-major order;
+ *   bcs_build_prepared then writes the rank-major receive rows of any range (a
+ *   transposition of that copy) and its send rows (the same transposition with row k
+ *   rotated by skips[k]: sendsched[r][k] = recvsched[(r+skips[k]) mod p][k], Algorithm 9).
+ * The workspace must stay untouched between the two calls; any number of
+ * bcs_build_prepared calls may follow one bcs_prepare.  Outputs, alignment and error codes
+ * as for bcs_build; a workspace that is NULL or too small is BCS_ERR_ARG. */
+size_t bcs_prepare_workspace_bytes(uint32_t p);
+bcs_status bcs_prepare(uint32_t p, void *workspace, size_t workspace_bytes, void *cuda_stream);
+bcs_status bcs_build_prepared(uint32_t p, uint64_t r_begin, uint64_t r_end,
+                              int8_t *recv_out, int8_t *send_out,
+                              const void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* bcs_build for callers that have no device memory to offer as a workspace and may not
  * allocate any (the paper has no counterpart; this is a convenience of the library).  Think of
  * code that runs after a framework has claimed the whole GPU for its own memory pool, or of a

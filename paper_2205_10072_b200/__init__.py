@@ -13,11 +13,14 @@ from .binding import (  # noqa: F401
     bcs_build,
     bcs_build_batch,
     bcs_build_batch_workspace_bytes,
+    bcs_build_prepared,
     bcs_build_static,
     bcs_build_workspace_bytes,
     bcs_build_to_host,
     bcs_checksum,
     bcs_expand,
+    bcs_prepare,
+    bcs_prepare_workspace_bytes,
     bcs_q,
     bcs_skips,
     bcs_status_str,

@@ -48,6 +48,12 @@ def lib():
         L.bcs_build_workspace_bytes.restype = _c.c_size_t
         L.bcs_build.argtypes = [u32, u64, u64, vp, vp, vp, _c.c_size_t, vp]
         L.bcs_build.restype = i32
+        L.bcs_prepare_workspace_bytes.argtypes = [u32]
+        L.bcs_prepare_workspace_bytes.restype = _c.c_size_t
+        L.bcs_prepare.argtypes = [u32, vp, _c.c_size_t, vp]
+        L.bcs_prepare.restype = i32
+        L.bcs_build_prepared.argtypes = [u32, u64, u64, vp, vp, vp, _c.c_size_t, vp]
+        L.bcs_build_prepared.restype = i32
         L.bcs_build_static.argtypes = [u32, u64, u64, vp, vp, vp]
         L.bcs_build_static.restype = i32
         L.bcs_build_to_host.argtypes = [u32, u64, u64, vp, vp, vp, _c.c_size_t, vp]
@@ -111,6 +117,24 @@ def bcs_build(p: int, r_begin: int, r_end: int, recv_out, send_out, workspace=No
     workspace: CUDA tensor of bcs_build_workspace_bytes(...) bytes (fast path) or None."""
     _check(lib().bcs_build(p, r_begin, r_end, _ptr(recv_out), _ptr(send_out), _ptr(workspace),
                            _nbytes(workspace), _stream(stream)), "bcs_build")
+
+
+def bcs_prepare_workspace_bytes(p: int) -> int:
+    return lib().bcs_prepare_workspace_bytes(p)
+
+
+def bcs_prepare(p: int, workspace, stream=None) -> None:
+    """Runs the construction once for all ranks of p into `workspace` (CUDA tensor of
+    bcs_prepare_workspace_bytes(p) bytes) for later bcs_build_prepared calls."""
+    _check(lib().bcs_prepare(p, _ptr(workspace), _nbytes(workspace), _stream(stream)), "bcs_prepare")
+
+
+def bcs_build_prepared(p: int, r_begin: int, r_end: int, recv_out, send_out, workspace,
+                       stream=None) -> None:
+    """Rank-major receive / send rows of a range from a workspace filled by bcs_prepare."""
+    _check(lib().bcs_build_prepared(p, r_begin, r_end, _ptr(recv_out), _ptr(send_out),
+                                    _ptr(workspace), _nbytes(workspace), _stream(stream)),
+           "bcs_build_prepared")
 
 
 def bcs_build_static(p: int, r_begin: int, r_end: int, recv_out, send_out, stream=None) -> None:

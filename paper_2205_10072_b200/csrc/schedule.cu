@@ -591,7 +591,8 @@ constexpr int kTrPitch = kTile + 32;      // bytes per round in shared memory: 2
 
 __global__ void __launch_bounds__(kTile)
 send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restrict__ recv_t,
-                      uint64_t t_stride, int8_t *send_out)
+                      uint64_t t_stride, int8_t *send_out, uint32_t r_begin, uint32_t count,
+                      bool rotate)
 {
     __shared__ __align__(16) uint8_t rounds[BCS_MAX_Q * kTrPitch];
     __shared__ __align__(16) uint8_t stage[kTile * 32];
@@ -599,8 +600,12 @@ send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restri
     __shared__ uint32_t wraps;             // rounds whose 256 bytes pass the end of the row
     const uint32_t p = tab.p;
     const int q = tab.q;
-    const uint32_t r0 = blockIdx.x * kTile;
-    const uint32_t n = p - r0 < (uint32_t)kTile ? p - r0 : (uint32_t)kTile;   // ranks of this tile
+    // recv_t holds all p ranks of every round; the tile is ranks r0..r0+n-1 of the range
+    // r_begin..r_begin+count-1.  rotate: send rows (rank r + skips[k] in round k); otherwise the
+    // rows of recv_t themselves, rank-major (rotation 0).
+    const uint32_t first = blockIdx.x * kTile;
+    const uint32_t r0 = r_begin + first;
+    const uint32_t n = count - first < (uint32_t)kTile ? count - first : (uint32_t)kTile;
     if (threadIdx.x == 0) wraps = 0;
     __syncthreads();
     // one 16-byte piece per (round, vector): kTrPitch / 16 = 18 vectors cover 256 bytes at any
@@ -610,7 +615,7 @@ send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restri
     for (int w = threadIdx.x; w < q * vecs; w += kTile) {
         const int k = w / vecs, v = w - k * vecs;
         const uint8_t *src_row = reinterpret_cast<const uint8_t *>(recv_t) + (uint64_t)k * t_stride;
-        uint32_t start = r0 + tab.s[k];
+        uint32_t start = r0 + (rotate ? tab.s[k] : 0u);
         if (start >= p) start -= p;
         const uint32_t mis = start & 15u;                 // rows start 16-byte aligned (t_stride % 16 == 0)
         const uint32_t run = p - start < n ? p - start : n;      // bytes before the wrap
@@ -626,7 +631,7 @@ send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restri
     __syncthreads();
     for (uint32_t left = wraps; left != 0; left &= left - 1u) {  // the part after the wrap, by bytes
         const int k = __ffs(left) - 1;
-        uint32_t start = r0 + tab.s[k];
+        uint32_t start = r0 + (rotate ? tab.s[k] : 0u);
         if (start >= p) start -= p;
         const uint32_t run = p - start;                           // < n for these rounds
         const uint8_t *src_row = reinterpret_cast<const uint8_t *>(recv_t) + (uint64_t)k * t_stride;
@@ -649,7 +654,7 @@ send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restri
         }
     }
     __syncthreads();
-    flush_span(stage, 0, n * (uint32_t)q, send_out, (uint64_t)r0 * (uint64_t)q);
+    flush_span(stage, 0, n * (uint32_t)q, send_out, (uint64_t)first * (uint64_t)q);
 }
 
 struct Workspace {
@@ -742,7 +747,7 @@ bcs_status bcs_build(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_
         if (send_out != nullptr) {
             if (count == p)
                 send_transpose_kernel<<<blocks, kTile, 0, stream>>>(tab, ws.recv_t, ws.t_stride,
-                                                                    send_out);
+                                                                    send_out, 0u, p, true);
             else
                 send_rm_kernel<false, false><<<blocks, kTile, 0, stream>>>(
                     tab, r_begin, r_end, none, ws.codes, ws.recv_t, ws.t_stride, send_out);
@@ -757,6 +762,69 @@ bcs_status bcs_build(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_
     if (send_out != nullptr) {
         send_kernel<false><<<blocks, kTile, 0, stream>>>(tab, r_begin, r_end, none, recv_out,
                                                          send_out);
+        if ((st = launch_status()) != BCS_OK) return st;
+    }
+    return BCS_OK;
+}
+
+size_t bcs_prepare_workspace_bytes(uint32_t p)
+{
+    if (p == 0 || p > 0x7fffffffu) return 0;
+    const int q = ceil_log2_u32(p);
+    if (q == 0) return 0;
+    return (size_t)(align_up(4ull * p, 256) + (uint64_t)q * align_up(p, 16));
+}
+
+bcs_status bcs_prepare(uint32_t p, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    PTable tab;
+    bcs_status st = make_table(p, &tab);
+    if (st != BCS_OK) return st;
+    if (tab.q == 0) return BCS_OK;
+    if (workspace == nullptr || workspace_bytes < bcs_prepare_workspace_bytes(p)) return BCS_ERR_ARG;
+    if (!aligned16(workspace)) return BCS_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint32_t *codes = static_cast<uint32_t *>(workspace);
+    int8_t *recv_t = static_cast<int8_t *>(workspace) + align_up(4ull * p, 256);
+    const uint64_t t_stride = align_up(p, 16);
+    const unsigned blocks = (unsigned)((p + kTile - 1) / kTile);
+    BatchArgs none = {};
+    codes_kernel<false><<<blocks, kTile, 0, stream>>>(tab, none, codes);
+    if ((st = launch_status()) != BCS_OK) return st;
+    if (p >= 64)
+        recv_codes_warp_kernel<false, true><<<blocks, kTile, 0, stream>>>(tab, 0, p, codes, nullptr,
+                                                                          recv_t, t_stride);
+    else
+        recv_codes_kernel<false, false, true><<<blocks, kTile, 0, stream>>>(
+            tab, 0, p, none, codes, nullptr, recv_t, t_stride);
+    return launch_status();
+}
+
+bcs_status bcs_build_prepared(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_out,
+                              int8_t *send_out, const void *workspace, size_t workspace_bytes,
+                              void *cuda_stream)
+{
+    bcs_status st = check_range(p, r_begin, r_end);
+    if (st != BCS_OK) return st;
+    PTable tab;
+    make_table(p, &tab);
+    const uint64_t count = r_end - r_begin;
+    if (count == 0 || tab.q == 0) return BCS_OK;
+    if (recv_out == nullptr && send_out == nullptr) return BCS_ERR_ARG;
+    if (workspace == nullptr || workspace_bytes < bcs_prepare_workspace_bytes(p)) return BCS_ERR_ARG;
+    if (!aligned16(recv_out) || !aligned16(send_out) || !aligned16(workspace)) return BCS_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int8_t *recv_t = static_cast<const int8_t *>(workspace) + align_up(4ull * p, 256);
+    const uint64_t t_stride = align_up(p, 16);
+    const unsigned blocks = (unsigned)((count + kTile - 1) / kTile);
+    if (recv_out != nullptr) {
+        send_transpose_kernel<<<blocks, kTile, 0, stream>>>(tab, recv_t, t_stride, recv_out,
+                                                            (uint32_t)r_begin, (uint32_t)count, false);
+        if ((st = launch_status()) != BCS_OK) return st;
+    }
+    if (send_out != nullptr) {
+        send_transpose_kernel<<<blocks, kTile, 0, stream>>>(tab, recv_t, t_stride, send_out,
+                                                            (uint32_t)r_begin, (uint32_t)count, true);
         if ((st = launch_status()) != BCS_OK) return st;
     }
     return BCS_OK;

@@ -157,6 +157,36 @@ def test_sub_ranges_ragged_tails_and_single_outputs(bcs, fast):
     assert q == 17
 
 
+def test_prepare_then_build_ranges(bcs):
+    """bcs_prepare once, then receive and send rows of arbitrary ranges by bcs_build_prepared."""
+    for p in (2, 3, 33, 63, 64, 1000, 4097, 100003):
+        q = oracle.q_of(p)
+        want_r, want_s = oracle.full_table(p)
+        raw_w, ws = _guarded(bcs.bcs_prepare_workspace_bytes(p))
+        bcs.bcs_prepare(p, ws)
+        ranges = [(0, p), (0, 1), (p - 1, p), (p // 3, p // 3 + min(p - p // 3, 700)),
+                  (max(0, p - 300), p), (1, min(p, 258))]
+        for r0, r1 in ranges:
+            nb = (r1 - r0) * q
+            raw_r, recv = _guarded(nb)
+            raw_s, send = _guarded(nb)
+            bcs.bcs_build_prepared(p, r0, r1, recv, send, ws)
+            torch.cuda.synchronize()
+            assert _guards_intact(raw_r, nb) and _guards_intact(raw_s, nb) and _guards_intact(raw_w, ws.numel())
+            assert np.array_equal(recv.cpu().numpy().reshape(-1, q), want_r[r0:r1]), (p, r0, r1)
+            assert np.array_equal(send.cpu().numpy().reshape(-1, q), want_s[r0:r1]), (p, r0, r1)
+        raw_s, send = _guarded(p * q)
+        bcs.bcs_build_prepared(p, 0, p, None, send, ws)          # one table only
+        torch.cuda.synchronize()
+        assert np.array_equal(send.cpu().numpy().reshape(p, q), want_s)
+    L = bcs.lib()
+    small = torch.zeros(64, dtype=torch.int8, device="cuda")
+    assert L.bcs_prepare(1000, small.data_ptr(), 64, None) == 1                # too small
+    assert L.bcs_build_prepared(1000, 0, 10, small.data_ptr(), None, small.data_ptr(), 64, None) == 1
+    assert L.bcs_prepare(1, None, 0, None) == 0 and bcs.bcs_prepare_workspace_bytes(1) == 0
+    assert bcs.bcs_prepare_workspace_bytes(20) == 256 + 5 * 32
+
+
 def test_degenerate_sizes_and_errors(bcs):
     L = bcs.lib()
     buf = torch.zeros(64, dtype=torch.int8, device="cuda")
@@ -368,7 +398,8 @@ def test_large_p_chunked_spot_checked(bcs):
     cap = (1 << 27) * q
     recv = torch.empty(cap, dtype=torch.int8, device="cuda")
     send = torch.empty(cap, dtype=torch.int8, device="cuda")
-    ws = torch.empty(bcs.bcs_build_workspace_bytes(p, 0, 1 << 27), dtype=torch.int8, device="cuda")
+    ws = torch.empty(bcs.bcs_prepare_workspace_bytes(p), dtype=torch.int8, device="cuda")   # 36.5 GB
+    bcs.bcs_prepare(p, ws)
     sums = torch.zeros(4, dtype=torch.int64, device="cuda")
     viol = torch.zeros(3, dtype=torch.int64, device="cuda")
     m64 = 2**64 - 1
@@ -376,7 +407,7 @@ def test_large_p_chunked_spot_checked(bcs):
     checked = 0
     for c, (r0, r1) in enumerate(chunks):
         nb = (r1 - r0) * q
-        bcs.bcs_build(p, r0, r1, recv, send, ws)
+        bcs.bcs_build_prepared(p, r0, r1, recv, send, ws)
         bcs.bcs_checksum(recv, r0 * q, sums[0:1], n_entries=nb)
         bcs.bcs_checksum(send, SEND_BASE + r0 * q, sums[1:2], n_entries=nb)
         bcs.bcs_validate(p, r0, r1, recv, send, viol)     # every rank of the chunk: row properties
@@ -399,10 +430,15 @@ def test_large_p_chunked_spot_checked(bcs):
         o_r, _ = oracle.build_range(p, r0, r0 + head, want_send=False)
         bcs.bcs_checksum(recv, r0 * q, sums[2:3], n_entries=head * q)
         assert int(sums.cpu()[2]) & m64 == oracle.checksum(o_r, r0 * q)
-        if c in (0, 7):     # rebuilt with the other (self-contained) construction: same sums
-            recv.fill_(0)
+        if c in (0, 7):     # rebuilt by bcs_build (self-contained construction; at the last chunk
+            recv.fill_(0)   # with its own workspace): same sums
             send.fill_(0)
-            bcs.bcs_build(p, r0, r1, recv, send, None)
+            own = None
+            if c == 7:
+                own = torch.empty(bcs.bcs_build_workspace_bytes(p, r0, r1), dtype=torch.int8,
+                                  device="cuda")
+            bcs.bcs_build(p, r0, r1, recv, send, own)
+            del own
             bcs.bcs_checksum(recv, r0 * q, sums[0:1], n_entries=nb)
             bcs.bcs_checksum(send, SEND_BASE + r0 * q, sums[1:2], n_entries=nb)
             again = [int(v) & m64 for v in sums.cpu()]
