@@ -368,7 +368,7 @@ recv_codes_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, BatchArgs ba,
 // same for all lanes.  These are the rounds in which neighbouring ranks disagree about which
 // path of the code search they take; the later rounds run the code search per lane.
 template <bool kRowOut, bool kColOut>
-__global__ void __launch_bounds__(kTile)
+__global__ void __launch_bounds__(kTile, 8)
 recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uint64_t r_end,
                        const uint32_t *__restrict__ codes, int8_t *recv_out, int8_t *recv_t,
                        uint64_t t_stride)
