@@ -385,6 +385,12 @@ def run_ours(args) -> None:
                 torch, lambda: bcs.bcs_validate(p, 0, p, recv, send, viol), flush, 20, 3))
             aux["validate"] = {"workload": "p=2^20+1, both tables, all ranks", "ms": v_ms,
                                "ranks_per_s": p / v_ms * 1e3, "violations": viol.cpu().tolist()}
+            state = torch.empty(2 * p, dtype=torch.int64, device="cuda")
+            counts = torch.zeros(5, dtype=torch.int64, device="cuda")
+            s_ms = statistics.mean(_event_ms(
+                torch, lambda: bcs.bcs_simulate(p, 5, recv, send, state, counts), flush, 5, 1))
+            aux["simulate"] = {"workload": "p=2^20+1, n=5 blocks, 25 rounds, all ranks", "ms": s_ms,
+                               "counts": counts.cpu().tolist()}
             del table
             aux.update(_bench_batch(torch, bcs, workloads, flush, full=True))
             aux["large_p_chunked"] = _bench_large(torch, bcs, workloads, hbm_gbs)

@@ -199,6 +199,22 @@ bcs_status bcs_validate(uint32_t p, uint64_t r_begin, uint64_t r_end,
                         const int8_t *recv, const int8_t *send,
                         uint64_t *violations_dev, void *cuda_stream);
 
+/* Brute-force run of the n-block broadcast (Algorithm 6 without the data) over the complete
+ * tables of one p, all ranks at once, n-1+q rounds, for p far beyond what a host can simulate.
+ * Rank 0 starts with all n blocks.  Counted over all rounds and ranks:
+ *   counts_dev[0]  a rank sends a block it does not hold at that time (condition a) of Section 2),
+ *   counts_dev[1]  what a rank sends differs from what its to-processor receives in that round,
+ *   counts_dev[2]  a non-root rank receives a block it already has (condition b)),
+ *   counts_dev[3]  ranks that do not hold all n blocks after the last round,
+ *   counts_dev[4]  ranks that already held all n blocks before the last round (the root always
+ *                  does; n-1+q rounds being necessary, at least one rank must not).
+ * A correct round-optimal schedule gives 0, 0, 0, 0 and counts_dev[4] < p.
+ *   recv, send: device int8, the FULL [p][q] tables; n <= 64 (BCS_ERR_UNSUPPORTED beyond);
+ *   state_dev: device scratch of 2 * p uint64, 8-byte aligned; counts_dev: five uint64,
+ *   overwritten.  n + q + 1 kernels are enqueued on the stream. */
+bcs_status bcs_simulate(uint32_t p, uint32_t n, const int8_t *recv, const int8_t *send,
+                        uint64_t *state_dev, uint64_t *counts_dev, void *cuda_stream);
+
 /* Position-weighted 64-bit checksum of a stretch of schedule entries, additive
  * over disjoint stretches (no counterpart in the paper; used to compare outputs
  * that are too large to copy back).  The bytes are read as little-endian 32-bit

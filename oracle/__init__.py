@@ -69,6 +69,8 @@ def _load():
         lib.bcso_validate.argtypes = [c.c_uint32, c.c_uint64, c.c_uint64, i8p, i8p,
                                       c.POINTER(c.c_uint64)]
         lib.bcso_validate.restype = None
+        lib.bcso_simulate.argtypes = [c.c_uint32, c.c_uint32, i8p, i8p, c.POINTER(c.c_uint64)]
+        lib.bcso_simulate.restype = c.c_int
         lib.bcso_set_root_mode.argtypes = [c.c_int]
         lib.bcso_set_root_mode.restype = None
         lib.bcso_num_threads.argtypes = []
@@ -209,6 +211,19 @@ def validate(p: int, r_begin: int, r_end: int, recv, send):
         send = np.ascontiguousarray(send, dtype=np.int8).reshape(n, q)
     out = (ctypes.c_uint64 * 3)()
     _load().bcso_validate(p, r_begin, r_end, _i8(recv), _i8(send), out)
+    return tuple(int(v) for v in out)
+
+
+def simulate(p: int, n: int, recv, send):
+    """Brute-force broadcast of n <= 64 blocks over the full tables -> (unheld sends, unpaired
+    rounds, repeated receipts, ranks incomplete at the end, ranks complete before the last round)."""
+    q = q_of(p)
+    recv = np.ascontiguousarray(recv, dtype=np.int8).reshape(p, q)
+    send = np.ascontiguousarray(send, dtype=np.int8).reshape(p, q)
+    out = (ctypes.c_uint64 * 5)()
+    rc = _load().bcso_simulate(p, n, _i8(recv), _i8(send), out)
+    if rc:
+        raise RuntimeError("oracle simulate failed: %d" % rc)
     return tuple(int(v) for v in out)
 
 

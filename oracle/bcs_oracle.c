@@ -545,6 +545,53 @@ void bcso_validate(uint32_t p, uint64_t r_begin, uint64_t r_end, const int8_t *r
     }
 }
 
+/* Brute-force run of Algorithm 6 for all p ranks at once (rank 0 holds the n
+ * blocks, n <= 64): every rank's rounds come from the literal loop of
+ * bcso_expand_rank; counts as the library's simulator reports them:
+ *   [0] sends of a block the sender does not hold, [1] rounds in which what r
+ *   sends is not what its to-processor receives, [2] receipts by a non-root
+ *   rank of a block it already has, [3] ranks incomplete after the last round,
+ *   [4] ranks already complete before the last round.  Returns -3 if out of
+ *   memory, -2 for n > 64. */
+int bcso_simulate(uint32_t p, uint32_t n, const int8_t *recv, const int8_t *send,
+                  uint64_t *counts)
+{
+    int q = bcso_q(p);
+    size_t rounds = (size_t)n - 1 + q, j;
+    uint64_t all = n >= 64 ? ~(uint64_t)0 : (((uint64_t)1 << n) - 1);
+    uint64_t *held, *next, r;
+    int32_t *tab;
+    counts[0] = counts[1] = counts[2] = counts[3] = counts[4] = 0;
+    if (n > 64) return -2;
+    if (q == 0) return 0;
+    held = (uint64_t *)calloc(p, sizeof(uint64_t));
+    next = (uint64_t *)calloc(p, sizeof(uint64_t));
+    tab = (int32_t *)malloc((size_t)p * rounds * 4 * sizeof(int32_t));
+    if (!held || !next || !tab) { free(held); free(next); free(tab); return -3; }
+    for (r = 0; r < p; r++)
+        bcso_expand_rank(p, n, (uint32_t)r, recv + r * q, send + r * q, tab + r * rounds * 4);
+    held[0] = all;
+    for (j = 0; j < rounds; j++) {
+        for (r = 0; r < p; r++) {
+            const int32_t *o = tab + (r * rounds + j) * 4;
+            int32_t sb = o[0], rb = o[1], to = o[2];
+            if (sb >= 0 && !((held[r] >> sb) & 1)) counts[0]++;
+            if (tab[((size_t)to * rounds + j) * 4 + 1] != sb) counts[1]++;
+            next[r] = held[r];
+            if (rb >= 0) {
+                if (r != 0 && ((held[r] >> rb) & 1)) counts[2]++;
+                next[r] |= (uint64_t)1 << rb;
+            }
+            if (j + 1 == rounds && held[r] == all) counts[4]++;
+        }
+        { uint64_t *t = held; held = next; next = t; }
+    }
+    for (r = 0; r < p; r++)
+        if (held[r] != all) counts[3]++;
+    free(held); free(next); free(tab);
+    return 0;
+}
+
 int bcso_num_threads(void)
 {
 #ifdef _OPENMP

@@ -22,6 +22,7 @@ from .binding import (  # noqa: F401
     bcs_prepare,
     bcs_prepare_workspace_bytes,
     bcs_q,
+    bcs_simulate,
     bcs_skips,
     bcs_status_str,
     bcs_validate,

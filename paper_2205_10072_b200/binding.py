@@ -68,6 +68,8 @@ def lib():
         L.bcs_expand.restype = i32
         L.bcs_validate.argtypes = [u32, u64, u64, vp, vp, vp, vp]
         L.bcs_validate.restype = i32
+        L.bcs_simulate.argtypes = [u32, u32, vp, vp, vp, vp, vp]
+        L.bcs_simulate.restype = i32
         L.bcs_checksum.argtypes = [vp, u64, u64, vp, vp]
         L.bcs_checksum.restype = i32
         _lib = L
@@ -227,6 +229,13 @@ def bcs_validate(p: int, r_begin: int, r_end: int, recv, send, violations_out, s
     three elements: ranks with a bad receive row, a bad send row, a send/receive mismatch."""
     _check(lib().bcs_validate(p, r_begin, r_end, _ptr(recv), _ptr(send), _ptr(violations_out),
                               _stream(stream)), "bcs_validate")
+
+
+def bcs_simulate(p: int, n: int, recv, send, state, counts_out, stream=None) -> None:
+    """recv/send: full [p][q] CUDA int8 tables; state: CUDA int64 tensor of 2*p elements (scratch);
+    counts_out: CUDA int64 tensor of five elements (see include/bcs.h)."""
+    _check(lib().bcs_simulate(p, n, _ptr(recv), _ptr(send), _ptr(state), _ptr(counts_out),
+                              _stream(stream)), "bcs_simulate")
 
 
 def bcs_checksum(buf, first_entry_index: int, sum_out, stream=None, n_entries: int | None = None) -> None:

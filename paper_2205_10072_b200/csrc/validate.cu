@@ -117,6 +117,75 @@ validate_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, const int8_t *__re
     }
 }
 
+// ---------------------------------------------------------------- broadcast simulation
+// One round of the n-block broadcast for every rank at once (Algorithm 6 with the blocks taken
+// from the int8 tables by the closed form block = entry - x + q * floor(i / q), i = j + x).
+// held[r]: bit b set iff rank r holds block b before the round; next[r]: after it.
+__global__ void __launch_bounds__(kTile)
+simulate_round_kernel(PTable tab, uint32_t n, uint32_t i, const int8_t *__restrict__ recv,
+                      const int8_t *__restrict__ send, const unsigned long long *__restrict__ held,
+                      unsigned long long *__restrict__ next, unsigned long long *counts,
+                      int last_round)
+{
+    const uint32_t p = tab.p;
+    const int q = tab.q;
+    const uint32_t k = i % (uint32_t)q;
+    const int shift = (int)(i / (uint32_t)q) * q;          // q * floor(i / q)
+    const int x = (int)(((uint32_t)q - (n - 1u + (uint32_t)q) % (uint32_t)q) % (uint32_t)q);
+    const int top = (int)n - 1;
+    const uint64_t r64 = (uint64_t)blockIdx.x * kTile + threadIdx.x;
+    unsigned unheld = 0, unpaired = 0, twice = 0, early = 0;
+    if (r64 < p) {
+        const uint32_t r = (uint32_t)r64;
+        const unsigned long long all = n >= 64u ? ~0ull : (1ull << n) - 1ull;
+        const unsigned long long mine = held[r];
+        int sb = (int)send[(uint64_t)r * q + k] - x + shift;
+        int rb = (int)recv[(uint64_t)r * q + k] - x + shift;
+        sb = sb < 0 ? -1 : (sb > top ? top : sb);
+        rb = rb < 0 ? -1 : (rb > top ? top : rb);
+        uint32_t to = r + tab.s[k];
+        if (to >= p) to -= p;
+        int rb_to = (int)recv[(uint64_t)to * q + k] - x + shift;   // what the to-processor receives
+        rb_to = rb_to < 0 ? -1 : (rb_to > top ? top : rb_to);
+        if (sb >= 0 && !((mine >> sb) & 1ull)) unheld = 1;         // condition a): sends only held blocks
+        if (rb_to != sb) unpaired = 1;
+        unsigned long long after = mine;
+        if (rb >= 0) {
+            if (r != 0 && ((mine >> rb) & 1ull)) twice = 1;        // condition b): every receipt is new
+            after |= 1ull << rb;
+        }
+        next[r] = after;
+        if (last_round && mine == all) early = 1;                  // complete before the last round
+    }
+    const unsigned c0 = __syncthreads_count(unheld);
+    const unsigned c1 = __syncthreads_count(unpaired);
+    const unsigned c2 = __syncthreads_count(twice);
+    const unsigned c3 = __syncthreads_count(early);
+    if (threadIdx.x == 0) {
+        if (c0) atomicAdd(counts + 0, (unsigned long long)c0);
+        if (c1) atomicAdd(counts + 1, (unsigned long long)c1);
+        if (c2) atomicAdd(counts + 2, (unsigned long long)c2);
+        if (c3) atomicAdd(counts + 4, (unsigned long long)c3);
+    }
+}
+
+__global__ void __launch_bounds__(kTile)
+simulate_init_kernel(uint32_t p, uint32_t n, unsigned long long *held)
+{
+    const uint64_t r = (uint64_t)blockIdx.x * kTile + threadIdx.x;
+    if (r < p) held[r] = r == 0 ? (n >= 64u ? ~0ull : (1ull << n) - 1ull) : 0ull;
+}
+
+__global__ void __launch_bounds__(kTile)
+simulate_final_kernel(uint32_t p, uint32_t n, const unsigned long long *__restrict__ held,
+                      unsigned long long *counts)
+{
+    const uint64_t r = (uint64_t)blockIdx.x * kTile + threadIdx.x;
+    const unsigned long long all = n >= 64u ? ~0ull : (1ull << n) - 1ull;
+    const unsigned c = __syncthreads_count(r < p && held[r] != all);
+    if (threadIdx.x == 0 && c) atomicAdd(counts + 3, (unsigned long long)c);
+}
+
 }  // namespace
 }  // namespace bcs
 
@@ -142,6 +211,40 @@ bcs_status bcs_validate(uint32_t p, uint64_t r_begin, uint64_t r_end, const int8
     const unsigned blocks = (unsigned)((count + kTile - 1) / kTile);
     validate_kernel<<<blocks, kTile, 0, stream>>>(
         tab, r_begin, r_end, recv, send, reinterpret_cast<unsigned long long *>(violations_dev));
+    return launch_status();
+}
+
+bcs_status bcs_simulate(uint32_t p, uint32_t n, const int8_t *recv, const int8_t *send,
+                        uint64_t *state_dev, uint64_t *counts_dev, void *cuda_stream)
+{
+    PTable tab;
+    bcs_status st = make_table(p, &tab);
+    if (st != BCS_OK) return st;
+    if (n == 0 || counts_dev == nullptr) return BCS_ERR_ARG;
+    if (n > 64) return BCS_ERR_UNSUPPORTED;           // the held blocks of a rank are one 64-bit set
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(counts_dev, 0, 5 * sizeof(uint64_t), stream) != cudaSuccess)
+        return BCS_ERR_CUDA;
+    if (tab.q == 0) return BCS_OK;
+    if (recv == nullptr || send == nullptr || state_dev == nullptr) return BCS_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(state_dev) & 7u) != 0) return BCS_ERR_ALIGN;
+    unsigned long long *held = reinterpret_cast<unsigned long long *>(state_dev);
+    unsigned long long *next = held + p;
+    unsigned long long *counts = reinterpret_cast<unsigned long long *>(counts_dev);
+    const unsigned blocks = (unsigned)((p + kTile - 1) / kTile);
+    const uint32_t rounds = n - 1u + (uint32_t)tab.q;
+    const uint32_t x = ((uint32_t)tab.q - rounds % (uint32_t)tab.q) % (uint32_t)tab.q;
+    simulate_init_kernel<<<blocks, kTile, 0, stream>>>(p, n, held);
+    if ((st = launch_status()) != BCS_OK) return st;
+    for (uint32_t j = 0; j < rounds; ++j) {
+        simulate_round_kernel<<<blocks, kTile, 0, stream>>>(tab, n, j + x, recv, send, held, next,
+                                                            counts, j + 1 == rounds);
+        if ((st = launch_status()) != BCS_OK) return st;
+        unsigned long long *t = held;
+        held = next;
+        next = t;
+    }
+    simulate_final_kernel<<<blocks, kTile, 0, stream>>>(p, n, held, counts);
     return launch_status();
 }
 

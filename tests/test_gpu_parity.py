@@ -381,6 +381,70 @@ def test_validate_counts_match_oracle(bcs):
     assert L.bcs_validate(10, 0, 11, out.data_ptr(), None, out.data_ptr(), None) == 2
 
 
+def test_simulate_counts_match_oracle(bcs):
+    """bcs_simulate against the oracle's brute-force run (and, for validity, the numpy simulation)
+    on valid and corrupted tables, then on the benchmark's p = 2^20+1 built by the library."""
+    rng = np.random.default_rng(29)
+    counts = torch.zeros(5, dtype=torch.int64, device="cuda")
+    for p in (2, 3, 9, 33, 100, 1000, 4097):
+        q = oracle.q_of(p)
+        recv, send = oracle.full_table(p)
+        state = torch.empty(2 * p, dtype=torch.int64, device="cuda")
+        for corrupt in (0, 1, 6):
+            br, bs = recv.copy(), send.copy()
+            for _ in range(corrupt):
+                tbl = br if rng.integers(2) else bs
+                tbl[rng.integers(p), rng.integers(q)] = rng.integers(-q, q)
+            for n in (1, 2, 5, q + 3, 64):
+                bcs.bcs_simulate(p, n, torch.from_numpy(br).cuda(), torch.from_numpy(bs).cuda(),
+                                 state, counts)
+                got = tuple(counts.cpu().tolist())
+                assert got == oracle.simulate(p, n, br, bs), (p, n, corrupt)
+                if corrupt == 0:
+                    assert got[:4] == (0, 0, 0, 0) and got[4] < p
+                    if n <= 13:
+                        assert bcast_sim.simulate(p, n, oracle.expand(p, n, br, bs)) is None
+    p = workloads.P_SINGLE
+    q = bcs.bcs_q(p)
+    recv = torch.empty(p * q, dtype=torch.int8, device="cuda")
+    send = torch.empty(p * q, dtype=torch.int8, device="cuda")
+    ws = torch.empty(bcs.bcs_build_workspace_bytes(p, 0, p), dtype=torch.int8, device="cuda")
+    bcs.bcs_build(p, 0, p, recv, send, ws)
+    state = torch.empty(2 * p, dtype=torch.int64, device="cuda")
+    for n in (1, 5, q + 3):
+        bcs.bcs_simulate(p, n, recv, send, state, counts)
+        got = counts.cpu().tolist()
+        assert got[:4] == [0, 0, 0, 0] and 1 <= got[4] < p, (n, got)
+    L = bcs.lib()
+    assert L.bcs_simulate(p, 65, recv.data_ptr(), send.data_ptr(), state.data_ptr(),
+                          counts.data_ptr(), None) == 4
+    assert L.bcs_simulate(p, 0, recv.data_ptr(), send.data_ptr(), state.data_ptr(),
+                          counts.data_ptr(), None) == 1
+
+
+def test_large_p_full_broadcast_simulation(bcs):
+    """Every rank of p = 2^30 - 1: both complete tables (64 GB) built from one bcs_prepare, then
+    the five-block broadcast simulated on the device -- 34 rounds, every rank receives every
+    block exactly once from a rank that holds it."""
+    torch.cuda.empty_cache()
+    p, q, n = workloads.P_LARGE, 30, 5
+    ws = torch.empty(bcs.bcs_prepare_workspace_bytes(p), dtype=torch.int8, device="cuda")
+    bcs.bcs_prepare(p, ws)
+    recv = torch.empty(p * q, dtype=torch.int8, device="cuda")
+    send = torch.empty(p * q, dtype=torch.int8, device="cuda")
+    bcs.bcs_build_prepared(p, 0, p, recv, send, ws)
+    torch.cuda.synchronize()
+    del ws
+    torch.cuda.empty_cache()
+    state = torch.empty(2 * p, dtype=torch.int64, device="cuda")
+    counts = torch.zeros(5, dtype=torch.int64, device="cuda")
+    bcs.bcs_simulate(p, n, recv, send, state, counts)
+    got = counts.cpu().tolist()
+    assert got[:4] == [0, 0, 0, 0] and 1 <= got[4] < p, got
+    del recv, send, state
+    torch.cuda.empty_cache()
+
+
 def test_large_p_chunked_spot_checked(bcs):
     """p = 2^30 - 1 (q = 30) in 8 rank chunks through one reused buffer: per chunk a checksum
     (two runs must agree; additive pieces must add up), the property checker over every rank of

@@ -311,6 +311,41 @@ def test_validator_accepts_valid_and_counts_planted_mistakes():
     assert oracle.validate(p, 20, 21, recv[20:21], bad[20:21]) == (0, 1, 0)  # to-processor outside
 
 
+def test_oracle_simulator_agrees_with_the_numpy_simulation():
+    """oracle.simulate (C, counts) against tests/bcast_sim.py (numpy, independent skips and round
+    semantics): zero counts exactly when the numpy simulation accepts, on valid and on corrupted
+    tables; hand-planted mistakes give the counts that follow from them."""
+    rng = np.random.default_rng(23)
+    for p in (2, 3, 9, 20, 31, 32, 33, 100, 257):
+        q = oracle.q_of(p)
+        recv, send = oracle.full_table(p)
+        for n in (1, 2, 5, q + 3, 64):
+            c = oracle.simulate(p, n, recv, send)
+            assert c[:4] == (0, 0, 0, 0) and 1 <= c[4] < p, (p, n, c)
+            assert bcast_sim.simulate(p, n, oracle.expand(p, n, recv, send)) is None
+        for _ in range(12):
+            br, bs = recv.copy(), send.copy()
+            tbl = br if rng.integers(2) else bs
+            j, k = rng.integers(p), rng.integers(q)
+            new = rng.integers(-q, q)
+            if new == tbl[j, k]:
+                continue
+            tbl[j, k] = new
+            n = int(rng.choice([2, 5, q + 3]))
+            c = oracle.simulate(p, n, br, bs)
+            ok_numpy = bcast_sim.simulate(p, n, oracle.expand(p, n, br, bs)) is None
+            assert (c[:4] == (0, 0, 0, 0) and c[4] < p) == ok_numpy, (p, n, j, k, new, c)
+    right = load(SECOND_P9)
+    assert oracle.simulate(9, 5, right["recv"], right["send"])[:4] == (0, 0, 0, 0)
+    # p = 9, n = 5 (q = 4, eight rounds, no virtual round): in round 0 the root sends block 0 to
+    # rank 1; a table in which rank 1 expects block 1 there is unpaired in that round, and rank 1
+    # then holds a block nobody sent while block 0 is missing when it has to forward it
+    recv, send = oracle.full_table(9)
+    bad = recv.copy(); bad[1, 0] = 1
+    c = oracle.simulate(9, 5, bad, send)
+    assert c[1] == 1 and c[0] >= 1, c
+
+
 # ---------------------------------------------------------------- checksum helper
 def test_checksum_definition_and_additivity():
     rng = np.random.default_rng(5)
