@@ -168,6 +168,27 @@ def _bench_expand(torch, bcs, workloads, flush, hbm_gbs, peak_src, steps):
     return res, table
 
 
+def _bench_allgather(torch, bcs, workloads, flush, hbm_gbs, peak_src, steps):
+    p, n = workloads.P_EXPAND, workloads.N_EXPAND
+    q = bcs.bcs_q(p)
+    er = torch.empty(p * q, dtype=torch.int8, device="cuda")
+    es = torch.empty(p * q, dtype=torch.int8, device="cuda")
+    ews = torch.empty(bcs.bcs_build_workspace_bytes(p, 0, p), dtype=torch.int8, device="cuda")
+    bcs.bcs_build(p, 0, p, er, es, ews)
+    rounds = n - 1 + q
+    pack = torch.empty((rounds, p), dtype=torch.int32, device="cuda")
+    unpack = torch.empty((rounds, p), dtype=torch.int32, device="cuda")
+    ms = statistics.mean(_event_ms(
+        torch, lambda: bcs.bcs_allgather_tables(p, n, 54607, er, es, pack, unpack), flush, steps, 3))
+    nbytes = 2 * rounds * p * 4
+    gbs = nbytes / ms / 1e6
+    return {"workload": "p=100003, n=1000, processor 54607: pack+unpack int32 [1016][100003]",
+            "ms": ms, "bytes": nbytes, "gbs": gbs,
+            "roofline": {"bound": "hbm", "kernel": "allgather_kernel", "achieved": gbs,
+                         "peak": hbm_gbs, "unit": "GB/s", "frac": gbs / hbm_gbs, "traffic": None,
+                         "peak_source": peak_src}}
+
+
 def _bench_checksum(torch, bcs, flush, hbm_gbs, peak_src, table, steps):
     sums = torch.zeros(1, dtype=torch.int64, device="cuda")
     tb = table.view(torch.int8).view(-1)
@@ -274,10 +295,13 @@ def run_ours(args) -> None:
     def flush():
         flush_buf.fill_(1)
 
-    if args.only in ("expand", "checksum", "batch"):       # small single-part runs (profiling)
+    if args.only in ("expand", "checksum", "batch", "allgather"):   # small single-part runs (profiling)
         if rank == 0:
             res = {}
-            if args.only in ("expand", "checksum"):
+            if args.only == "allgather":
+                res["allgather_tables"] = _bench_allgather(torch, bcs, workloads, flush, hbm_gbs,
+                                                           peak_src, args.steps)
+            elif args.only in ("expand", "checksum"):
                 ex, table = _bench_expand(torch, bcs, workloads, flush, hbm_gbs, peak_src,
                                           args.steps)
                 res["expand"] = ex
@@ -392,6 +416,8 @@ def run_ours(args) -> None:
             aux["simulate"] = {"workload": "p=2^20+1, n=5 blocks, 25 rounds, all ranks", "ms": s_ms,
                                "counts": counts.cpu().tolist()}
             del table
+            aux["allgather_tables"] = _bench_allgather(torch, bcs, workloads, flush, hbm_gbs,
+                                                       peak_src, 20)
             aux.update(_bench_batch(torch, bcs, workloads, flush, full=True))
             aux["large_p_chunked"] = _bench_large(torch, bcs, workloads, hbm_gbs)
             out["aux"] = aux
@@ -437,7 +463,8 @@ def main() -> None:
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--only", default="all", choices=["all", "build", "expand", "checksum", "batch"],
+    ap.add_argument("--only", default="all",
+                    choices=["all", "build", "expand", "checksum", "batch", "allgather"],
                     help="run one part only (small, profiler-friendly runs); 'all' is the benchmark")
     args = ap.parse_args()
     if args.impl == "reference":

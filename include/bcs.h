@@ -178,6 +178,22 @@ bcs_status bcs_expand(uint32_t p, uint32_t n, uint64_t r_begin, uint64_t r_end,
                       const int8_t *recv, const int8_t *send, int32_t *table_out,
                       void *cuda_stream);
 
+/* Index tables of the irregular allgather (Algorithm 9 without the pack / Send||Recv / unpack
+ * data movement) for ONE processor r: in round jr (0..n-2+q) processor r packs block
+ * pack_out[jr * p + j] of buffer[j] for its to-processor and unpacks what it receives into
+ * block unpack_out[jr * p + j] of buffer[j], j = 0..p-1; -1 = nothing for that buffer in that
+ * round, blocks above n-1 are n-1.  Processor r handles buffer j as virtual processor
+ * (r-j) mod p of the broadcast rooted at j, so the entries are the send / receive blocks of
+ * that virtual processor's round, with the schedule adjustment of Algorithm 6 (-x, first use
+ * of the first x entries in the second phase) applied to every row -- Algorithm 9 as printed
+ * omits it and would then start with block x instead of block 0.  The to- and from-processors
+ * of the round are those of bcs_expand.
+ *   recv, send: device int8, the FULL [p][q] tables; pack_out, unpack_out: device int32,
+ *   (n-1+q) * p entries each, 4-byte aligned, either may be NULL.  n-1+q <= 65535 * 64. */
+bcs_status bcs_allgather_tables(uint32_t p, uint32_t n, uint32_t r,
+                                const int8_t *recv, const int8_t *send,
+                                int32_t *pack_out, int32_t *unpack_out, void *cuda_stream);
+
 /* Counts the ranks of r_begin..r_end-1 whose rows break a property that every schedule of the
  * construction has (text after Theorem 1; Algorithms 4, 5 and 9) -- a check that scales to
  * tables far too large to compare entry by entry:

@@ -71,6 +71,9 @@ def _load():
         lib.bcso_validate.restype = None
         lib.bcso_simulate.argtypes = [c.c_uint32, c.c_uint32, i8p, i8p, c.POINTER(c.c_uint64)]
         lib.bcso_simulate.restype = c.c_int
+        lib.bcso_allgather_rank.argtypes = [c.c_uint32, c.c_uint32, c.c_uint32, i8p, i8p, c.c_int,
+                                            c.POINTER(c.c_int32), c.POINTER(c.c_int32)]
+        lib.bcso_allgather_rank.restype = c.c_int
         lib.bcso_set_root_mode.argtypes = [c.c_int]
         lib.bcso_set_root_mode.restype = None
         lib.bcso_num_threads.argtypes = []
@@ -225,6 +228,24 @@ def simulate(p: int, n: int, recv, send):
     if rc:
         raise RuntimeError("oracle simulate failed: %d" % rc)
     return tuple(int(v) for v in out)
+
+
+def allgather_rank(p: int, n: int, r: int, recv, send, adjust: bool = True):
+    """Algorithm 9's pack and unpack block numbers of processor r -> (pack, unpack), int32
+    [n-1+q][p]: entry [round][j] is the block of buffer[j] sent resp. received in that round.
+    adjust=False leaves out the schedule adjustment of Algorithm 6 (Algorithm 9 as printed; only
+    for the self-test that shows it is needed)."""
+    q = q_of(p)
+    recv = np.ascontiguousarray(recv, dtype=np.int8).reshape(p, q)
+    send = np.ascontiguousarray(send, dtype=np.int8).reshape(p, q)
+    pack = np.zeros((n - 1 + q, p), dtype=np.int32)
+    unpack = np.zeros((n - 1 + q, p), dtype=np.int32)
+    i32 = ctypes.POINTER(ctypes.c_int32)
+    rc = _load().bcso_allgather_rank(p, n, r, _i8(recv), _i8(send), int(adjust),
+                                     pack.ctypes.data_as(i32), unpack.ctypes.data_as(i32))
+    if rc:
+        raise RuntimeError("oracle allgather_rank failed: %d" % rc)
+    return pack, unpack
 
 
 def set_root_mode(mode: int) -> None:

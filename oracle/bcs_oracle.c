@@ -451,6 +451,58 @@ void bcso_expand_range(uint32_t p, uint32_t n, uint64_t r_begin, uint64_t r_end,
     }
 }
 
+/* Algorithm 9 without the data movement, for processor r: which block of
+ * buffer[j] is packed (sent) and which is unpacked (received) in every round.
+ * The full schedule is given (recv / send are the [p][q] tables of a root-0
+ * broadcast); working copies are adjusted as Algorithm 6 does (-x, and +q for
+ * the x entries whose first use falls into the second phase) -- Algorithm 9
+ * as printed leaves this adjustment out, without it the first real round
+ * would use block x instead of block 0 -- and then every use of an entry adds
+ * q to it, exactly as the pack and unpack loops are written.
+ * pack[jr * p + j], unpack[jr * p + j] for round jr = i - x and buffer j:
+ * block numbers after the rule "below 0: nothing (-1), above n-1: n-1".
+ * Returns -3 if out of memory. */
+int bcso_allgather_rank(uint32_t p, uint32_t n, uint32_t r, const int8_t *recv,
+                        const int8_t *send, int adjust, int32_t *pack, int32_t *unpack)
+{
+    uint32_t s[BCSO_MAXQ + 1];
+    int q = bcso_skips(p, s);
+    int64_t *rs, *ss, x, i, j, k;
+    if (q == 0) return 0;
+    rs = (int64_t *)malloc((size_t)p * q * sizeof(int64_t));
+    ss = (int64_t *)malloc((size_t)p * q * sizeof(int64_t));
+    if (!rs || !ss) { free(rs); free(ss); return -3; }
+    x = (q - ((int64_t)n - 1 + q) % q) % q;
+    for (j = 0; j < (int64_t)p; j++)
+        for (k = 0; k < q; k++) {
+            int64_t adj = !adjust ? 0 : k < x ? -x + q : -x;   /* adjust == 0: as printed (self-test) */
+            rs[j * q + k] = recv[j * q + k] + adj;
+            ss[j * q + k] = send[j * q + k] + adj;
+        }
+    i = x;
+    while (i < (int64_t)n + q - 1 + x) {
+        int64_t jr = i - x;
+        k = i % q;
+        for (j = 0; j < (int64_t)p; j++) {            /* pack */
+            int64_t rr = ((int64_t)r - j + p) % p, b = ss[rr * q + k];
+            if (b > (int64_t)n - 1) b = n - 1;
+            if (b < 0) b = -1;
+            pack[jr * p + j] = (int32_t)b;
+            ss[rr * q + k] += q;
+        }
+        for (j = 0; j < (int64_t)p; j++) {            /* unpack */
+            int64_t rr = ((int64_t)r - j + p) % p, b = rs[rr * q + k];
+            if (b > (int64_t)n - 1) b = n - 1;
+            if (b < 0) b = -1;
+            unpack[jr * p + j] = (int32_t)b;
+            rs[rr * q + k] += q;
+        }
+        i = i + 1;
+    }
+    free(rs); free(ss);
+    return 0;
+}
+
 /* Position-weighted 64-bit checksum of a stretch of schedule entries (not from
  * the paper: a tool for comparing outputs too large to copy).  Entry number e
  * of the whole stream is byte e mod 4 of the little-endian 32-bit word

@@ -9,6 +9,7 @@ library raises.
 from .binding import (  # noqa: F401
     BcsError,
     BatchPlan,
+    bcs_allgather_tables,
     bcs_batch_plan,
     bcs_build,
     bcs_build_batch,

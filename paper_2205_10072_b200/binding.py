@@ -68,6 +68,8 @@ def lib():
         L.bcs_expand.restype = i32
         L.bcs_validate.argtypes = [u32, u64, u64, vp, vp, vp, vp]
         L.bcs_validate.restype = i32
+        L.bcs_allgather_tables.argtypes = [u32, u32, u32, vp, vp, vp, vp, vp]
+        L.bcs_allgather_tables.restype = i32
         L.bcs_simulate.argtypes = [u32, u32, vp, vp, vp, vp, vp]
         L.bcs_simulate.restype = i32
         L.bcs_checksum.argtypes = [vp, u64, u64, vp, vp]
@@ -229,6 +231,14 @@ def bcs_validate(p: int, r_begin: int, r_end: int, recv, send, violations_out, s
     three elements: ranks with a bad receive row, a bad send row, a send/receive mismatch."""
     _check(lib().bcs_validate(p, r_begin, r_end, _ptr(recv), _ptr(send), _ptr(violations_out),
                               _stream(stream)), "bcs_validate")
+
+
+def bcs_allgather_tables(p: int, n: int, r: int, recv, send, pack_out, unpack_out,
+                         stream=None) -> None:
+    """recv/send: full [p][q] CUDA int8 tables; pack_out/unpack_out: CUDA int32 [n-1+q, p]
+    (or None): blocks of buffer[j] processor r packs / unpacks per round (Algorithm 9)."""
+    _check(lib().bcs_allgather_tables(p, n, r, _ptr(recv), _ptr(send), _ptr(pack_out),
+                                      _ptr(unpack_out), _stream(stream)), "bcs_allgather_tables")
 
 
 def bcs_simulate(p: int, n: int, recv, send, state, counts_out, stream=None) -> None:

@@ -81,3 +81,48 @@ def simulate(p, n, table, root=0):
         return "a non-root processor received a block %s times" % (
             "0" if (got[nonroot] == 0).any() else ">1")
     return None
+
+
+def simulate_allgather(p, n, pack, unpack):
+    """Brute-force run of the irregular allgather (Algorithm 9) on block numbers: pack[r] and
+    unpack[r] are processor r's int32 [n-1+q][p] tables (block of buffer j sent / received per
+    round).  Processor j owns all n blocks of buffer j.  Returns None if in every round every
+    sent block is held by its sender and is the one the to-processor unpacks for the same buffer,
+    every processor gets every block of every foreign buffer exactly once, and all are complete
+    after n-1+q rounds; else a description of the first violation."""
+    q = ceil_log2(p)
+    rounds = n - 1 + q
+    if p == 1:
+        return None
+    sk = closed_form_skips(p)
+    x = (q - (n - 1 + q) % q) % q
+    have = np.zeros((p, p, n), dtype=bool)          # [processor][buffer][block]
+    for j in range(p):
+        have[j, j, :] = True
+    got = np.zeros((p, p, n), dtype=np.int64)
+    procs = np.arange(p)
+    bufs = np.arange(p)
+    for jr in range(rounds):
+        k = (jr + x) % q
+        to = (procs + sk[k]) % p
+        sb = np.stack([pack[r][jr] for r in range(p)]).astype(np.int64)      # [proc][buffer]
+        rb = np.stack([unpack[r][jr] for r in range(p)]).astype(np.int64)
+        if (sb >= n).any() or (rb >= n).any() or (sb < -1).any() or (rb < -1).any():
+            return "round %d: block out of range" % jr
+        if not np.array_equal(rb[to], sb):
+            return "round %d: a packed block is not what the to-processor unpacks" % jr
+        snd = sb >= 0
+        pr, bf = np.nonzero(snd)
+        if not have[pr, bf, sb[snd]].all():
+            return "round %d: a processor packs a block it does not hold" % jr
+        rcv = rb >= 0
+        pr, bf = np.nonzero(rcv)
+        np.add.at(got, (pr, bf, rb[rcv]), 1)
+        have[pr, bf, rb[rcv]] = True
+    if not have.all():
+        return "not complete after n-1+q rounds"
+    foreign = procs[:, None] != bufs[None, :]
+    if not (got[foreign] == 1).all():
+        return "a block of a foreign buffer was received %s than once" % (
+            "fewer" if (got[foreign] == 0).any() else "more")
+    return None

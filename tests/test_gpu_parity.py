@@ -337,6 +337,53 @@ def test_expansion_small_cases_and_simulation(bcs):
                 assert bcast_sim.simulate(p, n, got) is None
 
 
+def test_allgather_tables_match_oracle(bcs):
+    """Algorithm 9's pack / unpack block numbers: every entry against the oracle's literal loops
+    for small p, the library's own tables simulated (all p processors) for tiny p, and the
+    expansion workload's size (p = 100003, n = 1000: 2 x 406 MB per processor) on sampled columns."""
+    for p in (2, 3, 9, 33, 257, 1000):
+        q = oracle.q_of(p)
+        want_r, want_s = oracle.full_table(p)
+        recv, send = torch.from_numpy(want_r).cuda(), torch.from_numpy(want_s).cuda()
+        for n in (1, 2, 5, q + 3, 70, 300):
+            rounds = n - 1 + q
+            tabs = []
+            for r in sorted({0, 1, p // 2, p - 1}) if p > 9 or n > 12 else range(p):
+                raw = torch.full((2 * rounds * p + 64,), -77, dtype=torch.int32, device="cuda")
+                pack = raw[32:32 + rounds * p].view(rounds, p)
+                unpack = raw[32 + rounds * p:32 + 2 * rounds * p].view(rounds, p)
+                bcs.bcs_allgather_tables(p, n, r, recv, send, pack, unpack)
+                torch.cuda.synchronize()
+                assert bool((raw[:32] == -77).all()) and bool((raw[-32:] == -77).all())
+                o_pack, o_unpack = oracle.allgather_rank(p, n, r, want_r, want_s)
+                assert np.array_equal(pack.cpu().numpy(), o_pack), (p, n, r)
+                assert np.array_equal(unpack.cpu().numpy(), o_unpack), (p, n, r)
+                tabs.append((pack.cpu().numpy(), unpack.cpu().numpy()))
+            if len(tabs) == p:
+                assert bcast_sim.simulate_allgather(p, n, [t[0] for t in tabs],
+                                                    [t[1] for t in tabs]) is None, (p, n)
+    p, n = workloads.P_EXPAND, workloads.N_EXPAND
+    q = oracle.q_of(p)
+    want_r, want_s = oracle.full_table(p)
+    recv, send = torch.from_numpy(want_r).cuda(), torch.from_numpy(want_s).cuda()
+    rounds = n - 1 + q
+    pack = torch.empty((rounds, p), dtype=torch.int32, device="cuda")
+    unpack = torch.empty((rounds, p), dtype=torch.int32, device="cuda")
+    r = 54607
+    bcs.bcs_allgather_tables(p, n, r, recv, send, pack, unpack)
+    E = oracle.expand(p, n, want_r, want_s)          # identity pinned on the CPU: virtual ranks
+    virt = (r - np.arange(p)) % p
+    assert np.array_equal(pack.cpu().numpy(), E[virt, :, 0].T)
+    assert np.array_equal(unpack.cpu().numpy(), E[virt, :, 1].T)
+    only = torch.full((rounds, p), -5, dtype=torch.int32, device="cuda")
+    bcs.bcs_allgather_tables(p, n, r, recv, send, None, only)
+    assert torch.equal(only, unpack)
+    L = bcs.lib()
+    assert L.bcs_allgather_tables(p, n, p, recv.data_ptr(), send.data_ptr(), pack.data_ptr(), None, None) == 2
+    assert L.bcs_allgather_tables(p, 0, 0, recv.data_ptr(), send.data_ptr(), pack.data_ptr(), None, None) == 1
+    assert L.bcs_allgather_tables(p, n, 0, recv.data_ptr(), send.data_ptr(), None, None, None) == 1
+
+
 def test_checksum_matches_oracle(bcs):
     rng = np.random.default_rng(11)
     out = torch.zeros(1, dtype=torch.int64, device="cuda")

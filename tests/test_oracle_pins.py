@@ -283,6 +283,46 @@ def test_simulation_rejects_planted_mistakes():
     assert bcast_sim.simulate(p, n, tab2) is not None
 
 
+# ---------------------------------------------------------------- Algorithm 9 index tables
+def test_allgather_tables_are_rerooted_broadcast_rounds():
+    """Processor r handles buffer j as virtual processor (r-j) mod p of a broadcast rooted at j
+    (Section 2.4): its pack / unpack blocks are the send / receive blocks of that virtual
+    processor's broadcast rounds (the expansion, pinned above)."""
+    for p in (2, 3, 9, 20, 33, 100):
+        q = oracle.q_of(p)
+        recv, send = oracle.full_table(p)
+        for n in (1, 2, 5, q + 3, 40):
+            E = oracle.expand(p, n, recv, send)                 # [virtual rank][round][4]
+            for r in {0, 1, p // 2, p - 1}:
+                pack, unpack = oracle.allgather_rank(p, n, r, recv, send)
+                virt = (r - np.arange(p)) % p
+                assert np.array_equal(pack, E[virt, :, 0].T), (p, n, r)
+                assert np.array_equal(unpack, E[virt, :, 1].T), (p, n, r)
+
+
+def test_allgather_simulation_and_the_need_for_the_adjustment():
+    """All p processors run Algorithm 9 on block numbers (tests/bcast_sim.py): every block of
+    every buffer arrives everywhere exactly once in n-1+q rounds.  Leaving out Algorithm 6's
+    adjustment of the schedules, as the printed Algorithm 9 does, breaks it whenever there are
+    virtual rounds (x != 0)."""
+    for p in (2, 3, 5, 9, 16, 20, 33):
+        q = oracle.q_of(p)
+        recv, send = oracle.full_table(p)
+        for n in (1, 2, 5, q + 3):
+            tabs = [oracle.allgather_rank(p, n, r, recv, send) for r in range(p)]
+            err = bcast_sim.simulate_allgather(p, n, [t[0] for t in tabs], [t[1] for t in tabs])
+            assert err is None, (p, n, err)
+            x = (q - (n - 1 + q) % q) % q
+            raw = [oracle.allgather_rank(p, n, r, recv, send, adjust=False) for r in range(p)]
+            err = bcast_sim.simulate_allgather(p, n, [t[0] for t in raw], [t[1] for t in raw])
+            assert (err is None) == (x == 0), (p, n, x, err)
+    p, n = 9, 5                                               # a planted mistake must be caught
+    recv, send = oracle.full_table(p)
+    tabs = [list(oracle.allgather_rank(p, n, r, recv, send)) for r in range(p)]
+    tabs[4][0][2, 3] = (tabs[4][0][2, 3] + 1) % n
+    assert bcast_sim.simulate_allgather(p, n, [t[0] for t in tabs], [t[1] for t in tabs]) is not None
+
+
 # ---------------------------------------------------------------- property checker
 def test_validator_accepts_valid_and_counts_planted_mistakes():
     """oracle.validate counts ranks whose rows break the promised properties.  Valid schedules
