@@ -178,6 +178,19 @@ bcs_status bcs_expand(uint32_t p, uint32_t n, uint64_t r_begin, uint64_t r_end,
                       const int8_t *recv, const int8_t *send, int32_t *table_out,
                       void *cuda_stream);
 
+/* Round tables of the two other algorithms on the same circulant graph (Section 2.3), whose
+ * edges run opposite to the broadcast's: q records of four int32 per rank, record of (r, k) at
+ * index (r - r_begin) * q + k.
+ *   census == 0, regular allgather (Algorithm 7): {to = (r - skips[k] + p) mod p,
+ *     from = (r + skips[k]) mod p, number of blocks exchanged = skips[k+1] - skips[k] (blocks
+ *     0..count-1 of the buffer are sent), offset skips[k] at which the received ones are stored};
+ *   census != 0, census / allreduce (Algorithm 8): {to, from, 1 if x_r (+) S is sent and 0 if S
+ *     alone, 0}; when skips[k] + skips[k] > skips[k+1] the edges are (r - skips[k] + 1) and
+ *     (r + skips[k] - 1) and S alone is sent (the listing writes skips[i]; k is meant).
+ * table_out: device, (r_end - r_begin) * q records, 16-byte aligned. */
+bcs_status bcs_circulant_rounds(uint32_t p, uint64_t r_begin, uint64_t r_end, int census,
+                                int32_t *table_out, void *cuda_stream);
+
 /* Index tables of the irregular allgather (Algorithm 9 without the pack / Send||Recv / unpack
  * data movement) for ONE processor r: in round jr (0..n-2+q) processor r packs block
  * pack_out[jr * p + j] of buffer[j] for its to-processor and unpacks what it receives into

@@ -74,6 +74,10 @@ def _load():
         lib.bcso_allgather_rank.argtypes = [c.c_uint32, c.c_uint32, c.c_uint32, i8p, i8p, c.c_int,
                                             c.POINTER(c.c_int32), c.POINTER(c.c_int32)]
         lib.bcso_allgather_rank.restype = c.c_int
+        lib.bcso_allgather_rounds.argtypes = [c.c_uint32, c.c_uint32, c.POINTER(c.c_int32)]
+        lib.bcso_allgather_rounds.restype = None
+        lib.bcso_census_rounds.argtypes = [c.c_uint32, c.c_uint32, c.POINTER(c.c_int32)]
+        lib.bcso_census_rounds.restype = None
         lib.bcso_set_root_mode.argtypes = [c.c_int]
         lib.bcso_set_root_mode.restype = None
         lib.bcso_num_threads.argtypes = []
@@ -246,6 +250,18 @@ def allgather_rank(p: int, n: int, r: int, recv, send, adjust: bool = True):
     if rc:
         raise RuntimeError("oracle allgather_rank failed: %d" % rc)
     return pack, unpack
+
+
+def circulant_rounds(p: int, r_begin: int, r_end: int, census: bool) -> np.ndarray:
+    """Round tables of Algorithm 7 (census=False: to, from, block count, receive offset) or
+    Algorithm 8 (census=True: to, from, 1 if x_r is added to what is sent, 0) -> int32 [ranks][q][4]."""
+    q = q_of(p)
+    out = np.zeros((r_end - r_begin, q, 4), dtype=np.int32)
+    fn = _load().bcso_census_rounds if census else _load().bcso_allgather_rounds
+    i32 = ctypes.POINTER(ctypes.c_int32)
+    for j, r in enumerate(range(r_begin, r_end)):
+        fn(p, r, out[j].ctypes.data_as(i32))
+    return out
 
 
 def set_root_mode(mode: int) -> None:

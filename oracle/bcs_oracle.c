@@ -451,6 +451,46 @@ void bcso_expand_range(uint32_t p, uint32_t n, uint64_t r_begin, uint64_t r_end,
     }
 }
 
+/* Algorithm 7 (regular allgather) without the data: for processor r and round k
+ * out[4k..4k+3] = to-processor (r - skips[k] + p) mod p, from-processor
+ * (r + skips[k]) mod p, number of blocks exchanged skips[k+1] - skips[k] (blocks
+ * 0..count-1 of the buffer are sent), offset skips[k] at which the received
+ * blocks are stored.  The edges run opposite to the broadcast's. */
+void bcso_allgather_rounds(uint32_t p, uint32_t r, int32_t *out)
+{
+    uint32_t s[BCSO_MAXQ + 1];
+    int q = bcso_skips(p, s), k;
+    for (k = 0; k < q; k++) {
+        out[4 * k + 0] = (int32_t)(((int64_t)r - s[k] + p) % p);
+        out[4 * k + 1] = (int32_t)(((int64_t)r + s[k]) % p);
+        out[4 * k + 2] = (int32_t)(s[k + 1] - s[k]);
+        out[4 * k + 3] = (int32_t)s[k];
+    }
+}
+
+/* Algorithm 8 (census / allreduce) without the data: for processor r and round
+ * k out[4k..4k+3] = to-processor, from-processor, 1 if the value sent is
+ * x_r (+) S and 0 if it is S alone, 0.  When skips[k] + skips[k] > skips[k+1]
+ * the edges are shortened by one and S alone is sent (the listing tests
+ * skips[i]; the round index k is meant). */
+void bcso_census_rounds(uint32_t p, uint32_t r, int32_t *out)
+{
+    uint32_t s[BCSO_MAXQ + 1];
+    int q = bcso_skips(p, s), k;
+    for (k = 0; k < q; k++) {
+        if ((uint64_t)s[k] + s[k] > s[k + 1]) {
+            out[4 * k + 0] = (int32_t)(((int64_t)r - s[k] + 1 + p) % p);
+            out[4 * k + 1] = (int32_t)(((int64_t)r + s[k] - 1) % p);
+            out[4 * k + 2] = 0;
+        } else {
+            out[4 * k + 0] = (int32_t)(((int64_t)r - s[k] + p) % p);
+            out[4 * k + 1] = (int32_t)(((int64_t)r + s[k]) % p);
+            out[4 * k + 2] = 1;
+        }
+        out[4 * k + 3] = 0;
+    }
+}
+
 /* Algorithm 9 without the data movement, for processor r: which block of
  * buffer[j] is packed (sent) and which is unpacked (received) in every round.
  * The full schedule is given (recv / send are the [p][q] tables of a root-0

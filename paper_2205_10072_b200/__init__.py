@@ -19,6 +19,7 @@ from .binding import (  # noqa: F401
     bcs_build_workspace_bytes,
     bcs_build_to_host,
     bcs_checksum,
+    bcs_circulant_rounds,
     bcs_expand,
     bcs_prepare,
     bcs_prepare_workspace_bytes,

@@ -68,6 +68,8 @@ def lib():
         L.bcs_expand.restype = i32
         L.bcs_validate.argtypes = [u32, u64, u64, vp, vp, vp, vp]
         L.bcs_validate.restype = i32
+        L.bcs_circulant_rounds.argtypes = [u32, u64, u64, i32, vp, vp]
+        L.bcs_circulant_rounds.restype = i32
         L.bcs_allgather_tables.argtypes = [u32, u32, u32, vp, vp, vp, vp, vp]
         L.bcs_allgather_tables.restype = i32
         L.bcs_simulate.argtypes = [u32, u32, vp, vp, vp, vp, vp]
@@ -231,6 +233,14 @@ def bcs_validate(p: int, r_begin: int, r_end: int, recv, send, violations_out, s
     three elements: ranks with a bad receive row, a bad send row, a send/receive mismatch."""
     _check(lib().bcs_validate(p, r_begin, r_end, _ptr(recv), _ptr(send), _ptr(violations_out),
                               _stream(stream)), "bcs_validate")
+
+
+def bcs_circulant_rounds(p: int, r_begin: int, r_end: int, census: bool, table_out,
+                         stream=None) -> None:
+    """table_out: CUDA int32 [(r_end-r_begin), q, 4]: rounds of Algorithm 7 (census=False) or
+    Algorithm 8 (census=True)."""
+    _check(lib().bcs_circulant_rounds(p, r_begin, r_end, int(census), _ptr(table_out),
+                                      _stream(stream)), "bcs_circulant_rounds")
 
 
 def bcs_allgather_tables(p: int, n: int, r: int, recv, send, pack_out, unpack_out,

@@ -61,6 +61,36 @@ expand_kernel(PTable tab, uint32_t n, uint64_t r_begin, uint64_t r_end,
     }
 }
 
+// ---------------------------------------------------------------- Algorithms 7 and 8: round tables
+// One 16-byte record per (rank, round k), q records per rank.  Regular allgather (Algorithm 7):
+// {to = r - skips[k], from = r + skips[k] (mod p), blocks exchanged skips[k+1] - skips[k],
+// receive offset skips[k]}.  Census (Algorithm 8): when 2 skips[k] > skips[k+1] the edges are one
+// shorter and only the partial sum S is sent: {to, from, 1 if x_r is added to what is sent, 0}.
+__global__ void __launch_bounds__(256)
+circulant_rounds_kernel(PTable tab, uint64_t r_begin, uint64_t n_records, int census,
+                        int4 *__restrict__ out)
+{
+    const uint64_t e = (uint64_t)blockIdx.x * 256 + threadIdx.x;
+    if (e >= n_records) return;
+    const uint32_t q = (uint32_t)tab.q, p = tab.p;
+    const uint64_t j = e / q;
+    const uint32_t k = (uint32_t)(e - j * q);
+    const uint32_t r = (uint32_t)(r_begin + j);
+    const uint32_t lo = tab.s[k], hi = tab.s[k + 1];
+    uint32_t step = lo;
+    int c = (int)(hi - lo), d = (int)lo;
+    if (census) {
+        const bool shorter = 2ull * lo > hi;
+        step = shorter ? lo - 1u : lo;
+        c = shorter ? 0 : 1;
+        d = 0;
+    }
+    const uint32_t to = r >= step ? r - step : r + p - step;
+    uint32_t from = r + step;
+    if (from >= p) from -= p;
+    __stcs(out + e, make_int4((int)to, (int)from, c, d));
+}
+
 }  // namespace
 }  // namespace bcs
 
@@ -85,6 +115,24 @@ bcs_status bcs_expand(uint32_t p, uint32_t n, uint64_t r_begin, uint64_t r_end,
     const unsigned blocks = (unsigned)((count + kExpandRanks - 1) / kExpandRanks);
     expand_kernel<<<blocks, kExpandThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
         tab, n, r_begin, r_end, recv, send, reinterpret_cast<int4 *>(table_out));
+    return launch_status();
+}
+
+bcs_status bcs_circulant_rounds(uint32_t p, uint64_t r_begin, uint64_t r_end, int census,
+                                int32_t *table_out, void *cuda_stream)
+{
+    bcs_status st = check_range(p, r_begin, r_end);
+    if (st != BCS_OK) return st;
+    PTable tab;
+    make_table(p, &tab);
+    const uint64_t records = (r_end - r_begin) * (uint64_t)tab.q;
+    if (records == 0) return BCS_OK;
+    if (table_out == nullptr) return BCS_ERR_ARG;
+    if (!aligned16(table_out)) return BCS_ERR_ALIGN;
+    const uint64_t blocks = (records + 255) / 256;
+    if (blocks > 0x7fffffffull) return BCS_ERR_UNSUPPORTED;
+    circulant_rounds_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        tab, r_begin, records, census != 0, reinterpret_cast<int4 *>(table_out));
     return launch_status();
 }
 

@@ -384,6 +384,20 @@ def test_allgather_tables_match_oracle(bcs):
     assert L.bcs_allgather_tables(p, n, 0, recv.data_ptr(), send.data_ptr(), None, None, None) == 1
 
 
+def test_circulant_round_tables_match_oracle(bcs):
+    """Algorithms 7 and 8: neighbour / range records for every rank and round."""
+    for p, r0, r1 in ((1, 0, 1), (2, 0, 2), (33, 0, 33), (1000, 0, 1000), (100003, 0, 100003),
+                      (100003, 4321, 5000), (2**31 - 1, 2**31 - 300, 2**31 - 1)):
+        q = oracle.q_of(p)
+        for census in (False, True):
+            raw = torch.full(((r1 - r0) * q * 4 + 128,), -9, dtype=torch.int32, device="cuda")
+            tab = raw[64:64 + (r1 - r0) * q * 4].view(r1 - r0, q, 4)
+            bcs.bcs_circulant_rounds(p, r0, r1, census, tab if q else raw[64:])
+            torch.cuda.synchronize()
+            assert bool((raw[:64] == -9).all()) and bool((raw[-64:] == -9).all())
+            assert np.array_equal(tab.cpu().numpy(), oracle.circulant_rounds(p, r0, r1, census)), (p, census)
+
+
 def test_checksum_matches_oracle(bcs):
     rng = np.random.default_rng(11)
     out = torch.zeros(1, dtype=torch.int64, device="cuda")

@@ -323,6 +323,50 @@ def test_allgather_simulation_and_the_need_for_the_adjustment():
     assert bcast_sim.simulate_allgather(p, n, [t[0] for t in tabs], [t[1] for t in tabs]) is not None
 
 
+# ---------------------------------------------------------------- Algorithms 7 and 8
+def test_regular_allgather_rounds_gather_everything():
+    """Algorithm 7 run on block identities: processor r starts with its own block in buffer[0];
+    after q rounds buffer[i] holds the block of processor (r+i) mod p for every i."""
+    for p in list(range(1, 70)) + [100, 127, 128, 129, 1000]:
+        q = oracle.q_of(p)
+        tab = oracle.circulant_rounds(p, 0, p, census=False)
+        buf = np.full((p, p), -1, dtype=np.int64)
+        buf[:, 0] = np.arange(p)
+        filled = 1
+        for k in range(q):
+            to, fr, cnt, off = (tab[:, k, c].astype(np.int64) for c in range(4))
+            assert (cnt == cnt[0]).all() and (off == off[0]).all() and off[0] == filled
+            assert np.array_equal(fr[to], np.arange(p))          # to/from are mutually consistent
+            c, o = int(cnt[0]), int(off[0])
+            assert c <= filled                                    # only blocks it already has
+            sent = buf[:, :c].copy()                              # everybody sends buffer[0..c-1]
+            buf[:, o:o + c] = sent[fr]                            # and stores what arrives at skips[k]
+            filled += c
+        assert filled == p
+        assert np.array_equal(buf, (np.arange(p)[:, None] + np.arange(p)[None, :]) % p), p
+
+
+def test_census_rounds_sum_every_input_once():
+    """Algorithm 8 with + on random integers: every processor ends with the total, i.e. every
+    input is counted exactly once (the invariant S = sum of the next skips[k+1]-1 inputs)."""
+    rng = np.random.default_rng(8)
+    for p in list(range(1, 70)) + [100, 127, 128, 129, 1000]:
+        q = oracle.q_of(p)
+        s = [int(v) for v in oracle.skips(p)]
+        tab = oracle.circulant_rounds(p, 0, p, census=True)
+        x = rng.integers(1, 10**6, p)
+        S = np.zeros(p, dtype=np.int64)
+        for k in range(q):
+            to, fr, own = (tab[:, k, c].astype(np.int64) for c in range(3))
+            assert np.array_equal(fr[to], np.arange(p))
+            assert (own == (0 if 2 * s[k] > s[k + 1] else 1)).all()
+            O = np.where(own == 1, x + S, S)
+            S = S + O[fr]
+            want = sum(np.roll(x, -i) for i in range(1, s[k + 1]))   # x_{r+1} .. x_{r+skips[k+1]-1}
+            assert np.array_equal(S, want if s[k + 1] > 1 else np.zeros(p, dtype=np.int64)), (p, k)
+        assert np.array_equal(S + x, np.full(p, x.sum())), p
+
+
 # ---------------------------------------------------------------- property checker
 def test_validator_accepts_valid_and_counts_planted_mistakes():
     """oracle.validate counts ranks whose rows break the promised properties.  Valid schedules
