@@ -367,27 +367,32 @@ recv_codes_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, BatchArgs ba,
 // sum_{j<=i} skips[j] <= 32 -- are OR-ed together from warp shuffles, one per distance, the
 // same for all lanes.  These are the rounds in which neighbouring ranks disagree about which
 // path of the code search they take; the later rounds run the code search per lane.
-template <bool kRowOut, bool kColOut>
-__global__ void __launch_bounds__(kTile, 8)
-recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uint64_t r_end,
-                       const uint32_t *__restrict__ codes, int8_t *recv_out, int8_t *recv_t,
-                       uint64_t t_stride)
+// Where the skips of the tile's p are read from: the kernel parameter (single p: immediate /
+// constant-bank operands) or a table row in shared memory (batch).
+struct ParamSkips {
+    const PTable &tab;
+    __device__ __forceinline__ uint32_t operator()(int k) const { return tab.s[k]; }
+};
+struct SharedSkips {
+    const uint32_t *s;
+    __device__ __forceinline__ uint32_t operator()(int k) const { return s[k]; }
+};
+
+// The tile is the n ranks first..first+n-1 of a p (n <= 256, one per thread); `stage` is where
+// the tile's rank-major rows start in shared memory, `col` this thread's element of round 0 in
+// the round-major copy.  All 256 threads must call (the warp rounds use every lane).
+template <bool kRowOut, bool kColOut, class Skips>
+__device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t *full_sh,
+                                               uint32_t p, int q, uint64_t first, uint32_t n,
+                                               const uint32_t *__restrict__ codes, uint8_t *stage,
+                                               int8_t *col, uint64_t t_stride)
 {
-    __shared__ __align__(16) uint8_t stage[kTile * 32];
-    __shared__ uint32_t full_sh[kRow];
     constexpr unsigned kAll = 0xffffffffu;
-    const uint32_t p = tab.p;
-    const int q = tab.q;
-    if (threadIdx.x < kRow) full_sh[threadIdx.x] = tab.full[threadIdx.x];
-    __syncthreads();
-    const uint64_t count = r_end - r_begin;
-    const uint64_t g0 = (uint64_t)blockIdx.x * kTile;
-    const uint64_t g = g0 + threadIdx.x;
-    const bool valid = g < count;
+    const bool valid = threadIdx.x < n;
     const uint32_t lane = threadIdx.x & 31u;
     // ranks of this lane and of the lane 32 ranks before it, mod p (defined for every lane of the
     // warp, also past the end of the range: only lower lanes and `before` are read by others)
-    uint64_t wrapped = r_begin + g;
+    uint64_t wrapped = first + threadIdx.x;
     while (wrapped >= p) wrapped -= p;
     const uint32_t r = (uint32_t)wrapped;
     const uint32_t r_before = r >= 32u ? r - 32u : r + p - 32u;
@@ -405,7 +410,6 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uin
     }
     st.sum = 0;
     uint8_t *row = stage + threadIdx.x * q;
-    int8_t *col = kColOut ? recv_t + g : nullptr;
     // run[j] / run_before[j]: baseblock bits OR-ed over the 2^j ranks ending at this lane's rank,
     // resp. at the rank 32 below it (doubling; a lane's run may start in the 32 ranks before the
     // warp).  A window of L ranks is the union of two runs of 2^floor(log2 L) ranks.
@@ -429,8 +433,8 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uin
     };
     int i = 0;
 #pragma unroll 1
-    for (; i < q && tab.s[i + 1] <= 33u; ++i) {            // uniform over the grid
-        const uint32_t lo = tab.s[i], hi = tab.s[i + 1];
+    for (; i < q && skip(i + 1) <= 33u; ++i) {            // uniform over the grid
+        const uint32_t lo = skip(i), hi = skip(i + 1);
         st.sum += lo;
         // ranks r - d, d = lo..hi-1: runs of 2^j ranks ending at r - lo and at r - (hi - 2^j)
         uint32_t acc;
@@ -476,12 +480,12 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uin
     if (valid && i < q) {
         // Per-lane rounds.  Before the home round h both window bounds are r - skip, after it
         // both are r + p - skip: two loops with the wrap decided once, the home round between.
-        const uint32_t edge = tab.s[i];
+        const uint32_t edge = skip(i);
         st.lo_skip = edge;
         st.upper = codes[r - edge + (r >= edge ? 0u : p)];  // code of r - skips[i]
         uint8_t *out = row + i;
         auto round = [&](int ii, uint32_t from) {           // from = r or r + p
-            const uint32_t hi = tab.s[ii + 1];
+            const uint32_t hi = skip(ii + 1);
             st.sum += st.lo_skip;
             st.lo_skip = hi;
             const uint32_t below = from - hi;
@@ -507,7 +511,7 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uin
 #pragma unroll 1
         for (; i < h; ++i) round(i, r);
         if (i == h) {                                        // home round: the baseblock itself
-            const uint32_t hi = tab.s[i + 1];
+            const uint32_t hi = skip(i + 1);
             st.sum += st.lo_skip;
             st.lo_skip = hi;
             st.upper = codes[r + p - hi];
@@ -522,12 +526,30 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uin
 #pragma unroll 1
         for (; i < q; ++i) round(i, rp);
     }
+}
+
+template <bool kRowOut, bool kColOut>
+__global__ void __launch_bounds__(kTile, 8)
+recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uint64_t r_end,
+                       const uint32_t *__restrict__ codes, int8_t *recv_out, int8_t *recv_t,
+                       uint64_t t_stride)
+{
+    __shared__ __align__(16) uint8_t stage[kTile * 32];
+    __shared__ uint32_t full_sh[kRow];
+    if (threadIdx.x < kRow) full_sh[threadIdx.x] = tab.full[threadIdx.x];
+    __syncthreads();
+    const uint64_t count = r_end - r_begin;
+    const uint64_t g0 = (uint64_t)blockIdx.x * kTile;
+    const uint32_t n = (uint32_t)(count - g0 < (uint64_t)kTile ? count - g0 : (uint64_t)kTile);
+    recv_warp_tile<kRowOut, kColOut>(ParamSkips{tab}, full_sh, tab.p, tab.q, r_begin + g0, n, codes,
+                                     stage, kColOut ? recv_t + g0 + threadIdx.x : nullptr,
+                                     t_stride);
     if (kRowOut) {
         __syncthreads();
-        const uint64_t g1 = g0 + kTile < count ? g0 + kTile : count;
-        flush_span(stage, 0, (uint32_t)((g1 - g0) * (uint64_t)q), recv_out, g0 * (uint64_t)q);
+        flush_span(stage, 0, n * (uint32_t)tab.q, recv_out, g0 * (uint64_t)tab.q);
     }
 }
+
 
 // Send rows from the round-major receive copy.  kAllInside: every to-processor's row is in
 // the copy (all ranks of the p).  Otherwise (single p, sub-range) to-processors outside the
