@@ -120,6 +120,23 @@ __device__ __forceinline__ uint32_t find_segment(const uint64_t *off, uint32_t l
     return lo;
 }
 
+// The same search by a whole warp: 32 probes per step instead of one, so a table of a few
+// thousand offsets takes three dependent loads instead of twelve.  All 32 lanes must call.
+__device__ __forceinline__ uint32_t find_segment_warp(const uint64_t *off, uint32_t num, uint64_t g)
+{
+    const uint32_t lane = threadIdx.x & 31u;
+    uint32_t lo = 0, hi = num;                       // answer in [lo, hi)
+    while (hi - lo > 1u) {
+        const uint32_t step = (hi - lo + 31u) / 32u;
+        const uint32_t idx = lo + lane * step;
+        const bool le = idx < hi && off[idx] <= g;
+        const uint32_t hits = __popc(__ballot_sync(0xffffffffu, le));   // lane 0 always hits
+        lo += (hits - 1u) * step;
+        hi = lo + step < hi ? lo + step : hi;
+    }
+    return lo;
+}
+
 // Resolves the rank this thread works on.  Single p: consecutive ranks from r_begin.
 // Batch: flattened index g over all (p_j, r); the CTA looks up the first and last p it
 // touches once, keeps the first few table rows in shared memory, and each thread finds
@@ -156,15 +173,17 @@ __device__ __forceinline__ RankCtx resolve_rank(TileShared &sh, const PTable &ta
         return c;
     }
     const uint64_t g1 = g0 + kTile < ba.total_ranks ? g0 + kTile : ba.total_ranks;
-    if (threadIdx.x == 0) {
-        uint32_t jf = find_segment(ba.rank_off, 0, ba.num_p - 1, g0);
-        uint32_t jl = find_segment(ba.rank_off, jf, ba.num_p - 1, g1 - 1);
+    if (threadIdx.x < 32) {
+        const uint32_t jf = find_segment_warp(ba.rank_off, ba.num_p, g0);
+        const uint32_t jl = ba.rank_off[jf + 1] >= g1 ? jf : find_segment_warp(ba.rank_off, ba.num_p, g1 - 1);
+        if (threadIdx.x == 0) {
         sh.j_first = jf;
         sh.j_last = jl;
         int qf = ceil_log2_fast(ba.p_list[jf]);
         int ql = ceil_log2_fast(ba.p_list[jl]);
         sh.span_begin = ba.entry_off[jf] + (g0 - ba.rank_off[jf]) * (uint64_t)qf;
         sh.span_end = ba.entry_off[jl] + (g1 - ba.rank_off[jl]) * (uint64_t)ql;
+        }
     }
     __syncthreads();
     const uint32_t jf = sh.j_first, jl = sh.j_last;

@@ -551,6 +551,36 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uin
 }
 
 
+// Batch: a CTA whose 256 flattened ranks all belong to one p >= 64 (nearly all CTAs when the p
+// are large) runs the warp-cooperative tile with that p's table rows from shared memory; a CTA
+// that straddles several p, or a small p, runs the per-lane search.
+template <bool kColOut>
+__global__ void __launch_bounds__(kTile)
+recv_codes_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t *recv_out,
+                        int8_t *recv_t)
+{
+    __shared__ TileShared sh;
+    PTable unused;
+    RankCtx c = resolve_rank<true>(sh, unused, 0, 0, ba);
+    const uint32_t shift = (uint32_t)(sh.span_begin & 15u);
+    if (sh.j_first == sh.j_last && c.p >= 64u) {             // uniform over the CTA
+        const uint64_t g0 = (uint64_t)blockIdx.x * kTile;
+        const uint32_t n = (uint32_t)(ba.total_ranks - g0 < (uint64_t)kTile ? ba.total_ranks - g0
+                                                                             : (uint64_t)kTile);
+        const uint64_t first = g0 - c.rank0;
+        int8_t *col = kColOut ? recv_t + ba.entry_off[c.pj] + first + threadIdx.x : nullptr;
+        recv_warp_tile<true, kColOut>(SharedSkips{sh.skips[0]}, sh.full[0], c.p, c.q, first, n,
+                                      codes + c.rank0, sh.stage + shift, col, (uint64_t)c.p);
+    } else if (c.valid && c.q > 0) {
+        int8_t *col = kColOut ? recv_t + ba.entry_off[c.pj] + c.r : nullptr;
+        uint8_t *row = sh.stage + shift + (c.entry - sh.span_begin);
+        recv_rounds_codes<true, kColOut>(codes + c.rank0, c.s, c.full, c.p, c.q, c.r, c.q - 1, row,
+                                         col, (uint64_t)c.p);
+    }
+    __syncthreads();
+    flush_span(sh.stage, shift, (uint32_t)(sh.span_end - sh.span_begin), recv_out, sh.span_begin);
+}
+
 // Send rows from the round-major receive copy.  kAllInside: every to-processor's row is in
 // the copy (all ranks of the p).  Otherwise (single p, sub-range) to-processors outside the
 // range are recomputed from the codes (Algorithm 5).
@@ -603,80 +633,116 @@ send_rm_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, BatchArgs ba,
     flush_span(sh.stage, shift, (uint32_t)(sh.span_end - sh.span_begin), send_out, sh.span_begin);
 }
 
-// All ranks of a single p: row k of the round-major send table is row k of the round-major
-// receive copy rotated by skips[k] (sendsched[r][k] = recvsched[(r+skips[k]) mod p][k]), so
-// the send table is a transposition with one rotation per row.  A CTA takes 256 consecutive
-// ranks: for every round it copies the 256 (rotated, possibly wrapping) bytes it needs with
-// 16-byte loads into shared memory, then every thread gathers its column into the rank-major
-// staging rows, which leave as one vectorised span.
+// Row k of the round-major send table is row k of the round-major receive copy rotated by
+// skips[k] (sendsched[r][k] = recvsched[(r+skips[k]) mod p][k]), so the send rows of a run of
+// ranks are a transposition with one rotation per row (and the receive rows the same with
+// rotation 0).  A CTA takes up to 256 consecutive ranks: for every round it copies the
+// (rotated, possibly wrapping) bytes it needs with 16-byte loads into shared memory, then every
+// thread gathers its column into the rank-major staging rows, which leave as one vectorised span.
 constexpr int kTrPitch = kTile + 32;      // bytes per round in shared memory: 256 + alignment slack
 
+struct TransposeShared {
+    __align__(16) uint8_t rounds[BCS_MAX_Q * kTrPitch];
+    uint32_t lead[BCS_MAX_Q];   // offset of the tile's first byte inside its pitch row
+    uint32_t wraps;             // rounds whose bytes pass the end of the row
+};
+
+// tbl: round 0 of the round-major table of this p (all p ranks per row, rows `stride` bytes
+// apart, any alignment; up to 15 bytes before a row's first and after its last needed byte are
+// read as well).  The tile is ranks r0..r0+n-1; stage: where its rank-major rows start.
+template <class Skips>
+__device__ __forceinline__ void transpose_tile(const Skips skip, uint32_t p, int q,
+                                               const int8_t *__restrict__ tbl, uint64_t stride,
+                                               uint32_t r0, uint32_t n, bool rotate,
+                                               TransposeShared &ts, uint8_t *stage)
+{
+    if (threadIdx.x == 0) ts.wraps = 0;
+    __syncthreads();
+    const int vecs = kTrPitch / 16;         // 18 vectors cover 256 bytes at any misalignment
+    for (int w = threadIdx.x; w < q * vecs; w += kTile) {
+        const int k = w / vecs, v = w - k * vecs;
+        const uint8_t *src_row = reinterpret_cast<const uint8_t *>(tbl) + (uint64_t)k * stride;
+        uint32_t start = r0 + (rotate ? skip(k) : 0u);
+        if (start >= p) start -= p;
+        const uint32_t mis = (uint32_t)(reinterpret_cast<uintptr_t>(src_row + start) & 15u);
+        const uint32_t run = p - start < n ? p - start : n;      // bytes before the wrap
+        if (v == 0) {
+            ts.lead[k] = mis;
+            if (run < n) atomicOr(&ts.wraps, 1u << k);
+        }
+        if ((uint32_t)v * 16u < mis + run)                        // the vector holds a needed byte
+            *reinterpret_cast<uint4 *>(ts.rounds + k * kTrPitch + v * 16) =
+                *reinterpret_cast<const uint4 *>(src_row + start - mis + v * 16);
+    }
+    __syncthreads();
+    for (uint32_t left = ts.wraps; left != 0; left &= left - 1u) {  // the part after the wrap, by bytes
+        const int k = __ffs(left) - 1;
+        uint32_t start = r0 + (rotate ? skip(k) : 0u);
+        if (start >= p) start -= p;
+        const uint32_t run = p - start;                           // < n for these rounds
+        const uint8_t *src_row = reinterpret_cast<const uint8_t *>(tbl) + (uint64_t)k * stride;
+        const uint32_t j = threadIdx.x;
+        if (j >= run && j < n) ts.rounds[k * kTrPitch + ts.lead[k] + j] = src_row[j - run];
+    }
+    if (ts.wraps) __syncthreads();
+    // lane l of warp w takes rank 128 * (w / 4) + 4 * l + (w % 4): the rows written by one
+    // warp start q * 4 bytes = q words apart, which is a different bank for every lane when q
+    // is odd, and the bytes it reads lie in 32 consecutive words.
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const uint32_t mine = 128u * (warp >> 2) + 4u * lane + (warp & 3u);
+    if (mine < n) {
+        uint8_t *__restrict__ row = stage + mine * q;
+        const uint8_t *__restrict__ column = ts.rounds + mine;
+        const uint32_t *__restrict__ lead_k = ts.lead;
+#pragma unroll 4
+        for (int k = 0; k < q; ++k) row[k] = column[k * kTrPitch + lead_k[k]];
+    }
+}
+
+// Single p: recv_t holds all p ranks of every round; the CTA's tile is ranks r0..r0+n-1 of the
+// range r_begin..r_begin+count-1.  rotate: send rows; otherwise the receive rows themselves.
 __global__ void __launch_bounds__(kTile)
 send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restrict__ recv_t,
                       uint64_t t_stride, int8_t *send_out, uint32_t r_begin, uint32_t count,
                       bool rotate)
 {
-    __shared__ __align__(16) uint8_t rounds[BCS_MAX_Q * kTrPitch];
+    __shared__ TransposeShared ts;
     __shared__ __align__(16) uint8_t stage[kTile * 32];
-    __shared__ uint32_t lead[BCS_MAX_Q];   // offset of the tile's first byte inside its pitch row
-    __shared__ uint32_t wraps;             // rounds whose 256 bytes pass the end of the row
-    const uint32_t p = tab.p;
-    const int q = tab.q;
-    // recv_t holds all p ranks of every round; the tile is ranks r0..r0+n-1 of the range
-    // r_begin..r_begin+count-1.  rotate: send rows (rank r + skips[k] in round k); otherwise the
-    // rows of recv_t themselves, rank-major (rotation 0).
     const uint32_t first = blockIdx.x * kTile;
-    const uint32_t r0 = r_begin + first;
     const uint32_t n = count - first < (uint32_t)kTile ? count - first : (uint32_t)kTile;
-    if (threadIdx.x == 0) wraps = 0;
+    transpose_tile(ParamSkips{tab}, tab.p, tab.q, recv_t, t_stride, r_begin + first, n, rotate, ts,
+                   stage);
     __syncthreads();
-    // one 16-byte piece per (round, vector): kTrPitch / 16 = 18 vectors cover 256 bytes at any
-    // misalignment.  The tile's bytes of round k are recv_t[k][(r0 + skips[k] + j) mod p], j < n:
-    // one run, or two when it passes the end of the row.
-    const int vecs = kTrPitch / 16;
-    for (int w = threadIdx.x; w < q * vecs; w += kTile) {
-        const int k = w / vecs, v = w - k * vecs;
-        const uint8_t *src_row = reinterpret_cast<const uint8_t *>(recv_t) + (uint64_t)k * t_stride;
-        uint32_t start = r0 + (rotate ? tab.s[k] : 0u);
-        if (start >= p) start -= p;
-        const uint32_t mis = start & 15u;                 // rows start 16-byte aligned (t_stride % 16 == 0)
-        const uint32_t run = p - start < n ? p - start : n;      // bytes before the wrap
-        if (v == 0) {
-            lead[k] = mis;
-            if (run < n) atomicOr(&wraps, 1u << k);
-        }
-        uint8_t *dst = rounds + k * kTrPitch + v * 16;
-        const uint32_t at = start - mis + (uint32_t)v * 16u;      // aligned position in the row
-        if (at < start + run)                                     // at + 16 <= t_stride follows
-            *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src_row + at);
-    }
-    __syncthreads();
-    for (uint32_t left = wraps; left != 0; left &= left - 1u) {  // the part after the wrap, by bytes
-        const int k = __ffs(left) - 1;
-        uint32_t start = r0 + (rotate ? tab.s[k] : 0u);
-        if (start >= p) start -= p;
-        const uint32_t run = p - start;                           // < n for these rounds
-        const uint8_t *src_row = reinterpret_cast<const uint8_t *>(recv_t) + (uint64_t)k * t_stride;
-        const uint32_t j = threadIdx.x;
-        if (j >= run && j < n) rounds[k * kTrPitch + (start & 15u) + j] = src_row[j - run];
-    }
-    if (wraps) __syncthreads();
-    {
-        // lane l of warp w takes rank 128 * (w / 4) + 4 * l + (w % 4): the rows written by one
-        // warp start q * 4 bytes = q words apart, which is a different bank for every lane when q
-        // is odd, and the bytes it reads lie in 32 consecutive words.
-        const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-        const uint32_t mine = 128u * (warp >> 2) + 4u * lane + (warp & 3u);
-        if (mine < n) {
-            uint8_t *__restrict__ row = stage + mine * q;
-            const uint8_t *__restrict__ column = rounds + mine;
-            const uint32_t *__restrict__ lead_k = lead;
-#pragma unroll 4
-            for (int k = 0; k < q; ++k) row[k] = column[k * kTrPitch + lead_k[k]];
+    flush_span(stage, 0, n * (uint32_t)tab.q, send_out, (uint64_t)first * (uint64_t)tab.q);
+}
+
+// Batch: a CTA inside one p transposes; a CTA that straddles several p gathers byte by byte.
+__global__ void __launch_bounds__(kTile)
+send_batch_kernel(BatchArgs ba, const int8_t *__restrict__ recv_t, int8_t *send_out)
+{
+    __shared__ TileShared sh;
+    __shared__ TransposeShared ts;
+    PTable unused;
+    RankCtx c = resolve_rank<true>(sh, unused, 0, 0, ba);
+    const uint32_t shift = (uint32_t)(sh.span_begin & 15u);
+    if (sh.j_first == sh.j_last) {                            // uniform over the CTA
+        const uint64_t g0 = (uint64_t)blockIdx.x * kTile;
+        const uint32_t n = (uint32_t)(ba.total_ranks - g0 < (uint64_t)kTile ? ba.total_ranks - g0
+                                                                             : (uint64_t)kTile);
+        if (c.q > 0)
+            transpose_tile(SharedSkips{sh.skips[0]}, c.p, c.q, recv_t + ba.entry_off[c.pj],
+                           (uint64_t)c.p, (uint32_t)(g0 - c.rank0), n, true, ts, sh.stage + shift);
+    } else if (c.valid) {
+        uint8_t *row = sh.stage + shift + (c.entry - sh.span_begin);
+        const int8_t *tbl = recv_t + ba.entry_off[c.pj];
+        for (int k = 0; k < c.q; ++k) {
+            uint32_t t = c.r + c.s[k];
+            if (t >= c.p) t -= c.p;
+            row[k] = (uint8_t)tbl[(uint64_t)k * c.p + t];
         }
     }
     __syncthreads();
-    flush_span(stage, 0, n * (uint32_t)q, send_out, (uint64_t)first * (uint64_t)q);
+    flush_span(sh.stage, shift, (uint32_t)(sh.span_end - sh.span_begin), send_out, sh.span_begin);
 }
 
 struct Workspace {
@@ -889,7 +955,7 @@ bcs_status bcs_build_to_host(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_
 size_t bcs_build_batch_workspace_bytes(uint64_t total_ranks, uint64_t total_entries)
 {
     if (total_ranks == 0 || total_entries == 0) return 0;
-    return (size_t)(align_up(4ull * total_ranks, 256) + total_entries);
+    return (size_t)(align_up(4ull * total_ranks, 256) + align_up(total_entries, 16) + 16);
 }
 
 bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_dev,
@@ -920,15 +986,12 @@ bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_
         codes_kernel<true><<<blocks, kTile, 0, stream>>>(none, ba, codes);
         if ((st = launch_status()) != BCS_OK) return st;
         if (send_out != nullptr)
-            recv_codes_kernel<true, true, true><<<blocks, kTile, 0, stream>>>(none, 0, 0, ba, codes,
-                                                                              recv_out, recv_t, 0);
+            recv_codes_batch_kernel<true><<<blocks, kTile, 0, stream>>>(ba, codes, recv_out, recv_t);
         else
-            recv_codes_kernel<true, true, false><<<blocks, kTile, 0, stream>>>(none, 0, 0, ba, codes,
-                                                                               recv_out, nullptr, 0);
+            recv_codes_batch_kernel<false><<<blocks, kTile, 0, stream>>>(ba, codes, recv_out, nullptr);
         if ((st = launch_status()) != BCS_OK) return st;
         if (send_out != nullptr) {
-            send_rm_kernel<true, true><<<blocks, kTile, 0, stream>>>(none, 0, 0, ba, codes, recv_t,
-                                                                     0, send_out);
+            send_batch_kernel<<<blocks, kTile, 0, stream>>>(ba, recv_t, send_out);
             if ((st = launch_status()) != BCS_OK) return st;
         }
         return BCS_OK;

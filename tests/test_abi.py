@@ -89,7 +89,7 @@ def test_argument_errors_need_no_gpu(lib):
     assert L.bcs_build(10, 3, 3, None, None, None, 0, None) == 0 # empty range
     assert L.bcs_build_workspace_bytes(2**20 + 1, 0, 2**20 + 1) == 4194560 + 21 * 1048592
     assert L.bcs_build_workspace_bytes(0, 0, 0) == 0
-    assert L.bcs_build_batch_workspace_bytes(1000, 9000) == 4096 + 9000
+    assert L.bcs_build_batch_workspace_bytes(1000, 9000) == 4096 + 9008 + 16
     assert L.bcs_expand(10, 0, 0, 10, 16, 16, 16, None) == 1     # n == 0
     assert L.bcs_expand(10, 4, 0, 10, None, 16, 16, None) == 1
     assert L.bcs_expand(10, 4, 0, 10, 16, 16, 8, None) == 3
