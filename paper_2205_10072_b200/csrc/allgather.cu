@@ -11,6 +11,39 @@ namespace {
 constexpr int kAgThreads = 256;   // buffers per CTA (one per thread)
 constexpr int kAgRounds = 64;     // rounds per CTA
 
+// Rows of `table` ([p][q] int8, 16-byte aligned) for the ranks hi, hi-1, ..., hi-n+1 (mod p), brought into shared
+// memory with 16-byte loads (the rows are one contiguous run, or two when the ranks pass 0) and
+// spread round-major: out[k][c] = table[(hi - c) mod p][k].
+__device__ __forceinline__ void stage_rows_descending(const int8_t *__restrict__ table, uint32_t p,
+                                                      int q, uint32_t hi, uint32_t n,
+                                                      uint8_t *rows /* (n * q + 32) bytes */,
+                                                      int8_t (*out)[kAgThreads])
+{
+    const uint32_t first = n <= hi + 1u ? n : hi + 1u;     // columns served by ranks hi-first+1..hi
+    const uint32_t lo = hi + 1u - first;
+    const uint64_t byte_a = (uint64_t)lo * q;
+    const uint32_t shift_a = (uint32_t)(byte_a & 15u);
+    load_span(rows, shift_a, first * (uint32_t)q, table, byte_a);
+    __syncthreads();
+    if (threadIdx.x < first) {
+        const uint8_t *row = rows + shift_a + (first - 1u - threadIdx.x) * q;
+        for (int k = 0; k < q; ++k) out[k][threadIdx.x] = (int8_t)row[k];
+    }
+    __syncthreads();
+    if (first < n) {                                       // the rest: ranks p-1, p-2, ...
+        const uint32_t rest = n - first;
+        const uint64_t byte_b = (uint64_t)(p - rest) * q;
+        const uint32_t shift_b = (uint32_t)(byte_b & 15u);
+        load_span(rows, shift_b, rest * (uint32_t)q, table, byte_b);
+        __syncthreads();
+        if (threadIdx.x >= first && threadIdx.x < n) {
+            const uint8_t *row = rows + shift_b + (n - 1u - threadIdx.x) * q;
+            for (int k = 0; k < q; ++k) out[k][threadIdx.x] = (int8_t)row[k];
+        }
+        __syncthreads();
+    }
+}
+
 __global__ void __launch_bounds__(kAgThreads)
 allgather_kernel(PTable tab, uint32_t n, uint32_t r, const int8_t *__restrict__ recv,
                  const int8_t *__restrict__ send, int32_t *__restrict__ pack_out,
@@ -20,48 +53,53 @@ allgather_kernel(PTable tab, uint32_t n, uint32_t r, const int8_t *__restrict__ 
     // warp read consecutive bytes
     __shared__ int8_t send_k[BCS_MAX_Q][kAgThreads];
     __shared__ int8_t recv_k[BCS_MAX_Q][kAgThreads];
+    __shared__ __align__(16) uint8_t rows[kAgThreads * BCS_MAX_Q + 32];
     const uint32_t p = tab.p;
     const int q = tab.q;
     const uint32_t rounds = n - 1u + (uint32_t)q;
     const int x = (int)(((uint32_t)q - rounds % (uint32_t)q) % (uint32_t)q);
-    const uint32_t j = blockIdx.x * kAgThreads + threadIdx.x;      // buffer
-    const bool valid = j < p;
-    if (valid) {
-        uint32_t v = r + p - j;                                    // (r - j) mod p, j <= p - 1
-        if (v >= p) v -= p;
-        const int8_t *srow = send + (uint64_t)v * q, *rrow = recv + (uint64_t)v * q;
-        for (int k = 0; k < q; ++k) {
-            send_k[k][threadIdx.x] = srow[k];
-            recv_k[k][threadIdx.x] = rrow[k];
-        }
-    }
-    // each thread reads back only what it wrote: no barrier needed
-    if (!valid) return;
+    const uint32_t j0 = blockIdx.x * kAgThreads;                   // first buffer of the CTA
+    const uint32_t cols = p - j0 < (uint32_t)kAgThreads ? p - j0 : (uint32_t)kAgThreads;
+    uint32_t hi = r + p - j0;                                      // (r - j0) mod p: virtual rank of column 0
+    if (hi >= p) hi -= p;
+    if (pack_out) stage_rows_descending(send, p, q, hi, cols, rows, send_k);
+    if (unpack_out) stage_rows_descending(recv, p, q, hi, cols, rows, recv_k);
+    if (threadIdx.x >= cols) return;
+    const uint32_t j = j0 + threadIdx.x;
     const uint32_t jr0 = blockIdx.y * kAgRounds;
     const uint32_t jr1 = jr0 + kAgRounds < rounds ? jr0 + kAgRounds : rounds;
     const int last = (int)n - 1;
-    uint32_t i = jr0 + (uint32_t)x;
-    uint32_t k = i % (uint32_t)q;
-    int base = (int)(i / (uint32_t)q) * q - x;                     // q * floor(i / q) - x
-    int32_t *pk = pack_out ? pack_out + (uint64_t)jr0 * p + j : nullptr;
-    int32_t *up = unpack_out ? unpack_out + (uint64_t)jr0 * p + j : nullptr;
-    for (uint32_t jr = jr0; jr < jr1; ++jr) {
+    const uint32_t i0 = jr0 + (uint32_t)x;
+    uint32_t k = i0 % (uint32_t)q;
+    int base = (int)(i0 / (uint32_t)q) * q - x;                    // q * floor(i / q) - x
+    const uint64_t at = (uint64_t)jr0 * p + j;
+    int32_t *pk = pack_out ? pack_out + at : nullptr;
+    int32_t *up = unpack_out ? unpack_out + at : nullptr;
+    const int8_t *sk = &send_k[0][threadIdx.x], *rk = &recv_k[0][threadIdx.x];
+    uint32_t jr = jr0;
+    while (jr < jr1) {                                             // one phase (or the rest of it) at a time
+        const uint32_t stop = jr1 - jr < (uint32_t)q - k ? jr1 - jr : (uint32_t)q - k;
         if (pk) {
-            int b = (int)send_k[k][threadIdx.x] + base;
-            b = b < 0 ? -1 : (b > last ? last : b);
-            __stcs(pk, b);
-            pk += p;
+#pragma unroll 4
+            for (uint32_t t = 0; t < stop; ++t) {
+                int b = (int)sk[(k + t) * kAgThreads] + base;
+                b = b < 0 ? -1 : (b > last ? last : b);
+                __stcs(pk + (uint64_t)t * p, b);
+            }
+            pk += (uint64_t)stop * p;
         }
         if (up) {
-            int b = (int)recv_k[k][threadIdx.x] + base;
-            b = b < 0 ? -1 : (b > last ? last : b);
-            __stcs(up, b);
-            up += p;
+#pragma unroll 4
+            for (uint32_t t = 0; t < stop; ++t) {
+                int b = (int)rk[(k + t) * kAgThreads] + base;
+                b = b < 0 ? -1 : (b > last ? last : b);
+                __stcs(up + (uint64_t)t * p, b);
+            }
+            up += (uint64_t)stop * p;
         }
-        if (++k == (uint32_t)q) {
-            k = 0;
-            base += q;
-        }
+        jr += stop;
+        k = 0;
+        base += q;
     }
 }
 
@@ -85,7 +123,8 @@ bcs_status bcs_allgather_tables(uint32_t p, uint32_t n, uint32_t r, const int8_t
     if (tab.q == 0) return BCS_OK;
     if (recv == nullptr || send == nullptr || (pack_out == nullptr && unpack_out == nullptr))
         return BCS_ERR_ARG;
-    if ((reinterpret_cast<uintptr_t>(pack_out) & 3u) || (reinterpret_cast<uintptr_t>(unpack_out) & 3u))
+    if ((reinterpret_cast<uintptr_t>(pack_out) & 3u) || (reinterpret_cast<uintptr_t>(unpack_out) & 3u) ||
+        !aligned16(recv) || !aligned16(send))
         return BCS_ERR_ALIGN;
     const uint32_t rounds = n - 1u + (uint32_t)tab.q;
     const uint64_t chunks = ((uint64_t)rounds + kAgRounds - 1) / kAgRounds;

@@ -109,6 +109,25 @@ __device__ __forceinline__ void flush_span(const uint8_t *stage, uint32_t shift,
     }
 }
 
+// Copies in[byte0, byte0+len) to stage[shift, shift+len), (byte0 & 15) == shift, `in` 16-byte
+// aligned: the mirror image of flush_span.
+__device__ __forceinline__ void load_span(uint8_t *stage, uint32_t shift, uint32_t len,
+                                          const int8_t *in, uint64_t byte0)
+{
+    const uint8_t *src = reinterpret_cast<const uint8_t *>(in) + (byte0 - shift);
+    const uint32_t end = shift + len;
+    const uint32_t nvec = (end + 15u) >> 4;
+    for (uint32_t v = threadIdx.x; v < nvec; v += blockDim.x) {
+        const uint32_t lo = v << 4, hi = lo + 16u;
+        if (lo >= shift && hi <= end) {
+            *reinterpret_cast<uint4 *>(stage + lo) = *reinterpret_cast<const uint4 *>(src + lo);
+        } else {
+            const uint32_t from = lo < shift ? shift : lo, to = hi > end ? end : hi;
+            for (uint32_t e = from; e < to; ++e) stage[e] = src[e];
+        }
+    }
+}
+
 // Largest j with off[j] <= g, searched in [lo, hi].
 __device__ __forceinline__ uint32_t find_segment(const uint64_t *off, uint32_t lo, uint32_t hi,
                                                  uint64_t g)
