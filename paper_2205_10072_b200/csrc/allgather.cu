@@ -64,42 +64,50 @@ allgather_kernel(PTable tab, uint32_t n, uint32_t r, const int8_t *__restrict__ 
     if (hi >= p) hi -= p;
     if (pack_out) stage_rows_descending(send, p, q, hi, cols, rows, send_k);
     if (unpack_out) stage_rows_descending(recv, p, q, hi, cols, rows, recv_k);
-    if (threadIdx.x >= cols) return;
-    const uint32_t j = j0 + threadIdx.x;
+    // Four rows at a time: thread t works on row jr + t / 64 and on four consecutive buffers, chosen
+    // per row and table so that its 16 bytes are 16-byte aligned in the output (rows are p * 4 bytes
+    // long, so the alignment of a row's start changes from row to row); the up to three buffers
+    // before the first and after the last aligned group of the CTA's 256 are written one by one.
     const uint32_t jr0 = blockIdx.y * kAgRounds;
     const uint32_t jr1 = jr0 + kAgRounds < rounds ? jr0 + kAgRounds : rounds;
     const int last = (int)n - 1;
-    const uint32_t i0 = jr0 + (uint32_t)x;
-    uint32_t k = i0 % (uint32_t)q;
-    int base = (int)(i0 / (uint32_t)q) * q - x;                    // q * floor(i / q) - x
-    const uint64_t at = (uint64_t)jr0 * p + j;
-    int32_t *pk = pack_out ? pack_out + at : nullptr;
-    int32_t *up = unpack_out ? unpack_out + at : nullptr;
-    const int8_t *sk = &send_k[0][threadIdx.x], *rk = &recv_k[0][threadIdx.x];
-    uint32_t jr = jr0;
-    while (jr < jr1) {                                             // one phase (or the rest of it) at a time
-        const uint32_t stop = jr1 - jr < (uint32_t)q - k ? jr1 - jr : (uint32_t)q - k;
-        if (pk) {
-#pragma unroll 4
-            for (uint32_t t = 0; t < stop; ++t) {
-                int b = (int)sk[(k + t) * kAgThreads] + base;
-                b = b < 0 ? -1 : (b > last ? last : b);
-                __stcs(pk + (uint64_t)t * p, b);
+    const uint32_t sub = threadIdx.x >> 6, grp = threadIdx.x & 63u;
+    for (uint32_t jr = jr0 + sub; jr < jr1; jr += 4) {
+        const uint32_t i = jr + (uint32_t)x;
+        const uint32_t k = i % (uint32_t)q;
+        const int base = (int)(i / (uint32_t)q) * q - x;           // q * floor(i / q) - x
+        const uint64_t at = (uint64_t)jr * p + j0;                 // element index of the CTA's first buffer
+#pragma unroll
+        for (int which = 0; which < 2; ++which) {
+            int32_t *out = which == 0 ? pack_out : unpack_out;
+            if (out == nullptr) continue;
+            const int8_t *src = which == 0 ? send_k[k] : recv_k[k];
+            // buffers before the first 16-byte boundary of this row's piece of this table
+            uint32_t head = (uint32_t)((16u - (uint32_t)(reinterpret_cast<uintptr_t>(out + at) & 15u)) & 15u) >> 2;
+            if (head > cols) head = cols;
+            const uint32_t c = head + 4u * grp;                    // first of this thread's four buffers
+            if (c + 4u <= cols) {
+                int4 v;
+                v.x = (int)src[c] + base;
+                v.y = (int)src[c + 1] + base;
+                v.z = (int)src[c + 2] + base;
+                v.w = (int)src[c + 3] + base;
+                v.x = v.x < 0 ? -1 : (v.x > last ? last : v.x);
+                v.y = v.y < 0 ? -1 : (v.y > last ? last : v.y);
+                v.z = v.z < 0 ? -1 : (v.z > last ? last : v.z);
+                v.w = v.w < 0 ? -1 : (v.w > last ? last : v.w);
+                __stcs(reinterpret_cast<int4 *>(out + at + c), v);
+            } else {
+                for (uint32_t e = c; e < cols; ++e) {              // ragged end of the CTA's columns
+                    int b = (int)src[e] + base;
+                    out[at + e] = b < 0 ? -1 : (b > last ? last : b);
+                }
             }
-            pk += (uint64_t)stop * p;
-        }
-        if (up) {
-#pragma unroll 4
-            for (uint32_t t = 0; t < stop; ++t) {
-                int b = (int)rk[(k + t) * kAgThreads] + base;
-                b = b < 0 ? -1 : (b > last ? last : b);
-                __stcs(up + (uint64_t)t * p, b);
+            if (grp < head) {                                      // ragged start
+                int b = (int)src[grp] + base;
+                out[at + grp] = b < 0 ? -1 : (b > last ? last : b);
             }
-            up += (uint64_t)stop * p;
         }
-        jr += stop;
-        k = 0;
-        base += q;
     }
 }
 
