@@ -1,16 +1,21 @@
 // Receive and send schedules (arXiv 2205.10072, Algorithms 2-5 and the lookup of Algorithm 9):
-// kernels and the entry points bcs_build, bcs_build_to_host, bcs_build_batch.
+// kernels and the entry points bcs_build, bcs_build_static, bcs_build_to_host, bcs_prepare,
+// bcs_build_prepared, bcs_build_batch.
 //
 // Two constructions, bit-identical in their results:
 //
-//  * workspace path (three kernels).  codes_kernel writes the skip code (bcs_common.cuh) of every
-//    rank x of a p once.  recv_codes_kernel then reads, per rank r and round i, the codes of the
-//    two ranks that bound the window of Algorithm 4 (r - skips[i+1], r - skips[i]; consecutive
-//    threads read consecutive words) and finds the largest new block of the window from the two
-//    codes alone: walking down from the first level where they differ, every step yields one
-//    "head" (a rank whose baseblock is that level) and a run of low blocks.  It writes the rows
-//    rank-major and a round-major copy from which send_rm_kernel reads
-//    sendsched[r][k] = recvsched[(r+skips[k]) mod p][k] with unit stride.
+//  * workspace path.  codes_kernel writes the skip code (bcs_common.cuh) of every rank x of a p
+//    once.  The receive kernels (recv_codes_warp_kernel for one p >= 64, recv_codes_batch_kernel
+//    for a batch, recv_codes_kernel for tiny p) then read, per rank r and round i, the codes of
+//    the two ranks that bound the window of Algorithm 4 (r - skips[i+1], r - skips[i];
+//    consecutive threads read consecutive words) and find the largest new block of the window
+//    from the two codes alone: walking down from the first level where they differ, every step
+//    yields one "head" (a rank whose baseblock is that level) and a run of low blocks; the rounds
+//    whose windows reach at most 32 ranks back are done by the whole warp with shuffles.  They
+//    write the rows rank-major and a round-major copy, from which send_transpose_kernel /
+//    send_batch_kernel produce sendsched[r][k] = recvsched[(r+skips[k]) mod p][k] as a
+//    transposition with row k rotated by skips[k] (send_rm_kernel: sub-ranges, byte gathers and
+//    recomputation for to-processors outside the range).
 //
 //  * self-contained path (no workspace).  One thread per rank runs Algorithm 4 with the range
 //    search done by descending the homeranges; the send schedule is looked up in the rank-major
