@@ -447,7 +447,7 @@ def run_ours(args) -> None:
 
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of the
 # current kernels); None until counters have been taken for the kernel as it stands.
-RECV_TRAFFIC_BYTES = 4212224 + 185088        # recv_codes_warp_kernel<true,true>, p = 2^20+1
+RECV_TRAFFIC_BYTES = 4218368 + 713728        # recv_codes_warp_kernel<true,true>, p = 2^20+1
 EXPAND_TRAFFIC_BYTES = 1567312000 + 3457280   # expand_kernel, p = 100003, n = 1000
 
 # integer operations per rank of the receive-schedule construction that the kernels run, by q:

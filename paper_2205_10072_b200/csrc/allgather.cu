@@ -51,8 +51,8 @@ allgather_kernel(PTable tab, uint32_t n, uint32_t r, const int8_t *__restrict__ 
 {
     // schedule entries of this CTA's 256 virtual processors, round-major so that the threads of a
     // warp read consecutive bytes
-    __shared__ int8_t send_k[BCS_MAX_Q][kAgThreads];
-    __shared__ int8_t recv_k[BCS_MAX_Q][kAgThreads];
+    __shared__ __align__(16) int8_t send_k[BCS_MAX_Q][kAgThreads];
+    __shared__ __align__(16) int8_t recv_k[BCS_MAX_Q][kAgThreads];
     __shared__ __align__(16) uint8_t rows[kAgThreads * BCS_MAX_Q + 32];
     const uint32_t p = tab.p;
     const int q = tab.q;
@@ -64,34 +64,47 @@ allgather_kernel(PTable tab, uint32_t n, uint32_t r, const int8_t *__restrict__ 
     if (hi >= p) hi -= p;
     if (pack_out) stage_rows_descending(send, p, q, hi, cols, rows, send_k);
     if (unpack_out) stage_rows_descending(recv, p, q, hi, cols, rows, recv_k);
-    // Four rows at a time: thread t works on row jr + t / 64 and on four consecutive buffers, chosen
-    // per row and table so that its 16 bytes are 16-byte aligned in the output (rows are p * 4 bytes
-    // long, so the alignment of a row's start changes from row to row); the up to three buffers
-    // before the first and after the last aligned group of the CTA's 256 are written one by one.
+    // Four rows at a time: thread t works on rows jr0 + t / 64, +4, +8, ... and on four consecutive
+    // buffers, chosen so that its 16 bytes are 16-byte aligned in the output.  Rows are p * 4 bytes
+    // long, so the alignment of a row's start differs from row to row -- but four rows on it is
+    // the same again (16 p bytes), so each thread finds its alignment once per table.  The up to
+    // three buffers before the first and after the last aligned group of the CTA's 256 are
+    // written one by one.
     const uint32_t jr0 = blockIdx.y * kAgRounds;
     const uint32_t jr1 = jr0 + kAgRounds < rounds ? jr0 + kAgRounds : rounds;
     const int last = (int)n - 1;
     const uint32_t sub = threadIdx.x >> 6, grp = threadIdx.x & 63u;
-    for (uint32_t jr = jr0 + sub; jr < jr1; jr += 4) {
-        const uint32_t i = jr + (uint32_t)x;
-        const uint32_t k = i % (uint32_t)q;
-        const int base = (int)(i / (uint32_t)q) * q - x;           // q * floor(i / q) - x
-        const uint64_t at = (uint64_t)jr * p + j0;                 // element index of the CTA's first buffer
+    uint32_t jr = jr0 + sub;
+    if (jr >= jr1) return;
+    const uint32_t i0 = jr + (uint32_t)x;
+    uint32_t k = i0 % (uint32_t)q;
+    int base = (int)(i0 / (uint32_t)q) * q - x;                    // q * floor(i / q) - x
+    uint64_t at = (uint64_t)jr * p + j0;                           // element index of the CTA's first buffer
+    uint32_t head[2] = {0, 0};                                     // buffers before the first 16-byte boundary
+    int32_t *const outs[2] = {pack_out, unpack_out};
+#pragma unroll
+    for (int which = 0; which < 2; ++which) {
+        if (outs[which] == nullptr) continue;
+        uint32_t hd = (uint32_t)((16u - (uint32_t)(reinterpret_cast<uintptr_t>(outs[which] + at) & 15u)) & 15u) >> 2;
+        head[which] = hd > cols ? cols : hd;
+    }
+    for (; jr < jr1; jr += 4) {
 #pragma unroll
         for (int which = 0; which < 2; ++which) {
-            int32_t *out = which == 0 ? pack_out : unpack_out;
+            int32_t *out = outs[which];
             if (out == nullptr) continue;
             const int8_t *src = which == 0 ? send_k[k] : recv_k[k];
-            // buffers before the first 16-byte boundary of this row's piece of this table
-            uint32_t head = (uint32_t)((16u - (uint32_t)(reinterpret_cast<uintptr_t>(out + at) & 15u)) & 15u) >> 2;
-            if (head > cols) head = cols;
-            const uint32_t c = head + 4u * grp;                    // first of this thread's four buffers
+            const uint32_t c = head[which] + 4u * grp;             // first of this thread's four buffers
             if (c + 4u <= cols) {
+                // four consecutive bytes from two aligned words
+                const uint32_t *words = reinterpret_cast<const uint32_t *>(src) + (c >> 2);
+                const uint32_t lo = words[0], hi = (c & 3u) ? words[1] : 0u;
+                const uint32_t four = __funnelshift_r(lo, hi, (c & 3u) * 8u);
                 int4 v;
-                v.x = (int)src[c] + base;
-                v.y = (int)src[c + 1] + base;
-                v.z = (int)src[c + 2] + base;
-                v.w = (int)src[c + 3] + base;
+                v.x = (int)(int8_t)(four & 0xffu) + base;
+                v.y = (int)(int8_t)((four >> 8) & 0xffu) + base;
+                v.z = (int)(int8_t)((four >> 16) & 0xffu) + base;
+                v.w = (int)(int8_t)(four >> 24) + base;
                 v.x = v.x < 0 ? -1 : (v.x > last ? last : v.x);
                 v.y = v.y < 0 ? -1 : (v.y > last ? last : v.y);
                 v.z = v.z < 0 ? -1 : (v.z > last ? last : v.z);
@@ -103,10 +116,16 @@ allgather_kernel(PTable tab, uint32_t n, uint32_t r, const int8_t *__restrict__ 
                     out[at + e] = b < 0 ? -1 : (b > last ? last : b);
                 }
             }
-            if (grp < head) {                                      // ragged start
+            if (grp < head[which]) {                               // ragged start
                 int b = (int)src[grp] + base;
                 out[at + grp] = b < 0 ? -1 : (b > last ? last : b);
             }
+        }
+        at += 4ull * p;
+        k += 4;
+        while (k >= (uint32_t)q) {
+            k -= (uint32_t)q;
+            base += q;
         }
     }
 }
