@@ -4,7 +4,7 @@
 //
 // Two constructions, bit-identical in their results:
 //
-//  * workspace path.  codes_kernel writes the skip code (bcs_common.cuh) of every rank x of a p
+//  * workspace path.  codes_single_kernel / codes_batch_kernel write the skip code (bcs_common.cuh) of every rank x of a p
 //    once.  The receive kernels (recv_codes_warp_kernel for one p >= 64, recv_codes_batch_kernel
 //    for a batch, recv_codes_kernel for tiny p) then read, per rank r and round i, the codes of
 //    the two ranks that bound the window of Algorithm 4 (r - skips[i+1], r - skips[i];
@@ -181,29 +181,53 @@ send_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, BatchArgs ba,
 }
 
 // ================================================================ workspace path
-// Skip code of every rank: codes[g] for the flattened rank g (single p: g = x).  For a single
-// p the scan over the levels is unrolled, so every skip is an immediate operand from the
-// kernel parameters; levels at and above q never match (a rank is below skips[q] = p).
-template <bool kBatch>
+// Skip code of every rank of one p: codes[x].  The scan over the levels is unrolled for the q at
+// hand (one instantiation per q), so every skip is an immediate operand from the kernel
+// parameters and no level is tested in vain.
+template <int kQ>
 __global__ void __launch_bounds__(kTile)
-codes_kernel(PTable tab, BatchArgs ba, uint32_t *__restrict__ codes)
+codes_single_kernel(const __grid_constant__ PTable tab, uint32_t *__restrict__ codes)
 {
-    if (!kBatch) {
-        const uint64_t g = (uint64_t)blockIdx.x * kTile + threadIdx.x;
-        if (g >= tab.p) return;
-        uint32_t x = (uint32_t)g, code = 0;
+    const uint64_t g = (uint64_t)blockIdx.x * kTile + threadIdx.x;
+    if (g >= tab.p) return;
+    uint32_t x = (uint32_t)g, code = 0;
 #pragma unroll
-        for (int k = BCS_MAX_Q - 1; k >= 0; --k) {
-            if (k < tab.q && x >= tab.s[k]) {
-                x -= tab.s[k];
-                code |= 1u << k;
-            }
+    for (int k = kQ - 1; k >= 0; --k) {
+        if (x >= tab.s[k]) {
+            x -= tab.s[k];
+            code |= 1u << k;
         }
-        codes[g] = code;
-        return;
     }
+    codes[g] = code;
+}
+
+template <int kQ>
+struct CodesLauncher {
+    static void launch(int q, const PTable &tab, uint32_t *codes, unsigned blocks, cudaStream_t stream)
+    {
+        if (q == kQ)
+            codes_single_kernel<kQ><<<blocks, kTile, 0, stream>>>(tab, codes);
+        else
+            CodesLauncher<kQ - 1>::launch(q, tab, codes, blocks, stream);
+    }
+};
+template <>
+struct CodesLauncher<0> {
+    static void launch(int, const PTable &, uint32_t *, unsigned, cudaStream_t) {}
+};
+
+inline void launch_codes(const PTable &tab, uint32_t *codes, cudaStream_t stream)
+{
+    CodesLauncher<BCS_MAX_Q>::launch(tab.q, tab, codes, (unsigned)((tab.p + kTile - 1) / kTile), stream);
+}
+
+// Batch: codes[g] for the flattened rank g.
+__global__ void __launch_bounds__(kTile)
+codes_batch_kernel(BatchArgs ba, uint32_t *__restrict__ codes)
+{
     __shared__ TileShared sh;
-    RankCtx c = resolve_rank<kBatch>(sh, tab, 0, tab.p, ba);
+    PTable unused;
+    RankCtx c = resolve_rank<true>(sh, unused, 0, 0, ba);
     if (c.valid) codes[c.rank0 + c.r] = skip_code(c.s, c.q, c.r);
 }
 
@@ -810,8 +834,7 @@ bcs_status bcs_build(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_
         ws.codes = static_cast<uint32_t *>(workspace);
         ws.recv_t = static_cast<int8_t *>(workspace) + align_up(4ull * p, 256);
         ws.t_stride = align_up(count, 16);
-        codes_kernel<false><<<(unsigned)((p + kTile - 1) / kTile), kTile, 0, stream>>>(tab, none,
-                                                                                      ws.codes);
+        launch_codes(tab, ws.codes, stream);
         if ((st = launch_status()) != BCS_OK) return st;
         const bool warp_rounds = p >= 64;      // the warp-cooperative kernel needs 32 ranks back
         if (recv_out != nullptr && send_out != nullptr) {
@@ -882,7 +905,7 @@ bcs_status bcs_prepare(uint32_t p, void *workspace, size_t workspace_bytes, void
     const uint64_t t_stride = align_up(p, 16);
     const unsigned blocks = (unsigned)((p + kTile - 1) / kTile);
     BatchArgs none = {};
-    codes_kernel<false><<<blocks, kTile, 0, stream>>>(tab, none, codes);
+    launch_codes(tab, codes, stream);
     if ((st = launch_status()) != BCS_OK) return st;
     if (p >= 64)
         recv_codes_warp_kernel<false, true><<<blocks, kTile, 0, stream>>>(tab, 0, p, codes, nullptr,
@@ -988,7 +1011,7 @@ bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_
         workspace_bytes >= bcs_build_batch_workspace_bytes(total_ranks, total_entries)) {
         uint32_t *codes = static_cast<uint32_t *>(workspace);
         int8_t *recv_t = static_cast<int8_t *>(workspace) + align_up(4ull * total_ranks, 256);
-        codes_kernel<true><<<blocks, kTile, 0, stream>>>(none, ba, codes);
+        codes_batch_kernel<<<blocks, kTile, 0, stream>>>(ba, codes);
         if ((st = launch_status()) != BCS_OK) return st;
         if (send_out != nullptr)
             recv_codes_batch_kernel<true><<<blocks, kTile, 0, stream>>>(ba, codes, recv_out, recv_t);
