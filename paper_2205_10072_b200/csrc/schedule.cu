@@ -679,12 +679,14 @@ struct TransposeShared {
 // tbl: round 0 of the round-major table of this p (all p ranks per row, rows `stride` bytes
 // apart, any alignment; up to 15 bytes before a row's first and after its last needed byte are
 // read as well).  The tile is ranks r0..r0+n-1; stage: where its rank-major rows start.
-template <class Skips>
-__device__ __forceinline__ void transpose_tile(const Skips skip, uint32_t p, int q,
+// kQ: q known at compile time (loops over the rounds unrolled), 0 = use the argument.
+template <int kQ, class Skips>
+__device__ __forceinline__ void transpose_tile(const Skips skip, uint32_t p, int q_arg,
                                                const int8_t *__restrict__ tbl, uint64_t stride,
                                                uint32_t r0, uint32_t n, bool rotate,
                                                TransposeShared &ts, uint8_t *stage)
 {
+    const int q = kQ ? kQ : q_arg;
     if (threadIdx.x == 0) ts.wraps = 0;
     __syncthreads();
     const int vecs = kTrPitch / 16;         // 18 vectors cover 256 bytes at any misalignment
@@ -723,13 +725,19 @@ __device__ __forceinline__ void transpose_tile(const Skips skip, uint32_t p, int
         uint8_t *__restrict__ row = stage + mine * q;
         const uint8_t *__restrict__ column = ts.rounds + mine;
         const uint32_t *__restrict__ lead_k = ts.lead;
+        if (kQ) {
+#pragma unroll
+            for (int k = 0; k < (kQ ? kQ : 1); ++k) row[k] = column[k * kTrPitch + lead_k[k]];
+        } else {
 #pragma unroll 4
-        for (int k = 0; k < q; ++k) row[k] = column[k * kTrPitch + lead_k[k]];
+            for (int k = 0; k < q; ++k) row[k] = column[k * kTrPitch + lead_k[k]];
+        }
     }
 }
 
 // Single p: recv_t holds all p ranks of every round; the CTA's tile is ranks r0..r0+n-1 of the
 // range r_begin..r_begin+count-1.  rotate: send rows; otherwise the receive rows themselves.
+template <int kQ>
 __global__ void __launch_bounds__(kTile)
 send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restrict__ recv_t,
                       uint64_t t_stride, int8_t *send_out, uint32_t r_begin, uint32_t count,
@@ -739,10 +747,35 @@ send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restri
     __shared__ __align__(16) uint8_t stage[kTile * 32];
     const uint32_t first = blockIdx.x * kTile;
     const uint32_t n = count - first < (uint32_t)kTile ? count - first : (uint32_t)kTile;
-    transpose_tile(ParamSkips{tab}, tab.p, tab.q, recv_t, t_stride, r_begin + first, n, rotate, ts,
-                   stage);
+    transpose_tile<kQ>(ParamSkips{tab}, tab.p, tab.q, recv_t, t_stride, r_begin + first, n, rotate,
+                       ts, stage);
     __syncthreads();
     flush_span(stage, 0, n * (uint32_t)tab.q, send_out, (uint64_t)first * (uint64_t)tab.q);
+}
+
+template <int kQ>
+struct TransposeLauncher {
+    static void launch(const PTable &tab, const int8_t *recv_t, uint64_t t_stride, int8_t *out,
+                       uint32_t r_begin, uint32_t count, bool rotate, cudaStream_t stream)
+    {
+        if (tab.q == kQ)
+            send_transpose_kernel<kQ><<<(count + kTile - 1) / kTile, kTile, 0, stream>>>(
+                tab, recv_t, t_stride, out, r_begin, count, rotate);
+        else
+            TransposeLauncher<kQ - 1>::launch(tab, recv_t, t_stride, out, r_begin, count, rotate,
+                                              stream);
+    }
+};
+template <>
+struct TransposeLauncher<0> {
+    static void launch(const PTable &, const int8_t *, uint64_t, int8_t *, uint32_t, uint32_t, bool,
+                       cudaStream_t) {}
+};
+
+inline void launch_transpose(const PTable &tab, const int8_t *recv_t, uint64_t t_stride, int8_t *out,
+                             uint32_t r_begin, uint32_t count, bool rotate, cudaStream_t stream)
+{
+    TransposeLauncher<BCS_MAX_Q>::launch(tab, recv_t, t_stride, out, r_begin, count, rotate, stream);
 }
 
 // Batch: a CTA inside one p transposes; a CTA that straddles several p gathers byte by byte.
@@ -759,7 +792,7 @@ send_batch_kernel(BatchArgs ba, const int8_t *__restrict__ recv_t, int8_t *send_
         const uint32_t n = (uint32_t)(ba.total_ranks - g0 < (uint64_t)kTile ? ba.total_ranks - g0
                                                                              : (uint64_t)kTile);
         if (c.q > 0)
-            transpose_tile(SharedSkips{sh.skips[0]}, c.p, c.q, recv_t + ba.entry_off[c.pj],
+            transpose_tile<0>(SharedSkips{sh.skips[0]}, c.p, c.q, recv_t + ba.entry_off[c.pj],
                            (uint64_t)c.p, (uint32_t)(g0 - c.rank0), n, true, ts, sh.stage + shift);
     } else if (c.valid) {
         uint8_t *row = sh.stage + shift + (c.entry - sh.span_begin);
@@ -862,8 +895,7 @@ bcs_status bcs_build(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_
         if ((st = launch_status()) != BCS_OK) return st;
         if (send_out != nullptr) {
             if (count == p)
-                send_transpose_kernel<<<blocks, kTile, 0, stream>>>(tab, ws.recv_t, ws.t_stride,
-                                                                    send_out, 0u, p, true);
+                launch_transpose(tab, ws.recv_t, ws.t_stride, send_out, 0u, p, true, stream);
             else
                 send_rm_kernel<false, false><<<blocks, kTile, 0, stream>>>(
                     tab, r_begin, r_end, none, ws.codes, ws.recv_t, ws.t_stride, send_out);
@@ -932,15 +964,14 @@ bcs_status bcs_build_prepared(uint32_t p, uint64_t r_begin, uint64_t r_end, int8
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int8_t *recv_t = static_cast<const int8_t *>(workspace) + align_up(4ull * p, 256);
     const uint64_t t_stride = align_up(p, 16);
-    const unsigned blocks = (unsigned)((count + kTile - 1) / kTile);
     if (recv_out != nullptr) {
-        send_transpose_kernel<<<blocks, kTile, 0, stream>>>(tab, recv_t, t_stride, recv_out,
-                                                            (uint32_t)r_begin, (uint32_t)count, false);
+        launch_transpose(tab, recv_t, t_stride, recv_out, (uint32_t)r_begin, (uint32_t)count, false,
+                         stream);
         if ((st = launch_status()) != BCS_OK) return st;
     }
     if (send_out != nullptr) {
-        send_transpose_kernel<<<blocks, kTile, 0, stream>>>(tab, recv_t, t_stride, send_out,
-                                                            (uint32_t)r_begin, (uint32_t)count, true);
+        launch_transpose(tab, recv_t, t_stride, send_out, (uint32_t)r_begin, (uint32_t)count, true,
+                         stream);
         if ((st = launch_status()) != BCS_OK) return st;
     }
     return BCS_OK;
