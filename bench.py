@@ -25,9 +25,8 @@ if ROOT not in sys.path:
 METRIC = "schedule ranks built/sec (int8 recv+send, q entries)"
 UNIT = "ranks/s"
 
-# Integer work the receive schedule of one rank needs in the construction that is timed
-# (descent steps of the range search, measured by a CPU count of the same loop structure, times
-# the integer operations of one step) -- see DESIGN.md, "Roofline".
+# Peak of the integer pipes that the schedule kernels are measured against: INT32 lanes per SM per
+# clock x number of SMs x SM clock.
 ALU_LANES_PER_SM = 64          # INT32 lanes per SM per clock
 SM_COUNT = 148
 

@@ -218,14 +218,25 @@ def test_degenerate_sizes_and_errors(bcs):
 
 def test_p_at_the_upper_limit(bcs):
     """p = 2^31 - 1 (q = 31): rank arithmetic near 2^32; a few ranges vs the per-rank oracle.
-    (Self-contained construction: the workspace of this p would be 8.6 GB; the skip-code
-    construction at large q is covered by the chunked p = 2^30 - 1 test.)"""
+    Both constructions."""
     p = 2**31 - 1
     for r0, r1 in ((0, 300), (2**30 - 100, 2**30 + 200), (p - 300, p)):
         want_r, want_s = oracle.build_range(p, r0, r1)
         recv, send = _build(bcs, p, r0, r1, fast=False)
         assert np.array_equal(recv, want_r), (r0, r1)
         assert np.array_equal(send, want_s), (r0, r1)
+    # the skip-code construction at the same p: 8.6 GB of codes in the workspace
+    for r0, r1 in ((0, 300), (2**30 - 100, 2**30 + 200), (p - 300, p)):
+        want_r, want_s = oracle.build_range(p, r0, r1)
+        q = 31
+        recv = torch.empty((r1 - r0) * q, dtype=torch.int8, device="cuda")
+        send = torch.empty((r1 - r0) * q, dtype=torch.int8, device="cuda")
+        ws = torch.empty(bcs.bcs_build_workspace_bytes(p, r0, r1), dtype=torch.int8, device="cuda")
+        bcs.bcs_build(p, r0, r1, recv, send, ws)
+        torch.cuda.synchronize()
+        assert np.array_equal(recv.cpu().numpy().reshape(-1, q), want_r), (r0, r1)
+        assert np.array_equal(send.cpu().numpy().reshape(-1, q), want_s), (r0, r1)
+        del ws
 
 
 # ---------------------------------------------------------------- full-size workloads
