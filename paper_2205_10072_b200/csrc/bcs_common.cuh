@@ -109,6 +109,27 @@ __device__ __forceinline__ void flush_span(const uint8_t *stage, uint32_t shift,
     }
 }
 
+// The same for a span that starts 16-byte aligned in shared and global memory and is a multiple
+// of 16 bytes long, as one bulk copy of the TMA unit (cp.async.bulk, shared -> global) issued by
+// one thread.  Call with all threads of the CTA, after the rows have been written and INSTEAD of
+// the barrier that precedes flush_span: every thread makes its shared-memory writes visible to
+// the asynchronous proxy, the CTA synchronises, thread 0 issues the copy and waits until the
+// unit has read the staging buffer (the global writes complete on their own).
+__device__ __forceinline__ void flush_span_bulk(const uint8_t *stage, uint32_t len, int8_t *out,
+                                                uint64_t byte0)
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x == 0 && len != 0) {
+        const uint32_t src = (uint32_t)__cvta_generic_to_shared(stage);
+        const uint64_t dst = reinterpret_cast<uint64_t>(out) + byte0;
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                     :: "l"(dst), "r"(src), "r"(len) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+    }
+}
+
 // Copies in[byte0, byte0+len) to stage[shift, shift+len), (byte0 & 15) == shift, `in` 16-byte
 // aligned: the mirror image of flush_span.
 __device__ __forceinline__ void load_span(uint8_t *stage, uint32_t shift, uint32_t len,

@@ -574,8 +574,13 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uin
                                      stage, kColOut ? recv_t + g0 + threadIdx.x : nullptr,
                                      t_stride);
     if (kRowOut) {
-        __syncthreads();
-        flush_span(stage, 0, n * (uint32_t)tab.q, recv_out, g0 * (uint64_t)tab.q);
+        const uint32_t len = n * (uint32_t)tab.q;          // the tile's rows start at byte g0 * q: 16-byte aligned
+        if ((len & 15u) == 0) {
+            flush_span_bulk(stage, len, recv_out, g0 * (uint64_t)tab.q);
+        } else {                                           // ragged last tile
+            __syncthreads();
+            flush_span(stage, 0, len, recv_out, g0 * (uint64_t)tab.q);
+        }
     }
 }
 
@@ -749,8 +754,13 @@ send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restri
     const uint32_t n = count - first < (uint32_t)kTile ? count - first : (uint32_t)kTile;
     transpose_tile<kQ>(ParamSkips{tab}, tab.p, tab.q, recv_t, t_stride, r_begin + first, n, rotate,
                        ts, stage);
-    __syncthreads();
-    flush_span(stage, 0, n * (uint32_t)tab.q, send_out, (uint64_t)first * (uint64_t)tab.q);
+    const uint32_t len = n * (uint32_t)tab.q;              // starts at byte first * q: 16-byte aligned
+    if ((len & 15u) == 0) {
+        flush_span_bulk(stage, len, send_out, (uint64_t)first * (uint64_t)tab.q);
+    } else {                                               // ragged last tile
+        __syncthreads();
+        flush_span(stage, 0, len, send_out, (uint64_t)first * (uint64_t)tab.q);
+    }
 }
 
 template <int kQ>
