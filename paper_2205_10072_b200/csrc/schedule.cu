@@ -359,32 +359,26 @@ __device__ __forceinline__ int recv_rounds_codes(const uint32_t *__restrict__ co
     return entry;
 }
 
-// recv_t: round-major copy.  Single p: recv_t[k * t_stride + (r - r_begin)].
-// Batch: recv_t[entry_off[j] + k * p_j + r].
-template <bool kBatch, bool kRowOut, bool kColOut>
+// One p, every round searched per lane (used for p < 64, where a warp's 32 predecessors would
+// wrap around the ring more than once).  recv_t: round-major copy, recv_t[k * t_stride + (r - r_begin)].
+template <bool kRowOut, bool kColOut>
 __global__ void __launch_bounds__(kTile)
-recv_codes_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, BatchArgs ba,
+recv_codes_kernel(PTable tab, uint64_t r_begin, uint64_t r_end,
                   const uint32_t *__restrict__ codes, int8_t *recv_out, int8_t *recv_t,
                   uint64_t t_stride)
 {
     __shared__ TileShared sh;
-    RankCtx c = resolve_rank<kBatch>(sh, tab, r_begin, r_end, ba);
-    const uint32_t shift = (uint32_t)(sh.span_begin & 15u);
+    BatchArgs none = {};
+    RankCtx c = resolve_rank<false>(sh, tab, r_begin, r_end, none);
     if (c.valid && c.q > 0) {
-        int8_t *col = nullptr;
-        uint64_t stride = 0;
-        if (kColOut) {
-            col = kBatch ? recv_t + ba.entry_off[c.pj] + c.r : recv_t + (c.r - r_begin);
-            stride = kBatch ? (uint64_t)c.p : t_stride;
-        }
-        uint8_t *row = kRowOut ? sh.stage + shift + (c.entry - sh.span_begin) : nullptr;
-        recv_rounds_codes<kRowOut, kColOut>(codes + c.rank0, c.s, c.full, c.p, c.q, c.r, c.q - 1,
-                                            row, col, stride);
+        int8_t *col = kColOut ? recv_t + (c.r - r_begin) : nullptr;
+        uint8_t *row = kRowOut ? sh.stage + (c.entry - sh.span_begin) : nullptr;
+        recv_rounds_codes<kRowOut, kColOut>(codes, c.s, c.full, c.p, c.q, c.r, c.q - 1, row, col,
+                                            t_stride);
     }
     if (kRowOut) {
         __syncthreads();
-        flush_span(sh.stage, shift, (uint32_t)(sh.span_end - sh.span_begin), recv_out,
-                   sh.span_begin);
+        flush_span(sh.stage, 0, (uint32_t)(sh.span_end - sh.span_begin), recv_out, sh.span_begin);
     }
 }
 
@@ -615,56 +609,36 @@ recv_codes_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t
     flush_span(sh.stage, shift, (uint32_t)(sh.span_end - sh.span_begin), recv_out, sh.span_begin);
 }
 
-// Send rows from the round-major receive copy.  kAllInside: every to-processor's row is in
-// the copy (all ranks of the p).  Otherwise (single p, sub-range) to-processors outside the
-// range are recomputed from the codes (Algorithm 5).
-template <bool kBatch, bool kAllInside>
+// Send rows of a sub-range of one p from the round-major receive copy of that range;
+// to-processors outside the range are recomputed from the codes (Algorithm 5).
 __global__ void __launch_bounds__(kTile)
-send_rm_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, BatchArgs ba,
-               const uint32_t *__restrict__ codes, const int8_t *__restrict__ recv_t,
-               uint64_t t_stride, int8_t *send_out)
+send_rm_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, const uint32_t *__restrict__ codes,
+               const int8_t *__restrict__ recv_t, uint64_t t_stride, int8_t *send_out)
 {
     __shared__ TileShared sh;
-    RankCtx c = resolve_rank<kBatch>(sh, tab, r_begin, r_end, ba);
-    const uint32_t shift = (uint32_t)(sh.span_begin & 15u);
+    BatchArgs none = {};
+    RankCtx c = resolve_rank<false>(sh, tab, r_begin, r_end, none);
     if (c.valid) {
-        uint8_t *row = sh.stage + shift + (c.entry - sh.span_begin);
-        const int8_t *tbl = kBatch ? recv_t + ba.entry_off[c.pj] : recv_t;
-        const uint64_t stride = kBatch ? (uint64_t)c.p : t_stride;
-        if (kAllInside) {
-            for (int k0 = 0; k0 < c.q; k0 += 8) {
-                int v[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int k = k0 + j < c.q ? k0 + j : c.q - 1;
-                    uint32_t t = c.r + c.s[k];
-                    if (t >= c.p) t -= c.p;
-                    v[j] = tbl[(uint64_t)k * stride + t];
-                }
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if (k0 + j < c.q) row[k0 + j] = (uint8_t)v[j];
+        uint8_t *row = sh.stage + (c.entry - sh.span_begin);
+        const int8_t *tbl = recv_t;
+        const uint32_t first = (uint32_t)r_begin, width = (uint32_t)(r_end - r_begin);
+        for (int k = 0; k < c.q; ++k) {
+            uint32_t t = c.r + c.s[k];
+            if (t >= c.p) t -= c.p;
+            const uint32_t rel = t - first;          // index into the round-major row
+            int v;
+            if (rel < width) {
+                v = tbl[rel];
+            } else {
+                v = recv_rounds_codes<false, false>(codes, c.s, c.full, c.p, c.q, t, k, nullptr,
+                                                    nullptr, 0);
             }
-        } else {
-            const uint32_t first = (uint32_t)r_begin, width = (uint32_t)(r_end - r_begin);
-            for (int k = 0; k < c.q; ++k) {
-                uint32_t t = c.r + c.s[k];
-                if (t >= c.p) t -= c.p;
-                const uint32_t rel = t - first;          // index into the round-major row
-                int v;
-                if (rel < width) {
-                    v = tbl[rel];
-                } else {
-                    v = recv_rounds_codes<false, false>(codes, c.s, c.full, c.p, c.q, t, k, nullptr,
-                                                        nullptr, 0);
-                }
-                row[k] = (uint8_t)v;
-                tbl += stride;
-            }
+            row[k] = (uint8_t)v;
+            tbl += t_stride;
         }
     }
     __syncthreads();
-    flush_span(sh.stage, shift, (uint32_t)(sh.span_end - sh.span_begin), send_out, sh.span_begin);
+    flush_span(sh.stage, 0, (uint32_t)(sh.span_end - sh.span_begin), send_out, sh.span_begin);
 }
 
 // Row k of the round-major send table is row k of the round-major receive copy rotated by
@@ -885,30 +859,30 @@ bcs_status bcs_build(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_
                 recv_codes_warp_kernel<true, true><<<blocks, kTile, 0, stream>>>(
                     tab, r_begin, r_end, ws.codes, recv_out, ws.recv_t, ws.t_stride);
             else
-                recv_codes_kernel<false, true, true><<<blocks, kTile, 0, stream>>>(
-                    tab, r_begin, r_end, none, ws.codes, recv_out, ws.recv_t, ws.t_stride);
+                recv_codes_kernel<true, true><<<blocks, kTile, 0, stream>>>(
+                    tab, r_begin, r_end, ws.codes, recv_out, ws.recv_t, ws.t_stride);
         } else if (recv_out != nullptr) {
             if (warp_rounds)
                 recv_codes_warp_kernel<true, false><<<blocks, kTile, 0, stream>>>(
                     tab, r_begin, r_end, ws.codes, recv_out, nullptr, 0);
             else
-                recv_codes_kernel<false, true, false><<<blocks, kTile, 0, stream>>>(
-                    tab, r_begin, r_end, none, ws.codes, recv_out, nullptr, 0);
+                recv_codes_kernel<true, false><<<blocks, kTile, 0, stream>>>(
+                    tab, r_begin, r_end, ws.codes, recv_out, nullptr, 0);
         } else {
             if (warp_rounds)
                 recv_codes_warp_kernel<false, true><<<blocks, kTile, 0, stream>>>(
                     tab, r_begin, r_end, ws.codes, nullptr, ws.recv_t, ws.t_stride);
             else
-                recv_codes_kernel<false, false, true><<<blocks, kTile, 0, stream>>>(
-                    tab, r_begin, r_end, none, ws.codes, nullptr, ws.recv_t, ws.t_stride);
+                recv_codes_kernel<false, true><<<blocks, kTile, 0, stream>>>(
+                    tab, r_begin, r_end, ws.codes, nullptr, ws.recv_t, ws.t_stride);
         }
         if ((st = launch_status()) != BCS_OK) return st;
         if (send_out != nullptr) {
             if (count == p)
                 launch_transpose(tab, ws.recv_t, ws.t_stride, send_out, 0u, p, true, stream);
             else
-                send_rm_kernel<false, false><<<blocks, kTile, 0, stream>>>(
-                    tab, r_begin, r_end, none, ws.codes, ws.recv_t, ws.t_stride, send_out);
+                send_rm_kernel<<<blocks, kTile, 0, stream>>>(tab, r_begin, r_end, ws.codes,
+                                                             ws.recv_t, ws.t_stride, send_out);
             if ((st = launch_status()) != BCS_OK) return st;
         }
         return BCS_OK;
@@ -946,15 +920,14 @@ bcs_status bcs_prepare(uint32_t p, void *workspace, size_t workspace_bytes, void
     int8_t *recv_t = static_cast<int8_t *>(workspace) + align_up(4ull * p, 256);
     const uint64_t t_stride = align_up(p, 16);
     const unsigned blocks = (unsigned)((p + kTile - 1) / kTile);
-    BatchArgs none = {};
     launch_codes(tab, codes, stream);
     if ((st = launch_status()) != BCS_OK) return st;
     if (p >= 64)
         recv_codes_warp_kernel<false, true><<<blocks, kTile, 0, stream>>>(tab, 0, p, codes, nullptr,
                                                                           recv_t, t_stride);
     else
-        recv_codes_kernel<false, false, true><<<blocks, kTile, 0, stream>>>(
-            tab, 0, p, none, codes, nullptr, recv_t, t_stride);
+        recv_codes_kernel<false, true><<<blocks, kTile, 0, stream>>>(tab, 0, p, codes, nullptr,
+                                                                     recv_t, t_stride);
     return launch_status();
 }
 
