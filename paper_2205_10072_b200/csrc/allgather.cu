@@ -13,7 +13,7 @@ constexpr int kAgRounds = 64;     // rounds per CTA
 
 // Rows of `table` ([p][q] int8, 16-byte aligned) for the ranks hi, hi-1, ..., hi-n+1 (mod p), brought into shared
 // memory with 16-byte loads (the rows are one contiguous run, or two when the ranks pass 0) and
-// spread round-major: out[k][c] = table[(hi - c) mod p][k].
+// spread round-major and made non-negative: out[k][c] = table[(hi - c) mod p][k] + 2q (< 128).
 __device__ __forceinline__ void stage_rows_descending(const int8_t *__restrict__ table, uint32_t p,
                                                       int q, uint32_t hi, uint32_t n,
                                                       uint8_t *rows /* (n * q + 32) bytes */,
@@ -27,7 +27,7 @@ __device__ __forceinline__ void stage_rows_descending(const int8_t *__restrict__
     __syncthreads();
     if (threadIdx.x < first) {
         const uint8_t *row = rows + shift_a + (first - 1u - threadIdx.x) * q;
-        for (int k = 0; k < q; ++k) out[k][threadIdx.x] = (int8_t)row[k];
+        for (int k = 0; k < q; ++k) out[k][threadIdx.x] = (int8_t)((int8_t)row[k] + 2 * q);
     }
     __syncthreads();
     if (first < n) {                                       // the rest: ranks p-1, p-2, ...
@@ -38,7 +38,7 @@ __device__ __forceinline__ void stage_rows_descending(const int8_t *__restrict__
         __syncthreads();
         if (threadIdx.x >= first && threadIdx.x < n) {
             const uint8_t *row = rows + shift_b + (n - 1u - threadIdx.x) * q;
-            for (int k = 0; k < q; ++k) out[k][threadIdx.x] = (int8_t)row[k];
+            for (int k = 0; k < q; ++k) out[k][threadIdx.x] = (int8_t)((int8_t)row[k] + 2 * q);
         }
         __syncthreads();
     }
@@ -78,7 +78,7 @@ allgather_kernel(PTable tab, uint32_t n, uint32_t r, const int8_t *__restrict__ 
     if (jr >= jr1) return;
     const uint32_t i0 = jr + (uint32_t)x;
     uint32_t k = i0 % (uint32_t)q;
-    int base = (int)(i0 / (uint32_t)q) * q - x;                    // q * floor(i / q) - x
+    int base = (int)(i0 / (uint32_t)q) * q - x - 2 * q;            // q * floor(i / q) - x, minus the staging offset
     uint64_t at = (uint64_t)jr * p + j0;                           // element index of the CTA's first buffer
     uint32_t head[2] = {0, 0};                                     // buffers before the first 16-byte boundary
     int32_t *const outs[2] = {pack_out, unpack_out};
@@ -100,24 +100,21 @@ allgather_kernel(PTable tab, uint32_t n, uint32_t r, const int8_t *__restrict__ 
                 const uint32_t *words = reinterpret_cast<const uint32_t *>(src) + (c >> 2);
                 const uint32_t lo = words[0], hi = (c & 3u) ? words[1] : 0u;
                 const uint32_t four = __funnelshift_r(lo, hi, (c & 3u) * 8u);
+                // the staged bytes are entries + 2q (unsigned); below 0 -> -1, above n-1 -> n-1
                 int4 v;
-                v.x = (int)(int8_t)(four & 0xffu) + base;
-                v.y = (int)(int8_t)((four >> 8) & 0xffu) + base;
-                v.z = (int)(int8_t)((four >> 16) & 0xffu) + base;
-                v.w = (int)(int8_t)(four >> 24) + base;
-                v.x = v.x < 0 ? -1 : (v.x > last ? last : v.x);
-                v.y = v.y < 0 ? -1 : (v.y > last ? last : v.y);
-                v.z = v.z < 0 ? -1 : (v.z > last ? last : v.z);
-                v.w = v.w < 0 ? -1 : (v.w > last ? last : v.w);
+                v.x = max(min((int)__byte_perm(four, 0u, 0x4440u) + base, last), -1);
+                v.y = max(min((int)__byte_perm(four, 0u, 0x4441u) + base, last), -1);
+                v.z = max(min((int)__byte_perm(four, 0u, 0x4442u) + base, last), -1);
+                v.w = max(min((int)__byte_perm(four, 0u, 0x4443u) + base, last), -1);
                 __stcs(reinterpret_cast<int4 *>(out + at + c), v);
             } else {
                 for (uint32_t e = c; e < cols; ++e) {              // ragged end of the CTA's columns
-                    int b = (int)src[e] + base;
+                    const int b = (int)(uint8_t)src[e] + base;
                     out[at + e] = b < 0 ? -1 : (b > last ? last : b);
                 }
             }
             if (grp < head[which]) {                               // ragged start
-                int b = (int)src[grp] + base;
+                const int b = (int)(uint8_t)src[grp] + base;
                 out[at + grp] = b < 0 ? -1 : (b > last ? last : b);
             }
         }
