@@ -244,6 +244,14 @@ bcs_status bcs_validate(uint32_t p, uint64_t r_begin, uint64_t r_end,
 bcs_status bcs_simulate(uint32_t p, uint32_t n, const int8_t *recv, const int8_t *send,
                         uint64_t *state_dev, uint64_t *counts_dev, void *cuda_stream);
 
+/* Bounded waits (no counterpart in the paper).  The transposition kernel of bcs_build and
+ * bcs_build_prepared waits for its bulk copies on a shared-memory barrier with a poll limit; a
+ * CTA whose copies did not arrive within the limit leaves its 256 ranks of the output unwritten
+ * and counts itself in a device-wide counter that is never reset.  This call synchronises the
+ * device and stores the counter of the current device in *count_host (host): 0 means that
+ * every output written so far is complete. */
+bcs_status bcs_wait_expired(uint64_t *count_host);
+
 /* Position-weighted 64-bit checksum of a stretch of schedule entries, additive
  * over disjoint stretches (no counterpart in the paper; used to compare outputs
  * that are too large to copy back).  The bytes are read as little-endian 32-bit

@@ -22,12 +22,14 @@ from .binding import (  # noqa: F401
     bcs_circulant_rounds,
     bcs_expand,
     bcs_prepare,
+    bcs_probe_int_rate,
     bcs_prepare_workspace_bytes,
     bcs_q,
     bcs_simulate,
     bcs_skips,
     bcs_status_str,
     bcs_validate,
+    bcs_wait_expired,
     lib,
     lib_path,
 )

@@ -74,6 +74,11 @@ def lib():
         L.bcs_allgather_tables.restype = i32
         L.bcs_simulate.argtypes = [u32, u32, vp, vp, vp, vp, vp]
         L.bcs_simulate.restype = i32
+        L.bcs_probe_int_rate.argtypes = [i32, u32, vp, _c.POINTER(_c.c_double),
+                                         _c.POINTER(_c.c_float), vp]
+        L.bcs_probe_int_rate.restype = i32
+        L.bcs_wait_expired.argtypes = [_c.POINTER(u64)]
+        L.bcs_wait_expired.restype = i32
         L.bcs_checksum.argtypes = [vp, u64, u64, vp, vp]
         L.bcs_checksum.restype = i32
         _lib = L
@@ -256,6 +261,24 @@ def bcs_simulate(p: int, n: int, recv, send, state, counts_out, stream=None) -> 
     counts_out: CUDA int64 tensor of five elements (see include/bcs.h)."""
     _check(lib().bcs_simulate(p, n, _ptr(recv), _ptr(send), _ptr(state), _ptr(counts_out),
                               _stream(stream)), "bcs_simulate")
+
+
+def bcs_wait_expired() -> int:
+    """CTAs of the transposition kernel that gave up waiting for their copies (0 = none)."""
+    v = _c.c_uint64(0)
+    _check(lib().bcs_wait_expired(_c.byref(v)), "bcs_wait_expired")
+    return v.value
+
+
+def bcs_probe_int_rate(mix: int, iters: int = 4096, stream=None) -> float:
+    """Measured thread-level integer instructions per second of the current device
+    (mix 0: logic only; 1: logic and multiply-add alternating; 2: logic and addition
+    alternating).  Benchmark helper."""
+    sink = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ops, ms = _c.c_double(0), _c.c_float(0)
+    _check(lib().bcs_probe_int_rate(mix, iters, sink.data_ptr(), _c.byref(ops), _c.byref(ms),
+                                    _stream(stream)), "bcs_probe_int_rate")
+    return ops.value / (ms.value * 1e-3)
 
 
 def bcs_checksum(buf, first_entry_index: int, sum_out, stream=None, n_entries: int | None = None) -> None:

@@ -714,26 +714,112 @@ __device__ __forceinline__ void transpose_tile(const Skips skip, uint32_t p, int
     }
 }
 
-// Single p: recv_t holds all p ranks of every round; the CTA's tile is ranks r0..r0+n-1 of the
-// range r_begin..r_begin+count-1.  rotate: send rows; otherwise the receive rows themselves.
+// Single p, the same transposition on the copy unit and in registers.  recv_t holds all p ranks
+// of every round; the CTA's tile is ranks r0..r0+n-1 of the range r_begin..r_begin+count-1.
+// rotate: send rows; otherwise the receive rows themselves.
+//   * Thread k < q brings the (rotated) bytes of round k into shared memory with one bulk copy
+//     (cp.async.bulk global -> shared, completion counted on an mbarrier); the copy starts at the
+//     16-byte boundary at or before the first needed byte and ends at the one at or after the
+//     last.  A round whose bytes pass the end of the row (at most q tiles of a table) gets the
+//     part after the wrap by plain loads.
+//   * Thread j then takes the four ranks 4j..4j+3: one 32-bit word per round (two aligned words
+//     and a funnel shift, as the rotation puts the tile anywhere in the word), and its 4q output
+//     bytes -- q aligned words of the rank-major rows, since 4q bytes start at a multiple of 4 --
+//     are put together by byte permutations with selectors known at compile time.  Shared memory
+//     sees 3 word accesses per four entries instead of 8 byte accesses.
+//   * The rows leave as one bulk store.
+// 64 threads per 256 ranks; the many small CTAs per SM overlap one another's copies.
+constexpr int kTrThreads = kTile / 4;
+constexpr uint32_t kWaitLimit = 1u << 22;   // polls of the mbarrier before a CTA gives up
+
+// CTAs whose bulk load did not complete within kWaitLimit polls (they leave their tile unwritten).
+__device__ unsigned long long g_wait_expired;
+
 template <int kQ>
-__global__ void __launch_bounds__(kTile)
+__global__ void __launch_bounds__(kTrThreads)
 send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restrict__ recv_t,
                       uint64_t t_stride, int8_t *send_out, uint32_t r_begin, uint32_t count,
                       bool rotate)
 {
-    __shared__ TransposeShared ts;
-    __shared__ __align__(16) uint8_t stage[kTile * 32];
+    __shared__ __align__(128) uint8_t rounds[kQ * kTrPitch];
+    __shared__ __align__(16) uint8_t stage[kTile * kQ];
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ uint32_t lead[kQ];            // offset of the tile's first byte inside its pitch row
+    __shared__ uint32_t wraps;               // rounds whose bytes pass the end of the row
+    const uint32_t p = tab.p;
     const uint32_t first = blockIdx.x * kTile;
     const uint32_t n = count - first < (uint32_t)kTile ? count - first : (uint32_t)kTile;
-    transpose_tile<kQ>(ParamSkips{tab}, tab.p, tab.q, recv_t, t_stride, r_begin + first, n, rotate,
-                       ts, stage);
-    const uint32_t len = n * (uint32_t)tab.q;              // starts at byte first * q: 16-byte aligned
+    const uint32_t r0 = r_begin + first;
+    const uint32_t bar_addr = (uint32_t)__cvta_generic_to_shared(&bar);
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar_addr), "r"(kQ) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        wraps = 0;
+    }
+    __syncthreads();
+    if (threadIdx.x < kQ) {
+        const int k = threadIdx.x;
+        uint32_t start = r0 + (rotate ? tab.s[k] : 0u);
+        if (start >= p) start -= p;
+        const uint32_t mis = start & 15u;                      // rows start 16-byte aligned
+        const uint32_t run = p - start < n ? p - start : n;    // bytes before the wrap
+        const uint32_t bytes = (mis + run + 15u) & ~15u;       // <= 272, inside the row's pitch
+        lead[k] = mis;
+        if (run < n) atomicOr(&wraps, 1u << k);
+        const uint64_t src = reinterpret_cast<uint64_t>(recv_t) + (uint64_t)k * t_stride + (start - mis);
+        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(rounds + k * kTrPitch);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                     :: "r"(bar_addr), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     :: "r"(dst), "l"(src), "r"(bytes), "r"(bar_addr) : "memory");
+    }
+    uint32_t done = 0;
+    for (uint32_t poll = 0; poll < kWaitLimit && !done; ++poll)
+        asm volatile("{\n\t.reg .pred ok;\n\t"
+                     "mbarrier.try_wait.parity.shared::cta.b64 ok, [%1], 0;\n\t"
+                     "selp.u32 %0, 1, 0, ok;\n\t}"
+                     : "=r"(done) : "r"(bar_addr) : "memory");
+    if (__syncthreads_or(!done)) {                             // uniform: nobody touches the tile
+        if (threadIdx.x == 0) atomicAdd(&g_wait_expired, 1ull);
+        return;
+    }
+    if (wraps) {                                               // the part after the wrap, by bytes
+        for (uint32_t left = wraps; left != 0; left &= left - 1u) {
+            const int k = __ffs(left) - 1;
+            uint32_t start = r0 + (rotate ? tab.s[k] : 0u);
+            if (start >= p) start -= p;
+            const uint32_t run = p - start;                    // < n for these rounds
+            const uint8_t *src_row = reinterpret_cast<const uint8_t *>(recv_t) + (uint64_t)k * t_stride;
+            for (uint32_t j = run + threadIdx.x; j < n; j += kTrThreads)
+                rounds[k * kTrPitch + lead[k] + j] = src_row[j - run];
+        }
+        __syncthreads();
+    }
+    // W[k]: the entries of round k of this thread's four ranks
+    uint32_t W[kQ];
+#pragma unroll
+    for (int k = 0; k < kQ; ++k) {
+        const uint32_t off = (uint32_t)k * kTrPitch + lead[k] + 4u * threadIdx.x;
+        const uint32_t *word = reinterpret_cast<const uint32_t *>(rounds + (off & ~3u));
+        W[k] = __funnelshift_r(word[0], word[1], (off & 3u) * 8u);
+    }
+    // output word m holds bytes 4m..4m+3 of the four rows: byte e is rank e / q, round e % q
+    uint32_t *rows = reinterpret_cast<uint32_t *>(stage) + threadIdx.x * kQ;
+#pragma unroll
+    for (int m = 0; m < kQ; ++m) {
+        const int e = 4 * m;
+        const uint32_t lo = __byte_perm(W[e % kQ], W[(e + 1) % kQ],
+                                        (uint32_t)(e / kQ) | (uint32_t)(4 + (e + 1) / kQ) << 4);
+        const uint32_t hi = __byte_perm(W[(e + 2) % kQ], W[(e + 3) % kQ],
+                                        (uint32_t)((e + 2) / kQ) | (uint32_t)(4 + (e + 3) / kQ) << 4);
+        rows[m] = __byte_perm(lo, hi, 0x5410u);
+    }
+    const uint32_t len = n * (uint32_t)kQ;                 // starts at byte first * q: 16-byte aligned
     if ((len & 15u) == 0) {
-        flush_span_bulk(stage, len, send_out, (uint64_t)first * (uint64_t)tab.q);
+        flush_span_bulk(stage, len, send_out, (uint64_t)first * (uint64_t)kQ);
     } else {                                               // ragged last tile
         __syncthreads();
-        flush_span(stage, 0, len, send_out, (uint64_t)first * (uint64_t)tab.q);
+        flush_span(stage, 0, len, send_out, (uint64_t)first * (uint64_t)kQ);
     }
 }
 
@@ -743,7 +829,7 @@ struct TransposeLauncher {
                        uint32_t r_begin, uint32_t count, bool rotate, cudaStream_t stream)
     {
         if (tab.q == kQ)
-            send_transpose_kernel<kQ><<<(count + kTile - 1) / kTile, kTile, 0, stream>>>(
+            send_transpose_kernel<kQ><<<(count + kTile - 1) / kTile, kTrThreads, 0, stream>>>(
                 tab, recv_t, t_stride, out, r_begin, count, rotate);
         else
             TransposeLauncher<kQ - 1>::launch(tab, recv_t, t_stride, out, r_begin, count, rotate,
@@ -1049,6 +1135,15 @@ bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_
 
 // Device address of g_static_scratch on the current device, looked up once per device (with that
 // device current) and remembered; nullptr if the runtime refuses.
+bcs_status bcs_wait_expired(uint64_t *count_host)
+{
+    if (count_host == nullptr) return BCS_ERR_ARG;
+    unsigned long long v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_wait_expired, sizeof(v)) != cudaSuccess) return BCS_ERR_CUDA;
+    *count_host = v;
+    return BCS_OK;
+}
+
 static void *static_scratch_address()
 {
     constexpr int kMaxDevices = 64;

@@ -46,6 +46,7 @@ def _build(bcs, p, r0, r1, want_recv=True, want_send=True, fast=True):
         raw_w, ws = _guarded(need)
     bcs.bcs_build(p, r0, r1, recv, send, ws)
     torch.cuda.synchronize()
+    assert bcs.bcs_wait_expired() == 0      # no CTA gave up waiting for its copies
     if raw_w is not None:
         assert _guards_intact(raw_w, ws.numel())
     out = []
@@ -513,6 +514,7 @@ def test_large_p_full_broadcast_simulation(bcs):
     bcs.bcs_simulate(p, n, recv, send, state, counts)
     got = counts.cpu().tolist()
     assert got[:4] == [0, 0, 0, 0] and 1 <= got[4] < p, got
+    assert bcs.bcs_wait_expired() == 0
     del recv, send, state
     torch.cuda.empty_cache()
 
