@@ -252,8 +252,43 @@ __device__ __forceinline__ RankCtx resolve_rank(TileShared &sh, const PTable &ta
     return c;
 }
 
+// ---------------------------------------------------------------- dependent launches
+// The kernels of one construction run back to back on one stream, each a few tens of
+// microseconds long, so the time in which one grid drains and the next is brought onto the SMs
+// counts.  A kernel launched with launch_dependent() may be made resident as soon as every CTA
+// of the kernel before it on the stream has called grid_launch_dependents() (or has exited); it
+// runs its set-up and then blocks in grid_dependency_wait() until that kernel has completed and
+// its writes are visible.  Both calls do nothing in a kernel that was launched the ordinary way.
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+__device__ __forceinline__ void grid_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ---------------------------------------------------------------- host helpers
 bcs_status make_table(uint32_t p, PTable *tab);
+
+// Launch with programmatic stream serialisation (see above); `dependent` false: ordinary launch.
+template <class... Params, class... Args>
+inline void launch_dependent(bool dependent, void (*kernel)(Params...), unsigned grid, unsigned block,
+                             cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, Params(args)...);
+}
 
 inline bool aligned16(const void *ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
 

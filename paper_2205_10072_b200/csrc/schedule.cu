@@ -188,6 +188,7 @@ template <int kQ>
 __global__ void __launch_bounds__(kTile)
 codes_single_kernel(const __grid_constant__ PTable tab, uint32_t *__restrict__ codes)
 {
+    grid_launch_dependents();
     const uint64_t g = (uint64_t)blockIdx.x * kTile + threadIdx.x;
     if (g >= tab.p) return;
     uint32_t x = (uint32_t)g, code = 0;
@@ -559,11 +560,13 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uin
 {
     __shared__ __align__(16) uint8_t stage[kTile * 32];
     __shared__ uint32_t full_sh[kRow];
+    grid_launch_dependents();
     if (threadIdx.x < kRow) full_sh[threadIdx.x] = tab.full[threadIdx.x];
     __syncthreads();
     const uint64_t count = r_end - r_begin;
     const uint64_t g0 = (uint64_t)blockIdx.x * kTile;
     const uint32_t n = (uint32_t)(count - g0 < (uint64_t)kTile ? count - g0 : (uint64_t)kTile);
+    grid_dependency_wait();                                // the codes are complete from here on
     recv_warp_tile<kRowOut, kColOut>(ParamSkips{tab}, full_sh, tab.p, tab.q, r_begin + g0, n, codes,
                                      stage, kColOut ? recv_t + g0 + threadIdx.x : nullptr,
                                      t_stride);
@@ -756,7 +759,9 @@ send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restri
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         wraps = 0;
     }
+    grid_launch_dependents();
     __syncthreads();
+    grid_dependency_wait();                                    // the round-major copy is complete
     if (threadIdx.x < kQ) {
         const int k = threadIdx.x;
         uint32_t start = r0 + (rotate ? tab.s[k] : 0u);
@@ -826,26 +831,30 @@ send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restri
 template <int kQ>
 struct TransposeLauncher {
     static void launch(const PTable &tab, const int8_t *recv_t, uint64_t t_stride, int8_t *out,
-                       uint32_t r_begin, uint32_t count, bool rotate, cudaStream_t stream)
+                       uint32_t r_begin, uint32_t count, bool rotate, bool dependent,
+                       cudaStream_t stream)
     {
         if (tab.q == kQ)
-            send_transpose_kernel<kQ><<<(count + kTile - 1) / kTile, kTrThreads, 0, stream>>>(
-                tab, recv_t, t_stride, out, r_begin, count, rotate);
+            launch_dependent(dependent, send_transpose_kernel<kQ>, (count + kTile - 1) / kTile,
+                             kTrThreads, stream, tab, recv_t, t_stride, out, r_begin, count, rotate);
         else
             TransposeLauncher<kQ - 1>::launch(tab, recv_t, t_stride, out, r_begin, count, rotate,
-                                              stream);
+                                              dependent, stream);
     }
 };
 template <>
 struct TransposeLauncher<0> {
     static void launch(const PTable &, const int8_t *, uint64_t, int8_t *, uint32_t, uint32_t, bool,
-                       cudaStream_t) {}
+                       bool, cudaStream_t) {}
 };
 
+// dependent: the kernel before this one on the stream calls grid_launch_dependents().
 inline void launch_transpose(const PTable &tab, const int8_t *recv_t, uint64_t t_stride, int8_t *out,
-                             uint32_t r_begin, uint32_t count, bool rotate, cudaStream_t stream)
+                             uint32_t r_begin, uint32_t count, bool rotate, bool dependent,
+                             cudaStream_t stream)
 {
-    TransposeLauncher<BCS_MAX_Q>::launch(tab, recv_t, t_stride, out, r_begin, count, rotate, stream);
+    TransposeLauncher<BCS_MAX_Q>::launch(tab, recv_t, t_stride, out, r_begin, count, rotate,
+                                         dependent, stream);
 }
 
 // Batch: a CTA inside one p transposes; a CTA that straddles several p gathers byte by byte.
@@ -942,22 +951,22 @@ bcs_status bcs_build(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_
         const bool warp_rounds = p >= 64;      // the warp-cooperative kernel needs 32 ranks back
         if (recv_out != nullptr && send_out != nullptr) {
             if (warp_rounds)
-                recv_codes_warp_kernel<true, true><<<blocks, kTile, 0, stream>>>(
-                    tab, r_begin, r_end, ws.codes, recv_out, ws.recv_t, ws.t_stride);
+                launch_dependent(true, recv_codes_warp_kernel<true, true>, blocks, kTile, stream, tab,
+                                 r_begin, r_end, ws.codes, recv_out, ws.recv_t, ws.t_stride);
             else
                 recv_codes_kernel<true, true><<<blocks, kTile, 0, stream>>>(
                     tab, r_begin, r_end, ws.codes, recv_out, ws.recv_t, ws.t_stride);
         } else if (recv_out != nullptr) {
             if (warp_rounds)
-                recv_codes_warp_kernel<true, false><<<blocks, kTile, 0, stream>>>(
-                    tab, r_begin, r_end, ws.codes, recv_out, nullptr, 0);
+                launch_dependent(true, recv_codes_warp_kernel<true, false>, blocks, kTile, stream, tab,
+                                 r_begin, r_end, ws.codes, recv_out, nullptr, 0);
             else
                 recv_codes_kernel<true, false><<<blocks, kTile, 0, stream>>>(
                     tab, r_begin, r_end, ws.codes, recv_out, nullptr, 0);
         } else {
             if (warp_rounds)
-                recv_codes_warp_kernel<false, true><<<blocks, kTile, 0, stream>>>(
-                    tab, r_begin, r_end, ws.codes, nullptr, ws.recv_t, ws.t_stride);
+                launch_dependent(true, recv_codes_warp_kernel<false, true>, blocks, kTile, stream, tab,
+                                 r_begin, r_end, ws.codes, nullptr, ws.recv_t, ws.t_stride);
             else
                 recv_codes_kernel<false, true><<<blocks, kTile, 0, stream>>>(
                     tab, r_begin, r_end, ws.codes, nullptr, ws.recv_t, ws.t_stride);
@@ -965,7 +974,8 @@ bcs_status bcs_build(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_
         if ((st = launch_status()) != BCS_OK) return st;
         if (send_out != nullptr) {
             if (count == p)
-                launch_transpose(tab, ws.recv_t, ws.t_stride, send_out, 0u, p, true, stream);
+                launch_transpose(tab, ws.recv_t, ws.t_stride, send_out, 0u, p, true, warp_rounds,
+                                 stream);
             else
                 send_rm_kernel<<<blocks, kTile, 0, stream>>>(tab, r_begin, r_end, ws.codes,
                                                              ws.recv_t, ws.t_stride, send_out);
@@ -1009,8 +1019,8 @@ bcs_status bcs_prepare(uint32_t p, void *workspace, size_t workspace_bytes, void
     launch_codes(tab, codes, stream);
     if ((st = launch_status()) != BCS_OK) return st;
     if (p >= 64)
-        recv_codes_warp_kernel<false, true><<<blocks, kTile, 0, stream>>>(tab, 0, p, codes, nullptr,
-                                                                          recv_t, t_stride);
+        launch_dependent(true, recv_codes_warp_kernel<false, true>, blocks, kTile, stream, tab,
+                         (uint64_t)0, (uint64_t)p, codes, nullptr, recv_t, t_stride);
     else
         recv_codes_kernel<false, true><<<blocks, kTile, 0, stream>>>(tab, 0, p, codes, nullptr,
                                                                      recv_t, t_stride);
@@ -1035,12 +1045,12 @@ bcs_status bcs_build_prepared(uint32_t p, uint64_t r_begin, uint64_t r_end, int8
     const uint64_t t_stride = align_up(p, 16);
     if (recv_out != nullptr) {
         launch_transpose(tab, recv_t, t_stride, recv_out, (uint32_t)r_begin, (uint32_t)count, false,
-                         stream);
+                         false, stream);
         if ((st = launch_status()) != BCS_OK) return st;
     }
     if (send_out != nullptr) {
         launch_transpose(tab, recv_t, t_stride, send_out, (uint32_t)r_begin, (uint32_t)count, true,
-                         stream);
+                         recv_out != nullptr, stream);
         if ((st = launch_status()) != BCS_OK) return st;
     }
     return BCS_OK;
