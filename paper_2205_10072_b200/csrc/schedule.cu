@@ -383,14 +383,18 @@ recv_codes_kernel(PTable tab, uint64_t r_begin, uint64_t r_end,
     }
 }
 
-// Single p, p >= 64: the same rows with the first rounds done by the whole warp.  A warp holds 32
-// consecutive ranks, and the windows of the rounds with skips[i+1] <= 33 reach at most 32
-// ranks back, so every baseblock they can contain is the lowest code bit of a rank held by
-// this warp's lanes (rank r of each lane) or by the 32 ranks before them (one more load per
-// lane): the window sets of those rounds -- and of their second windows while
-// sum_{j<=i} skips[j] <= 32 -- are OR-ed together from warp shuffles, one per distance, the
-// same for all lanes.  These are the rounds in which neighbouring ranks disagree about which
-// path of the code search they take; the later rounds run the code search per lane.
+// Single p, p >= 64: the same rows with the first rounds decided from a table of the tile.  The
+// windows of the rounds with skips[i+1] <= 33 (at most six rounds, i <= 5) reach only a few
+// ranks back: the first window ends skips[i+1] - 1 ranks below r, the second at
+// sum_{j<=i} skips[j] <= skips[i+1] + i <= 38 (every halving rounds up by at most one), and a run
+// of the table adds at most 3 more to the second and none beyond skips[i+1] - 1 to the first.  So
+// every baseblock those windows can contain is the lowest code bit of one of the tile's ranks or
+// of the 64 ranks before the tile.  The tile keeps, for x = every one of those 320 ranks and
+// j = 0..4, the baseblock bits OR-ed over the 2^j ranks that end at x (doubling, one barrier
+// per level); a window of L ranks is the union of two such runs of 2^floor(log2 L) ranks: two
+// shared-memory words per window, whatever its length.  These are the rounds in which
+// neighbouring ranks disagree about which path of the code search they take; the later rounds
+// run the code search per lane.
 // Where the skips of the tile's p are read from: the kernel parameter (single p: immediate /
 // constant-bank operands) or a table row in shared memory (batch).
 struct ParamSkips {
@@ -402,28 +406,66 @@ struct SharedSkips {
     __device__ __forceinline__ uint32_t operator()(int k) const { return s[k]; }
 };
 
+constexpr int kRunBack = 64;                   // ranks before the tile that the run table covers
+constexpr int kRunLevels = 5;                  // runs of 1, 2, 4, 8, 16 ranks
+constexpr int kRunPitch = kTile + kRunBack;    // words per level
+struct RunTable {
+    uint32_t bits[kRunLevels][kRunPitch];
+    // Round i of the table rounds reads the four words at these byte offsets from a thread's own
+    // level-0 entry: .x | .y is its first window, .z | .w its second (a repeat of the first when
+    // the round has no second window).
+    int4 window[8];
+    uint32_t len2[kRow];     // length of the second window of round i: sum_{j<=i} skips[j] - skips[i+1] + 1, or 0
+};
+
 // The tile is the n ranks first..first+n-1 of a p (n <= 256, one per thread); `stage` is where
 // the tile's rank-major rows start in shared memory, `col` this thread's element of round 0 in
-// the round-major copy.  All 256 threads must call (the warp rounds use every lane).
+// the round-major copy.  All 256 threads must call (the table is built by all of them).
 template <bool kRowOut, bool kColOut, class Skips>
 __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t *full_sh,
                                                uint32_t p, int q, uint64_t first, uint32_t n,
                                                const uint32_t *__restrict__ codes, uint8_t *stage,
-                                               int8_t *col, uint64_t t_stride)
+                                               int8_t *col, uint64_t t_stride, RunTable &runs)
 {
-    constexpr unsigned kAll = 0xffffffffu;
     const bool valid = threadIdx.x < n;
-    const uint32_t lane = threadIdx.x & 31u;
-    // ranks of this lane and of the lane 32 ranks before it, mod p (defined for every lane of the
-    // warp, also past the end of the range: only lower lanes and `before` are read by others)
+    // rank of this thread mod p (defined for every thread, also past the end of the range: the
+    // table entries of such ranks are never read by a valid thread)
     uint64_t wrapped = first + threadIdx.x;
     while (wrapped >= p) wrapped -= p;
     const uint32_t r = (uint32_t)wrapped;
-    const uint32_t r_before = r >= 32u ? r - 32u : r + p - 32u;
     const uint32_t own = codes[r];
-    const uint32_t before = codes[r_before];
     const uint32_t own_bit = own & (0u - own);            // baseblock of r as a bit, 0 for the root
-    const uint32_t before_bit = before & (0u - before);
+    runs.bits[0][kRunBack + threadIdx.x] = own_bit;
+    if (threadIdx.x < kRunBack) {                         // the 64 ranks before the tile, mod p (p >= 64)
+        uint64_t back = first + threadIdx.x + p - kRunBack;
+        while (back >= p) back -= p;
+        const uint32_t c = codes[(uint32_t)back];
+        runs.bits[0][threadIdx.x] = c & (0u - c);
+    }
+    if (threadIdx.x < (uint32_t)q) {                      // per-round constants of this p
+        const int i = threadIdx.x;
+        uint32_t sum = 0;
+        for (int j = 0; j <= i; ++j) sum += skip(j);
+        const uint32_t lo = skip(i), hi = skip(i + 1);
+        const uint32_t len2 = sum >= hi ? sum - hi + 1u : 0u;
+        runs.len2[i] = len2;
+        if (hi <= 33u) {
+            // the len >= 1 ranks that end d ranks below: runs of 2^j ranks, j = floor(log2 len),
+            // ending d and d + len - 2^j ranks below
+            const int j1 = 31 - __clz(hi - lo);
+            int4 w;
+            w.x = 4 * (j1 * kRunPitch - (int)lo);
+            w.y = 4 * (j1 * kRunPitch - (int)(hi - (1u << j1)));
+            w.z = w.x;
+            w.w = w.y;
+            if (len2) {
+                const int j2 = 31 - __clz(len2);
+                w.z = 4 * (j2 * kRunPitch - (int)hi);
+                w.w = 4 * (j2 * kRunPitch - (int)(sum + 1u - (1u << j2)));
+            }
+            runs.window[i] = w;
+        }
+    }
     int h = -1, bb = 0;
     RoundState st;
     st.B = 0;
@@ -432,71 +474,38 @@ __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t 
         bb = __ffs(own) - 1;
         st.B = own_bit;
     }
-    st.sum = 0;
     uint8_t *row = stage + threadIdx.x * q;
-    // run[j] / run_before[j]: baseblock bits OR-ed over the 2^j ranks ending at this lane's rank,
-    // resp. at the rank 32 below it (doubling; a lane's run may start in the 32 ranks before the
-    // warp).  A window of L ranks is the union of two runs of 2^floor(log2 L) ranks.
-    uint32_t run[5], run_before[5];
-    run[0] = own_bit;
-    run_before[0] = before_bit;
+    __syncthreads();
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const unsigned w = 1u << j;
-        const uint32_t up = __shfl_up_sync(kAll, run[j], w);
-        const uint32_t wrap = __shfl_down_sync(kAll, run_before[j], 32u - w);
-        const uint32_t up_before = __shfl_up_sync(kAll, run_before[j], w);
-        run[j + 1] = run[j] | (lane >= w ? up : wrap);
-        run_before[j + 1] = run_before[j] | up_before;   // complete for lanes >= 2w - 1, all that is read
+    for (int j = 0; j + 1 < kRunLevels; ++j) {            // level j+1 from level j
+        const int w = 1 << j;
+        const uint32_t *from = runs.bits[j];
+        uint32_t *to = runs.bits[j + 1];
+        const int x = kRunBack + threadIdx.x;
+        to[x] = from[x] | from[x - w];
+        if (threadIdx.x < kRunBack && (int)threadIdx.x >= w)   // complete from x = 2^(j+1) - 1 on
+            to[threadIdx.x] = from[threadIdx.x] | from[threadIdx.x - w];
+        __syncthreads();
     }
-    // OR over the 2^j ranks ending d ranks below this lane's rank (1 <= d <= 32)
-    auto run_below = [&](int j, uint32_t d) {
-        const uint32_t a = __shfl_up_sync(kAll, run[j], d);
-        const uint32_t b = __shfl_down_sync(kAll, run_before[j], 32u - d);
-        return lane >= d ? a : b;
-    };
+    const char *mine = reinterpret_cast<const char *>(&runs.bits[0][kRunBack + threadIdx.x]);
+    auto word = [&](int byte_offset) { return *reinterpret_cast<const uint32_t *>(mine + byte_offset); };
     int i = 0;
 #pragma unroll 1
     for (; i < q && skip(i + 1) <= 33u; ++i) {            // uniform over the grid
-        const uint32_t lo = skip(i), hi = skip(i + 1);
-        st.sum += lo;
-        // ranks r - d, d = lo..hi-1: runs of 2^j ranks ending at r - lo and at r - (hi - 2^j)
-        uint32_t acc;
-        switch (31 - __clz(hi - lo)) {                      // uniform
-            case 0: acc = run_below(0, lo); break;
-            case 1: acc = run_below(1, lo) | run_below(1, hi - 2u); break;
-            case 2: acc = run_below(2, lo) | run_below(2, hi - 4u); break;
-            case 3: acc = run_below(3, lo) | run_below(3, hi - 8u); break;
-            default: acc = run_below(4, lo) | run_below(4, hi - 16u); break;
-        }
-        uint32_t U = acc & ~st.B;
-        const bool second = U == 0 && i != h;
-        if (__any_sync(kAll, second)) {
-            if (st.sum <= 32u) {                             // ranks r - d, d = skips[i+1]..sum
-                uint32_t acc2 = 0;
-                for (uint32_t d = hi; d <= st.sum; ++d) {
-                    const uint32_t a = __shfl_up_sync(kAll, own_bit, d);
-                    const uint32_t b = __shfl_down_sync(kAll, before_bit, 32u - d);
-                    acc2 |= lane >= d ? a : b;
-                }
-                if (second) U = acc2 & ~st.B;
-            } else if (second) {
-                const uint32_t below = r - hi + (r >= hi ? 0u : p);
-                const int b2 = pick_second_window(codes, full_sh, p, q, below, codes[below],
-                                                  st.sum - hi + 1u, st.B);
-                U = b2 >= 0 ? 1u << b2 : 0u;
-            }
-        }
-        int entry;
+        const int4 w = runs.window[i];
+        const uint32_t free_blocks = ~st.B;
+        uint32_t U = (word(w.x) | word(w.y)) & free_blocks;       // ranks r - d, d = skips[i]..skips[i+1]-1
+        const uint32_t U2 = (word(w.z) | word(w.w)) & free_blocks; // d = skips[i+1]..sum_{j<=i} skips[j]
+        if (U == 0) U = U2;
+        // largest block of U; the home round takes the baseblock and leaves B alone
+        const int lead = __clz(U);                                 // 32 when U == 0
+        uint32_t bit = U ? 0x80000000u >> lead : 0u;
+        int entry = U ? 31 - q - lead : BCS_BAD_ENTRY;
         if (i == h) {
             entry = bb;
-        } else if (U == 0) {
-            entry = BCS_BAD_ENTRY;
-        } else {
-            const int blk = 31 - __clz(U);
-            st.B |= 1u << blk;
-            entry = blk - q;
+            bit = 0;
         }
+        st.B |= bit;
         if (kRowOut) row[i] = (uint8_t)entry;
         if (kColOut && valid) *col = (int8_t)entry;
         if (kColOut) col += t_stride;
@@ -505,20 +514,16 @@ __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t 
         // Per-lane rounds.  Before the home round h both window bounds are r - skip, after it
         // both are r + p - skip: two loops with the wrap decided once, the home round between.
         const uint32_t edge = skip(i);
-        st.lo_skip = edge;
         st.upper = codes[r - edge + (r >= edge ? 0u : p)];  // code of r - skips[i]
         uint8_t *out = row + i;
         auto round = [&](int ii, uint32_t from) {           // from = r or r + p
-            const uint32_t hi = skip(ii + 1);
-            st.sum += st.lo_skip;
-            st.lo_skip = hi;
-            const uint32_t below = from - hi;
+            const uint32_t below = from - skip(ii + 1);
             const uint32_t lower = codes[below];
             const uint32_t diff = lower ^ st.upper;
             int blk = 31 - __clz(diff);                      // first head; -1 for an empty window
             int entry;
             if (diff == 0 || ((st.B >> blk) & 1u)) {
-                blk = pick_rest(codes, full_sh, p, q, below, lower, st.upper, st.sum - hi + 1u, st.B);
+                blk = pick_rest(codes, full_sh, p, q, below, lower, st.upper, runs.len2[ii], st.B);
                 entry = blk < 0 ? BCS_BAD_ENTRY : blk - q;
                 if (blk >= 0) st.B |= 1u << blk;
             } else {
@@ -532,13 +537,10 @@ __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t 
                 col += t_stride;
             }
         };
-#pragma unroll 1
+#pragma unroll 2
         for (; i < h; ++i) round(i, r);
         if (i == h) {                                        // home round: the baseblock itself
-            const uint32_t hi = skip(i + 1);
-            st.sum += st.lo_skip;
-            st.lo_skip = hi;
-            st.upper = codes[r + p - hi];
+            st.upper = codes[r + p - skip(i + 1)];
             if (kRowOut) *out++ = (uint8_t)bb;
             if (kColOut) {
                 *col = (int8_t)bb;
@@ -547,7 +549,7 @@ __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t 
             ++i;
         }
         const uint32_t rp = r + p;
-#pragma unroll 1
+#pragma unroll 2
         for (; i < q; ++i) round(i, rp);
     }
 }
@@ -560,6 +562,7 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uin
 {
     __shared__ __align__(16) uint8_t stage[kTile * 32];
     __shared__ uint32_t full_sh[kRow];
+    __shared__ RunTable runs;
     grid_launch_dependents();
     if (threadIdx.x < kRow) full_sh[threadIdx.x] = tab.full[threadIdx.x];
     __syncthreads();
@@ -569,7 +572,7 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uin
     grid_dependency_wait();                                // the codes are complete from here on
     recv_warp_tile<kRowOut, kColOut>(ParamSkips{tab}, full_sh, tab.p, tab.q, r_begin + g0, n, codes,
                                      stage, kColOut ? recv_t + g0 + threadIdx.x : nullptr,
-                                     t_stride);
+                                     t_stride, runs);
     if (kRowOut) {
         const uint32_t len = n * (uint32_t)tab.q;          // the tile's rows start at byte g0 * q: 16-byte aligned
         if ((len & 15u) == 0) {
@@ -591,6 +594,7 @@ recv_codes_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t
                         int8_t *recv_t)
 {
     __shared__ TileShared sh;
+    __shared__ RunTable runs;
     PTable unused;
     RankCtx c = resolve_rank<true>(sh, unused, 0, 0, ba);
     const uint32_t shift = (uint32_t)(sh.span_begin & 15u);
@@ -601,7 +605,7 @@ recv_codes_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t
         const uint64_t first = g0 - c.rank0;
         int8_t *col = kColOut ? recv_t + ba.entry_off[c.pj] + first + threadIdx.x : nullptr;
         recv_warp_tile<true, kColOut>(SharedSkips{sh.skips[0]}, sh.full[0], c.p, c.q, first, n,
-                                      codes + c.rank0, sh.stage + shift, col, (uint64_t)c.p);
+                                      codes + c.rank0, sh.stage + shift, col, (uint64_t)c.p, runs);
     } else if (c.valid && c.q > 0) {
         int8_t *col = kColOut ? recv_t + ba.entry_off[c.pj] + c.r : nullptr;
         uint8_t *row = sh.stage + shift + (c.entry - sh.span_begin);
