@@ -734,8 +734,9 @@ __device__ __forceinline__ void transpose_tile(const Skips skip, uint32_t p, int
 //     bytes -- q aligned words of the rank-major rows, since 4q bytes start at a multiple of 4 --
 //     are put together by byte permutations with selectors known at compile time.  Shared memory
 //     sees 3 word accesses per four entries instead of 8 byte accesses.
-//   * The rows leave as one bulk store.
-// 64 threads per 256 ranks; the many small CTAs per SM overlap one another's copies.
+//   * The rows are written over the round buffer (after a barrier) and leave as one bulk store.
+// 64 threads and 6 KB (q = 21) per 256 ranks: the whole grid of a million-rank table is resident
+// at once, and the many small CTAs per SM overlap one another's copies.
 constexpr int kTrThreads = kTile / 4;
 constexpr uint32_t kWaitLimit = 1u << 22;   // polls of the mbarrier before a CTA gives up
 
@@ -748,8 +749,7 @@ send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restri
                       uint64_t t_stride, int8_t *send_out, uint32_t r_begin, uint32_t count,
                       bool rotate)
 {
-    __shared__ __align__(128) uint8_t rounds[kQ * kTrPitch];
-    __shared__ __align__(16) uint8_t stage[kTile * kQ];
+    __shared__ __align__(128) uint8_t rounds[kQ * kTrPitch];   // later the rank-major rows (256 q bytes)
     __shared__ __align__(8) uint64_t bar;
     __shared__ uint32_t lead[kQ];            // offset of the tile's first byte inside its pitch row
     __shared__ uint32_t wraps;               // rounds whose bytes pass the end of the row
@@ -812,6 +812,8 @@ send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restri
         const uint32_t *word = reinterpret_cast<const uint32_t *>(rounds + (off & ~3u));
         W[k] = __funnelshift_r(word[0], word[1], (off & 3u) * 8u);
     }
+    __syncthreads();                                       // everyone has read: the rows take the buffer over
+    uint8_t *stage = rounds;
     // output word m holds bytes 4m..4m+3 of the four rows: byte e is rank e / q, round e % q
     uint32_t *rows = reinterpret_cast<uint32_t *>(stage) + threadIdx.x * kQ;
 #pragma unroll
