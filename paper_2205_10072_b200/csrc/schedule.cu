@@ -397,26 +397,79 @@ recv_codes_kernel(PTable tab, uint64_t r_begin, uint64_t r_end,
 // run the code search per lane.
 // Where the skips of the tile's p are read from: the kernel parameter (single p: immediate /
 // constant-bank operands) or a table row in shared memory (batch).
+struct RoundConsts;
+struct RunTable;
 struct ParamSkips {
     const PTable &tab;
+    const RoundConsts &rc;
+    static constexpr bool kHostConsts = true;          // per-round constants come with the launch
     __device__ __forceinline__ uint32_t operator()(int k) const { return tab.s[k]; }
+    __device__ __forceinline__ int4 window(int i, const RunTable &) const;
+    __device__ __forceinline__ uint32_t len2(int i, const RunTable &) const;
 };
 struct SharedSkips {
     const uint32_t *s;
+    static constexpr bool kHostConsts = false;         // the CTA computes them into its RunTable
     __device__ __forceinline__ uint32_t operator()(int k) const { return s[k]; }
+    __device__ __forceinline__ int4 window(int i, const RunTable &runs) const;
+    __device__ __forceinline__ uint32_t len2(int i, const RunTable &runs) const;
 };
 
 constexpr int kRunBack = 64;                   // ranks before the tile that the run table covers
 constexpr int kRunLevels = 5;                  // runs of 1, 2, 4, 8, 16 ranks
 constexpr int kRunPitch = kTile + kRunBack;    // words per level
-struct RunTable {
-    uint32_t bits[kRunLevels][kRunPitch];
+// Per-round constants of one p.
+struct RoundConsts {
     // Round i of the table rounds reads the four words at these byte offsets from a thread's own
     // level-0 entry: .x | .y is its first window, .z | .w its second (a repeat of the first when
     // the round has no second window).
     int4 window[8];
     uint32_t len2[kRow];     // length of the second window of round i: sum_{j<=i} skips[j] - skips[i+1] + 1, or 0
 };
+struct RunTable {
+    uint32_t bits[kRunLevels][kRunPitch];
+    RoundConsts rc;          // used by the batch kernel only
+};
+
+// Constants of round i (host and device) from the skips of the p at hand.
+__host__ __device__ inline void round_consts(const uint32_t *skips, int i, RoundConsts *rc)
+{
+    uint32_t sum = 0;
+    for (int j = 0; j <= i; ++j) sum += skips[j];
+    const uint32_t lo = skips[i], hi = skips[i + 1];
+    const uint32_t len2 = sum >= hi ? sum - hi + 1u : 0u;
+    rc->len2[i] = len2;
+    if (hi <= 33u) {
+        // the len >= 1 ranks that end d ranks below: runs of 2^j ranks, j = floor(log2 len),
+        // ending d and d + len - 2^j ranks below
+        int j1 = 0;
+        while ((2u << j1) <= hi - lo) ++j1;
+        int4 w;
+        w.x = 4 * (j1 * kRunPitch - (int)lo);
+        w.y = 4 * (j1 * kRunPitch - (int)(hi - (1u << j1)));
+        w.z = w.x;
+        w.w = w.y;
+        if (len2) {
+            int j2 = 0;
+            while ((2u << j2) <= len2) ++j2;
+            w.z = 4 * (j2 * kRunPitch - (int)hi);
+            w.w = 4 * (j2 * kRunPitch - (int)(sum + 1u - (1u << j2)));
+        }
+        rc->window[i] = w;
+    }
+}
+
+__device__ __forceinline__ int4 ParamSkips::window(int i, const RunTable &) const { return rc.window[i]; }
+__device__ __forceinline__ uint32_t ParamSkips::len2(int i, const RunTable &) const { return rc.len2[i]; }
+__device__ __forceinline__ int4 SharedSkips::window(int i, const RunTable &runs) const { return runs.rc.window[i]; }
+__device__ __forceinline__ uint32_t SharedSkips::len2(int i, const RunTable &runs) const { return runs.rc.len2[i]; }
+
+inline RoundConsts make_round_consts(const PTable &tab)
+{
+    RoundConsts rc = {};
+    for (int i = 0; i < tab.q; ++i) round_consts(tab.s, i, &rc);
+    return rc;
+}
 
 // The tile is the n ranks first..first+n-1 of a p (n <= 256, one per thread); `stage` is where
 // the tile's rank-major rows start in shared memory, `col` this thread's element of round 0 in
@@ -442,29 +495,8 @@ __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t 
         const uint32_t c = codes[(uint32_t)back];
         runs.bits[0][threadIdx.x] = c & (0u - c);
     }
-    if (threadIdx.x < (uint32_t)q) {                      // per-round constants of this p
-        const int i = threadIdx.x;
-        uint32_t sum = 0;
-        for (int j = 0; j <= i; ++j) sum += skip(j);
-        const uint32_t lo = skip(i), hi = skip(i + 1);
-        const uint32_t len2 = sum >= hi ? sum - hi + 1u : 0u;
-        runs.len2[i] = len2;
-        if (hi <= 33u) {
-            // the len >= 1 ranks that end d ranks below: runs of 2^j ranks, j = floor(log2 len),
-            // ending d and d + len - 2^j ranks below
-            const int j1 = 31 - __clz(hi - lo);
-            int4 w;
-            w.x = 4 * (j1 * kRunPitch - (int)lo);
-            w.y = 4 * (j1 * kRunPitch - (int)(hi - (1u << j1)));
-            w.z = w.x;
-            w.w = w.y;
-            if (len2) {
-                const int j2 = 31 - __clz(len2);
-                w.z = 4 * (j2 * kRunPitch - (int)hi);
-                w.w = 4 * (j2 * kRunPitch - (int)(sum + 1u - (1u << j2)));
-            }
-            runs.window[i] = w;
-        }
+    if constexpr (!Skips::kHostConsts) {                  // per-round constants of this p
+        if (threadIdx.x < (uint32_t)q) round_consts(skip.s, threadIdx.x, &runs.rc);
     }
     int h = -1, bb = 0;
     RoundState st;
@@ -476,23 +508,32 @@ __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t 
     }
     uint8_t *row = stage + threadIdx.x * q;
     __syncthreads();
-#pragma unroll
-    for (int j = 0; j + 1 < kRunLevels; ++j) {            // level j+1 from level j
-        const int w = 1 << j;
-        const uint32_t *from = runs.bits[j];
-        uint32_t *to = runs.bits[j + 1];
-        const int x = kRunBack + threadIdx.x;
-        to[x] = from[x] | from[x - w];
-        if (threadIdx.x < kRunBack && (int)threadIdx.x >= w)   // complete from x = 2^(j+1) - 1 on
-            to[threadIdx.x] = from[threadIdx.x] | from[threadIdx.x - w];
-        __syncthreads();
-    }
+    // levels 1 and 2 from level 0, then levels 3 and 4 from level 2: entry x of level j is
+    // complete from x = 2^j - 1 on, and nothing below x = 23 is ever read
+    auto build = [&](int x) {
+        const uint32_t *b = &runs.bits[0][x];
+        const uint32_t pair = b[0] | b[-1];
+        runs.bits[1][x] = pair;
+        runs.bits[2][x] = pair | b[-2] | b[-3];
+    };
+    build(kRunBack + threadIdx.x);
+    if (threadIdx.x < kRunBack && threadIdx.x >= 3u) build(threadIdx.x);
+    __syncthreads();
+    auto build_wide = [&](int x) {
+        const uint32_t *b = &runs.bits[2][x];
+        const uint32_t eight = b[0] | b[-4];
+        runs.bits[3][x] = eight;
+        runs.bits[4][x] = eight | b[-8] | b[-12];
+    };
+    build_wide(kRunBack + threadIdx.x);
+    if (threadIdx.x < kRunBack && threadIdx.x >= 15u) build_wide(threadIdx.x);
+    __syncthreads();
     const char *mine = reinterpret_cast<const char *>(&runs.bits[0][kRunBack + threadIdx.x]);
     auto word = [&](int byte_offset) { return *reinterpret_cast<const uint32_t *>(mine + byte_offset); };
     int i = 0;
 #pragma unroll 1
     for (; i < q && skip(i + 1) <= 33u; ++i) {            // uniform over the grid
-        const int4 w = runs.window[i];
+        const int4 w = skip.window(i, runs);
         const uint32_t free_blocks = ~st.B;
         uint32_t U = (word(w.x) | word(w.y)) & free_blocks;       // ranks r - d, d = skips[i]..skips[i+1]-1
         const uint32_t U2 = (word(w.z) | word(w.w)) & free_blocks; // d = skips[i+1]..sum_{j<=i} skips[j]
@@ -523,7 +564,7 @@ __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t 
             int blk = 31 - __clz(diff);                      // first head; -1 for an empty window
             int entry;
             if (diff == 0 || ((st.B >> blk) & 1u)) {
-                blk = pick_rest(codes, full_sh, p, q, below, lower, st.upper, runs.len2[ii], st.B);
+                blk = pick_rest(codes, full_sh, p, q, below, lower, st.upper, skip.len2(ii, runs), st.B);
                 entry = blk < 0 ? BCS_BAD_ENTRY : blk - q;
                 if (blk >= 0) st.B |= 1u << blk;
             } else {
@@ -556,9 +597,9 @@ __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t 
 
 template <bool kRowOut, bool kColOut>
 __global__ void __launch_bounds__(kTile, 8)
-recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uint64_t r_end,
-                       const uint32_t *__restrict__ codes, int8_t *recv_out, int8_t *recv_t,
-                       uint64_t t_stride)
+recv_codes_warp_kernel(const __grid_constant__ PTable tab, const __grid_constant__ RoundConsts rc,
+                       uint64_t r_begin, uint64_t r_end, const uint32_t *__restrict__ codes,
+                       int8_t *recv_out, int8_t *recv_t, uint64_t t_stride)
 {
     __shared__ __align__(16) uint8_t stage[kTile * 32];
     __shared__ uint32_t full_sh[kRow];
@@ -570,7 +611,7 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, uint64_t r_begin, uin
     const uint64_t g0 = (uint64_t)blockIdx.x * kTile;
     const uint32_t n = (uint32_t)(count - g0 < (uint64_t)kTile ? count - g0 : (uint64_t)kTile);
     grid_dependency_wait();                                // the codes are complete from here on
-    recv_warp_tile<kRowOut, kColOut>(ParamSkips{tab}, full_sh, tab.p, tab.q, r_begin + g0, n, codes,
+    recv_warp_tile<kRowOut, kColOut>(ParamSkips{tab, rc}, full_sh, tab.p, tab.q, r_begin + g0, n, codes,
                                      stage, kColOut ? recv_t + g0 + threadIdx.x : nullptr,
                                      t_stride, runs);
     if (kRowOut) {
@@ -954,24 +995,25 @@ bcs_status bcs_build(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_
         ws.t_stride = align_up(count, 16);
         launch_codes(tab, ws.codes, stream);
         if ((st = launch_status()) != BCS_OK) return st;
-        const bool warp_rounds = p >= 64;      // the warp-cooperative kernel needs 32 ranks back
+        const bool warp_rounds = p >= 64;      // the table kernel needs 64 distinct ranks back
+        const RoundConsts rc = make_round_consts(tab);
         if (recv_out != nullptr && send_out != nullptr) {
             if (warp_rounds)
-                launch_dependent(true, recv_codes_warp_kernel<true, true>, blocks, kTile, stream, tab,
+                launch_dependent(true, recv_codes_warp_kernel<true, true>, blocks, kTile, stream, tab, rc,
                                  r_begin, r_end, ws.codes, recv_out, ws.recv_t, ws.t_stride);
             else
                 recv_codes_kernel<true, true><<<blocks, kTile, 0, stream>>>(
                     tab, r_begin, r_end, ws.codes, recv_out, ws.recv_t, ws.t_stride);
         } else if (recv_out != nullptr) {
             if (warp_rounds)
-                launch_dependent(true, recv_codes_warp_kernel<true, false>, blocks, kTile, stream, tab,
+                launch_dependent(true, recv_codes_warp_kernel<true, false>, blocks, kTile, stream, tab, rc,
                                  r_begin, r_end, ws.codes, recv_out, nullptr, 0);
             else
                 recv_codes_kernel<true, false><<<blocks, kTile, 0, stream>>>(
                     tab, r_begin, r_end, ws.codes, recv_out, nullptr, 0);
         } else {
             if (warp_rounds)
-                launch_dependent(true, recv_codes_warp_kernel<false, true>, blocks, kTile, stream, tab,
+                launch_dependent(true, recv_codes_warp_kernel<false, true>, blocks, kTile, stream, tab, rc,
                                  r_begin, r_end, ws.codes, nullptr, ws.recv_t, ws.t_stride);
             else
                 recv_codes_kernel<false, true><<<blocks, kTile, 0, stream>>>(
@@ -1026,6 +1068,7 @@ bcs_status bcs_prepare(uint32_t p, void *workspace, size_t workspace_bytes, void
     if ((st = launch_status()) != BCS_OK) return st;
     if (p >= 64)
         launch_dependent(true, recv_codes_warp_kernel<false, true>, blocks, kTile, stream, tab,
+                         make_round_consts(tab),
                          (uint64_t)0, (uint64_t)p, codes, nullptr, recv_t, t_stride);
     else
         recv_codes_kernel<false, true><<<blocks, kTile, 0, stream>>>(tab, 0, p, codes, nullptr,
@@ -1149,8 +1192,6 @@ bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_
     return BCS_OK;
 }
 
-// Device address of g_static_scratch on the current device, looked up once per device (with that
-// device current) and remembered; nullptr if the runtime refuses.
 bcs_status bcs_wait_expired(uint64_t *count_host)
 {
     if (count_host == nullptr) return BCS_ERR_ARG;
@@ -1160,6 +1201,8 @@ bcs_status bcs_wait_expired(uint64_t *count_host)
     return BCS_OK;
 }
 
+// Device address of g_static_scratch on the current device, looked up once per device (with that
+// device current) and remembered; nullptr if the runtime refuses.
 static void *static_scratch_address()
 {
     constexpr int kMaxDevices = 64;
