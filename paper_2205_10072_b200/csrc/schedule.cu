@@ -557,14 +557,14 @@ __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t 
         const uint32_t edge = skip(i);
         st.upper = codes[r - edge + (r >= edge ? 0u : p)];  // code of r - skips[i]
         uint8_t *out = row + i;
-        auto round = [&](int ii, uint32_t from) {           // from = r or r + p
-            const uint32_t below = from - skip(ii + 1);
-            const uint32_t lower = codes[below];
+        // lower = code of the rank at the lower end of the window, from - skips[ii+1]
+        auto round = [&](int ii, uint32_t from, uint32_t lower) {
             const uint32_t diff = lower ^ st.upper;
             int blk = 31 - __clz(diff);                      // first head; -1 for an empty window
             int entry;
             if (diff == 0 || ((st.B >> blk) & 1u)) {
-                blk = pick_rest(codes, full_sh, p, q, below, lower, st.upper, skip.len2(ii, runs), st.B);
+                blk = pick_rest(codes, full_sh, p, q, from - skip(ii + 1), lower, st.upper,
+                                skip.len2(ii, runs), st.B);
                 entry = blk < 0 ? BCS_BAD_ENTRY : blk - q;
                 if (blk >= 0) st.B |= 1u << blk;
             } else {
@@ -578,8 +578,19 @@ __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t 
                 col += t_stride;
             }
         };
+        // The code a round needs depends on the rank and the round only, not on the rounds
+        // before: it is loaded one round ahead, so its latency overlaps the round in between.
+        auto rounds_until = [&](int end, uint32_t from) {    // from = r or r + p
+            if (i >= end) return;
+            uint32_t ahead = codes[from - skip(i + 1)];
 #pragma unroll 2
-        for (; i < h; ++i) round(i, r);
+            for (; i < end; ++i) {
+                const uint32_t lower = ahead;
+                if (i + 1 < end) ahead = codes[from - skip(i + 2)];
+                round(i, from, lower);
+            }
+        };
+        rounds_until(h < q ? h : q, r);
         if (i == h) {                                        // home round: the baseblock itself
             st.upper = codes[r + p - skip(i + 1)];
             if (kRowOut) *out++ = (uint8_t)bb;
@@ -589,9 +600,7 @@ __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t 
             }
             ++i;
         }
-        const uint32_t rp = r + p;
-#pragma unroll 2
-        for (; i < q; ++i) round(i, rp);
+        rounds_until(q, r + p);
     }
 }
 
@@ -605,8 +614,7 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, const __grid_constant
     __shared__ uint32_t full_sh[kRow];
     __shared__ RunTable runs;
     grid_launch_dependents();
-    if (threadIdx.x < kRow) full_sh[threadIdx.x] = tab.full[threadIdx.x];
-    __syncthreads();
+    if (threadIdx.x < kRow) full_sh[threadIdx.x] = tab.full[threadIdx.x];   // read after the tile's first barrier
     const uint64_t count = r_end - r_begin;
     const uint64_t g0 = (uint64_t)blockIdx.x * kTile;
     const uint32_t n = (uint32_t)(count - g0 < (uint64_t)kTile ? count - g0 : (uint64_t)kTile);
