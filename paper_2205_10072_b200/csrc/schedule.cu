@@ -11,11 +11,13 @@
 //    consecutive threads read consecutive words) and find the largest new block of the window
 //    from the two codes alone: walking down from the first level where they differ, every step
 //    yields one "head" (a rank whose baseblock is that level) and a run of low blocks; the rounds
-//    whose windows reach at most 32 ranks back are done by the whole warp with shuffles.  They
-//    write the rows rank-major and a round-major copy, from which send_transpose_kernel /
-//    send_batch_kernel produce sendsched[r][k] = recvsched[(r+skips[k]) mod p][k] as a
-//    transposition with row k rotated by skips[k] (send_rm_kernel: sub-ranges, byte gathers and
-//    recomputation for to-processors outside the range).
+//    whose windows reach only a few ranks back read them from a table of the tile's baseblock
+//    bits in shared memory.  They write the rows rank-major and a round-major copy, from which
+//    send_transpose_kernel / send_batch_kernel produce
+//    sendsched[r][k] = recvsched[(r+skips[k]) mod p][k] as a transposition with row k rotated by
+//    skips[k] (send_rm_kernel: sub-ranges, byte gathers and recomputation for to-processors
+//    outside the range).  The three kernels of a single-p build are launched as dependents of one
+//    another (bcs_common.cuh), so each is brought onto the SMs while the one before it drains.
 //
 //  * self-contained path (no workspace).  One thread per rank runs Algorithm 4 with the range
 //    search done by descending the homeranges; the send schedule is looked up in the rank-major
