@@ -301,10 +301,15 @@ def run_ours(args) -> None:
     def flush():
         flush_buf.fill_(1)
 
-    if args.only in ("expand", "checksum", "batch", "allgather"):   # small single-part runs (profiling)
+    if args.only in ("expand", "checksum", "batch", "allgather", "probe"):   # small single-part runs (profiling)
         if rank == 0:
             res = {}
-            if args.only == "allgather":
+            if args.only == "probe":
+                names = ("logic_only", "logic_imad_mix", "logic_add_mix")
+                res["int_rate_probe"] = {nm: [bcs.bcs_probe_int_rate(mix, 1024) / 1e12 for _ in range(2)]
+                                         for mix, nm in enumerate(names)}
+                res["int_rate_probe"]["unit"] = "Tint-op/s"
+            elif args.only == "allgather":
                 res["allgather_tables"] = _bench_allgather(torch, bcs, workloads, flush, hbm_gbs,
                                                            peak_src, args.steps)
             elif args.only in ("expand", "checksum"):
@@ -477,7 +482,7 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--only", default="all",
-                    choices=["all", "build", "expand", "checksum", "batch", "allgather"],
+                    choices=["all", "build", "expand", "checksum", "batch", "allgather", "probe"],
                     help="run one part only (small, profiler-friendly runs); 'all' is the benchmark")
     args = ap.parse_args()
     if args.impl == "reference":
