@@ -383,6 +383,14 @@ def run_ours(args) -> None:
         roof["peak_measured"] = {"logic_only": meas[0], "logic_imad_mix": meas[1],
                                  "logic_add_mix": meas[2], "unit": "Tint-op/s"}
         roof["frac_of_measured_logic_only"] = achieved / meas[0]
+        # the same time against the issue limit (one warp instruction per cycle and SM
+        # sub-partition), with the instructions the kernels really execute
+        issue_peak = SM_COUNT * 4 * 32 * sm_max_mhz * 1e6 / 1e12
+        executed = EXECUTED_INST_PER_RANK[q] * p / (recv_ms * 1e-3) / 1e12
+        roof["issue"] = {"executed_thread_inst_per_rank": EXECUTED_INST_PER_RANK[q],
+                         "achieved": executed, "peak": issue_peak, "unit": "Tthread-inst/s",
+                         "frac": executed / issue_peak,
+                         "frac_of_measured_two_pipe_mix": executed / max(meas[1], meas[2])}
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -465,7 +473,10 @@ def run_ours(args) -> None:
 
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of the
 # current kernels); None until counters have been taken for the kernel as it stands.
-RECV_TRAFFIC_BYTES = 4218368 + 713728        # recv_codes_warp_kernel<true,true>, p = 2^20+1
+RECV_TRAFFIC_BYTES = 4218368 + 434944        # recv_codes_warp_kernel<true,true>, p = 2^20+1
+# thread instructions per rank that the codes and receive kernels execute on that workload
+# (smsp__thread_inst_executed.sum of the same capture / p): 111 + 1006
+EXECUTED_INST_PER_RANK = {21: 111 + 1006}
 EXPAND_TRAFFIC_BYTES = 1567312000 + 3457280   # expand_kernel, p = 100003, n = 1000
 
 # integer operations per rank of the receive-schedule construction that the kernels run, by q:
