@@ -391,6 +391,28 @@ def run_ours(args) -> None:
                          "achieved": executed, "peak": issue_peak, "unit": "Tthread-inst/s",
                          "frac": executed / issue_peak,
                          "frac_of_measured_two_pipe_mix": executed / max(meas[1], meas[2])}
+        # ---- the same step timed in other ways (reported beside the headline, not instead of it)
+        def back_to_back(count):
+            e0 = torch.cuda.Event(enable_timing=True)
+            e1 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(count):
+                step()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / count
+        b2b_ms = back_to_back(2000)                      # no L2 flush: the workspace stays in L2
+        sustained_steps, sustained_ms, t_s0 = 0, 0.0, time.perf_counter()
+        with ClockSampler(local) as clk_sustained:
+            while time.perf_counter() - t_s0 < 2.0:      # at least 2 s of back-to-back steps
+                sustained_ms += back_to_back(4000) * 4000
+                sustained_steps += 4000
+        timing = {"best_of_10_ms": min(ms[:10]) if len(ms) >= 10 else min(ms), "min_ms": min(ms),
+                  "median_ms": statistics.median(ms),
+                  "back_to_back_ms_per_step": b2b_ms,
+                  "sustained_ms_per_step": sustained_ms / sustained_steps,
+                  "sustained_steps": sustained_steps,
+                  "sustained_clocks": clk_sustained.summary()}
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -404,7 +426,7 @@ def run_ours(args) -> None:
             "out_gbs": 2 * nb / ms_per_step / 1e6,
             "kernel_ms": {"codes+recv_codes": recv_ms, "send_rm": send_ms,
                           "self_contained_path_step": slow_ms},
-            "workspace_bytes": ws_bytes,
+            "workspace_bytes": ws_bytes, "timing": timing,
             "roofline": roof, "gpu_launches": 3 * args.steps, "clocks": clk.summary(),
         }
         if args.only == "all":

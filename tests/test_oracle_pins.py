@@ -462,3 +462,31 @@ def test_checksum_definition_and_additivity():
     assert oracle.checksum(buf, big) == by_words(buf, big)
     swapped = buf.copy(); swapped[[3, 700]] = swapped[[700, 3]]
     assert buf[3] != buf[700] and oracle.checksum(swapped, 16) != want
+
+
+# ---------------------------------------------------------------- independent tripwire digests
+def _witness_lines():
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "witness_digests.txt")
+    with open(path) as f:
+        return [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+
+
+def test_table_digests_of_an_independent_implementation():
+    """Digests and one printed row computed by an independent implementation of the same reading
+    (see the fixture's header): not the paper's, so a tripwire beside the printed tables."""
+    import hashlib
+    for f in _witness_lines():
+        if f[0] == "row":
+            p, r = int(f[1]), int(f[2])
+            want = [int(v) for v in f[4].split(",")]
+            assert list(oracle.skips(p)) == [1, 2, 4, 7, 13, 25, 49, 98, 196, 391, 782, 1563, 3126,
+                                              6251, 12501, 25001, 50002, 100003]
+            got = oracle.recvsched(p, r) if f[3] == "recv" else oracle.sendsched(p, r)
+            assert list(got) == want, f
+            continue
+        p = int(f[0])
+        recv, send = oracle.full_table(p)
+        assert hashlib.sha256(recv.astype(np.int8).tobytes()).hexdigest()[:16] == f[1], p
+        assert hashlib.sha256(send.astype(np.int8).tobytes()).hexdigest()[:16] == f[2], p
+        assert int(recv.astype(np.int64).sum()) == int(f[3]) == int(send.astype(np.int64).sum()), p
