@@ -533,8 +533,10 @@ __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t 
     const char *mine = reinterpret_cast<const char *>(&runs.bits[0][kRunBack + threadIdx.x]);
     auto word = [&](int byte_offset) { return *reinterpret_cast<const uint32_t *>(mine + byte_offset); };
     int i = 0;
-#pragma unroll 1
-    for (; i < q && skip(i + 1) <= 33u; ++i) {            // uniform over the grid
+#pragma unroll
+    for (int unrolled = 0; unrolled < 6; ++unrolled) {    // at most six such rounds; uniform over the grid
+        if (!(unrolled < q && skip(unrolled + 1) <= 33u)) break;
+        i = unrolled;
         const int4 w = skip.window(i, runs);
         const uint32_t free_blocks = ~st.B;
         uint32_t U = (word(w.x) | word(w.y)) & free_blocks;       // ranks r - d, d = skips[i]..skips[i+1]-1
@@ -552,6 +554,7 @@ __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t 
         if (kRowOut) row[i] = (uint8_t)entry;
         if (kColOut && valid) *col = (int8_t)entry;
         if (kColOut) col += t_stride;
+        i = unrolled + 1;
     }
     if (valid && i < q) {
         // Per-lane rounds.  Before the home round h both window bounds are r - skip, after it
