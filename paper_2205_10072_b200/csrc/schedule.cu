@@ -392,9 +392,11 @@ recv_codes_kernel(PTable tab, uint64_t r_begin, uint64_t r_end,
 // of the table adds at most 3 more to the second and none beyond skips[i+1] - 1 to the first.  So
 // every baseblock those windows can contain is the lowest code bit of one of the tile's ranks or
 // of the 64 ranks before the tile.  The tile keeps, for x = every one of those 320 ranks and
-// j = 0..4, the baseblock bits OR-ed over the 2^j ranks that end at x (doubling, one barrier
-// per level); a window of L ranks is the union of two such runs of 2^floor(log2 L) ranks: two
-// shared-memory words per window, whatever its length.  These are the rounds in which
+// j = 0..4, the baseblock bits OR-ed over the 2^j ranks that end at x (runs of 2 and 4 from the
+// single bits, runs of 8 and 16 from the runs of 4: two barriers after the one that publishes the
+// bits); a window of L ranks is the union of two such runs of 2^floor(log2 L) ranks: two
+// shared-memory words per window, whatever its length, at offsets that depend on p and the round
+// only (RoundConsts).  These are the rounds in which
 // neighbouring ranks disagree about which path of the code search they take; the later rounds
 // run the code search per lane.
 // Where the skips of the tile's p are read from: the kernel parameter (single p: immediate /
