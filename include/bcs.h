@@ -124,6 +124,24 @@ bcs_status bcs_build_prepared(uint32_t p, uint64_t r_begin, uint64_t r_end,
 bcs_status bcs_build_static(uint32_t p, uint64_t r_begin, uint64_t r_end,
                             int8_t *recv_out, int8_t *send_out, void *cuda_stream);
 
+/* Schedules of a broadcast rooted at processor `root` (Section 2: the processors are renumbered
+ * by subtracting the root, so processor r uses the rank-0-rooted rows of virtual rank
+ * (r - root) mod p; the skips, and with them the neighbours (r +- skips[k]) mod p, do not depend
+ * on the root).  A thin remap over bcs_build:
+ *   out[(r - r_begin)*q + k] = entry k of virtual rank (r - root) mod p,  r in [r_begin, r_end).
+ * The virtual ranks of the range are one run, or two when they pass p - 1; each run is built
+ * by bcs_build.  The second run starts (p - v0)*q bytes into the outputs (v0 the first virtual
+ * rank); where that is not a multiple of 16 it is built in the workspace and copied into place
+ * on the stream (cudaMemcpyAsync, device to device).
+ *   root < p, else BCS_ERR_RANGE.  Outputs as for bcs_build.
+ *   workspace, workspace_bytes: at least bcs_build_rooted_workspace_bytes(...) bytes (16-byte
+ *   aligned) select the fast construction; NULL or less: the self-contained construction, which
+ *   is then refused with BCS_ERR_ARG if the range needs the copy described above. */
+size_t bcs_build_rooted_workspace_bytes(uint32_t p, uint32_t root, uint64_t r_begin, uint64_t r_end);
+bcs_status bcs_build_rooted(uint32_t p, uint32_t root, uint64_t r_begin, uint64_t r_end,
+                            int8_t *recv_out, int8_t *send_out, void *workspace,
+                            size_t workspace_bytes, void *cuda_stream);
+
 /* As bcs_build, then copies the tables to HOST memory on the same stream
  * (cudaMemcpyAsync; pinned host memory makes the copies asynchronous).
  *   recv_host, send_host: host, (r_end-r_begin)*q bytes each, either may be NULL.

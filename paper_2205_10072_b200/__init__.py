@@ -15,6 +15,8 @@ from .binding import (  # noqa: F401
     bcs_build_batch,
     bcs_build_batch_workspace_bytes,
     bcs_build_prepared,
+    bcs_build_rooted,
+    bcs_build_rooted_workspace_bytes,
     bcs_build_static,
     bcs_build_workspace_bytes,
     bcs_build_to_host,

@@ -77,6 +77,10 @@ def lib():
         L.bcs_probe_int_rate.argtypes = [i32, u32, vp, _c.POINTER(_c.c_double),
                                          _c.POINTER(_c.c_float), vp]
         L.bcs_probe_int_rate.restype = i32
+        L.bcs_build_rooted_workspace_bytes.argtypes = [u32, u32, u64, u64]
+        L.bcs_build_rooted_workspace_bytes.restype = _c.c_size_t
+        L.bcs_build_rooted.argtypes = [u32, u32, u64, u64, vp, vp, vp, _c.c_size_t, vp]
+        L.bcs_build_rooted.restype = i32
         L.bcs_wait_expired.argtypes = [_c.POINTER(u64)]
         L.bcs_wait_expired.restype = i32
         L.bcs_checksum.argtypes = [vp, u64, u64, vp, vp]
@@ -128,6 +132,19 @@ def bcs_build(p: int, r_begin: int, r_end: int, recv_out, send_out, workspace=No
     workspace: CUDA tensor of bcs_build_workspace_bytes(...) bytes (fast path) or None."""
     _check(lib().bcs_build(p, r_begin, r_end, _ptr(recv_out), _ptr(send_out), _ptr(workspace),
                            _nbytes(workspace), _stream(stream)), "bcs_build")
+
+
+def bcs_build_rooted_workspace_bytes(p: int, root: int, r_begin: int, r_end: int) -> int:
+    return lib().bcs_build_rooted_workspace_bytes(p, root, r_begin, r_end)
+
+
+def bcs_build_rooted(p: int, root: int, r_begin: int, r_end: int, recv_out, send_out,
+                     workspace=None, stream=None) -> None:
+    """As bcs_build for a broadcast rooted at `root`: row r is the rank-0-rooted row of virtual
+    rank (r - root) mod p."""
+    _check(lib().bcs_build_rooted(p, root, r_begin, r_end, _ptr(recv_out), _ptr(send_out),
+                                  _ptr(workspace), _nbytes(workspace), _stream(stream)),
+           "bcs_build_rooted")
 
 
 def bcs_prepare_workspace_bytes(p: int) -> int:

@@ -1120,6 +1120,74 @@ bcs_status bcs_build_prepared(uint32_t p, uint64_t r_begin, uint64_t r_end, int8
     return BCS_OK;
 }
 
+// The runs of virtual ranks (r - root) mod p of the range [r_begin, r_end): [v0, v0 + len_a) and,
+// when the range passes virtual rank p - 1, [0, len_b).
+struct RootedRuns {
+    uint64_t v0, len_a, len_b;
+};
+
+static RootedRuns rooted_runs(uint32_t p, uint32_t root, uint64_t r_begin, uint64_t r_end)
+{
+    RootedRuns rr;
+    const uint64_t count = r_end - r_begin;
+    rr.v0 = count ? (r_begin + p - root) % p : 0;
+    rr.len_a = count < p - rr.v0 ? count : p - rr.v0;
+    rr.len_b = count - rr.len_a;
+    return rr;
+}
+
+size_t bcs_build_rooted_workspace_bytes(uint32_t p, uint32_t root, uint64_t r_begin, uint64_t r_end)
+{
+    if (check_range(p, r_begin, r_end) != BCS_OK || root >= p) return 0;
+    const int q = ceil_log2_u32(p);
+    const RootedRuns rr = rooted_runs(p, root, r_begin, r_end);
+    const size_t a = bcs_build_workspace_bytes(p, rr.v0, rr.v0 + rr.len_a);
+    const size_t b = bcs_build_workspace_bytes(p, 0, rr.len_b);
+    // two staging tables for the second run (used only where it lands off a 16-byte boundary)
+    return (size_t)align_up(a > b ? a : b, 256) + 2 * (size_t)align_up(rr.len_b * (uint64_t)q, 256);
+}
+
+bcs_status bcs_build_rooted(uint32_t p, uint32_t root, uint64_t r_begin, uint64_t r_end,
+                            int8_t *recv_out, int8_t *send_out, void *workspace,
+                            size_t workspace_bytes, void *cuda_stream)
+{
+    bcs_status st = check_range(p, r_begin, r_end);
+    if (st != BCS_OK) return st;
+    if (root >= p) return BCS_ERR_RANGE;
+    const int q = ceil_log2_u32(p);
+    if (r_begin == r_end || q == 0) return BCS_OK;
+    if (recv_out == nullptr && send_out == nullptr) return BCS_ERR_ARG;
+    if (!aligned16(recv_out) || !aligned16(send_out) || !aligned16(workspace)) return BCS_ERR_ALIGN;
+    const RootedRuns rr = rooted_runs(p, root, r_begin, r_end);
+    const bool fast = workspace != nullptr &&
+                      workspace_bytes >= bcs_build_rooted_workspace_bytes(p, root, r_begin, r_end);
+    const uint64_t bytes_a = rr.len_a * (uint64_t)q, bytes_b = rr.len_b * (uint64_t)q;
+    const bool staged = rr.len_b != 0 && (bytes_a & 15u) != 0;
+    if (staged && !fast) return BCS_ERR_ARG;
+    // workspace = [construction scratch, a multiple of 256 bytes][recv staging][send staging]
+    const size_t need_a = bcs_build_workspace_bytes(p, rr.v0, rr.v0 + rr.len_a);
+    const size_t need_b = bcs_build_workspace_bytes(p, 0, rr.len_b);
+    const size_t build_ws = fast ? (size_t)align_up(need_a > need_b ? need_a : need_b, 256) : 0;
+    st = bcs_build(p, rr.v0, rr.v0 + rr.len_a, recv_out, send_out, fast ? workspace : nullptr, build_ws,
+                   cuda_stream);
+    if (st != BCS_OK || rr.len_b == 0) return st;
+    int8_t *recv_b = recv_out ? recv_out + bytes_a : nullptr;
+    int8_t *send_b = send_out ? send_out + bytes_a : nullptr;
+    if (!staged)
+        return bcs_build(p, 0, rr.len_b, recv_b, send_b, fast ? workspace : nullptr, build_ws, cuda_stream);
+    int8_t *stage_recv = static_cast<int8_t *>(workspace) + build_ws;
+    int8_t *stage_send = stage_recv + align_up(bytes_b, 256);
+    st = bcs_build(p, 0, rr.len_b, recv_out ? stage_recv : nullptr, send_out ? stage_send : nullptr,
+                   workspace, build_ws, cuda_stream);
+    if (st != BCS_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (recv_out && cudaMemcpyAsync(recv_b, stage_recv, bytes_b, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+        return BCS_ERR_CUDA;
+    if (send_out && cudaMemcpyAsync(send_b, stage_send, bytes_b, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+        return BCS_ERR_CUDA;
+    return BCS_OK;
+}
+
 bcs_status bcs_build_to_host(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_host,
                              int8_t *send_host, void *stage_dev, size_t stage_bytes,
                              void *cuda_stream)

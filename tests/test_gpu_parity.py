@@ -188,6 +188,58 @@ def test_prepare_then_build_ranges(bcs):
     assert bcs.bcs_prepare_workspace_bytes(20) == 256 + 5 * 32
 
 
+def test_rooted_builds_are_the_renumbered_schedule(bcs):
+    """Section 2: a broadcast from root rho uses the rank-0-rooted rows of virtual rank
+    (r - rho) mod p.  Full and partial ranges, runs that pass virtual rank p-1 on and off a
+    16-byte boundary, with and without a workspace; and the rooted tables drive a correct
+    n-block broadcast from rho in the brute-force simulation."""
+    L = bcs.lib()
+    for p, roots in ((2, (0, 1)), (20, (0, 7, 19)), (33, (5, 32)), (64, (63,)), (1000, (1, 16, 999)),
+                     (4097, (4000,)), (100003, (54607,))):
+        q = oracle.q_of(p)
+        want_r, want_s = oracle.full_table(p)
+        for root in roots:
+            virt = (np.arange(p) - root) % p
+            for r0, r1 in ((0, p), (root, min(p, root + 1)), (0, min(p, root + 3)),
+                           (max(0, root - 5), min(p, root + 300)), (p // 2, p)):
+                if r0 >= r1:
+                    continue
+                nb = (r1 - r0) * q
+                for fast in (True, False):
+                    raw_r, recv = _guarded(nb)
+                    raw_s, send = _guarded(nb)
+                    need = bcs.bcs_build_rooted_workspace_bytes(p, root, r0, r1)
+                    raw_w, ws = _guarded(need) if fast else (None, None)
+                    code = L.bcs_build_rooted(p, root, r0, r1, recv.data_ptr(), send.data_ptr(),
+                                              ws.data_ptr() if fast else None, need if fast else 0, None)
+                    torch.cuda.synchronize()
+                    v0 = (r0 - root) % p
+                    len_a = min(r1 - r0, p - v0)
+                    staged = (r1 - r0) > len_a and (len_a * q) % 16 != 0
+                    if not fast and staged:
+                        assert code == 1, (p, root, r0, r1)      # needs the workspace for the copy
+                        continue
+                    assert code == 0, (p, root, r0, r1, fast)
+                    assert _guards_intact(raw_r, nb) and _guards_intact(raw_s, nb)
+                    if fast:
+                        assert _guards_intact(raw_w, need)
+                    assert np.array_equal(recv.cpu().numpy().reshape(-1, q), want_r[virt[r0:r1]]), (p, root, r0, r1)
+                    assert np.array_equal(send.cpu().numpy().reshape(-1, q), want_s[virt[r0:r1]]), (p, root, r0, r1)
+    # the rooted tables, expanded, broadcast correctly from the root
+    p, root, n = 1000, 321, 7
+    q = oracle.q_of(p)
+    recv = torch.empty(p * q, dtype=torch.int8, device="cuda")
+    send = torch.empty(p * q, dtype=torch.int8, device="cuda")
+    ws = torch.empty(bcs.bcs_build_rooted_workspace_bytes(p, root, 0, p), dtype=torch.int8, device="cuda")
+    bcs.bcs_build_rooted(p, root, 0, p, recv, send, ws)
+    table = torch.empty((p, n - 1 + q, 4), dtype=torch.int32, device="cuda")
+    bcs.bcs_expand(p, n, 0, p, recv, send, table)
+    assert bcast_sim.simulate(p, n, table.cpu().numpy(), root=root) is None
+    assert L.bcs_build_rooted(20, 20, 0, 20, recv.data_ptr(), None, None, 0, None) == 2   # root out of range
+    assert bcs.bcs_build_rooted_workspace_bytes(20, 20, 0, 20) == 0
+    assert bcs.bcs_wait_expired() == 0
+
+
 def test_degenerate_sizes_and_errors(bcs):
     L = bcs.lib()
     buf = torch.zeros(64, dtype=torch.int8, device="cuda")
