@@ -191,17 +191,29 @@ __global__ void __launch_bounds__(kTile)
 codes_single_kernel(const __grid_constant__ PTable tab, uint32_t *__restrict__ codes)
 {
     grid_launch_dependents();
-    const uint64_t g = (uint64_t)blockIdx.x * kTile + threadIdx.x;
+    // four consecutive ranks per thread: four independent scans, one 16-byte store
+    const uint32_t g = (blockIdx.x * kTile + threadIdx.x) * 4u;
     if (g >= tab.p) return;
-    uint32_t x = (uint32_t)g, code = 0;
+    uint32_t x[4], code[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) x[e] = g + e;            // ranks >= p give unused codes
 #pragma unroll
     for (int k = kQ - 1; k >= 0; --k) {
-        if (x >= tab.s[k]) {
-            x -= tab.s[k];
-            code |= 1u << k;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (x[e] >= tab.s[k]) {
+                x[e] -= tab.s[k];
+                code[e] |= 1u << k;
+            }
         }
     }
-    codes[g] = code;
+    if (g + 4u <= tab.p) {
+        *reinterpret_cast<uint4 *>(codes + g) = make_uint4(code[0], code[1], code[2], code[3]);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (g + e < tab.p) codes[g + e] = code[e];
+    }
 }
 
 template <int kQ>
@@ -221,7 +233,8 @@ struct CodesLauncher<0> {
 
 inline void launch_codes(const PTable &tab, uint32_t *codes, cudaStream_t stream)
 {
-    CodesLauncher<BCS_MAX_Q>::launch(tab.q, tab, codes, (unsigned)((tab.p + kTile - 1) / kTile), stream);
+    CodesLauncher<BCS_MAX_Q>::launch(tab.q, tab, codes, (unsigned)((tab.p + 4 * kTile - 1) / (4 * kTile)),
+                                     stream);
 }
 
 // Batch: codes[g] for the flattened rank g.
