@@ -720,136 +720,71 @@ send_rm_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, const uint32_t *__r
 // Row k of the round-major send table is row k of the round-major receive copy rotated by
 // skips[k] (sendsched[r][k] = recvsched[(r+skips[k]) mod p][k]), so the send rows of a run of
 // ranks are a transposition with one rotation per row (and the receive rows the same with
-// rotation 0).  A CTA takes up to 256 consecutive ranks: for every round it copies the
-// (rotated, possibly wrapping) bytes it needs with 16-byte loads into shared memory, then every
-// thread gathers its column into the rank-major staging rows, which leave as one vectorised span.
-constexpr int kTrPitch = kTile + 32;      // bytes per round in shared memory: 256 + alignment slack
-
-struct TransposeShared {
-    __align__(16) uint8_t rounds[BCS_MAX_Q * kTrPitch];
-    uint32_t lead[BCS_MAX_Q];   // offset of the tile's first byte inside its pitch row
-    uint32_t wraps;             // rounds whose bytes pass the end of the row
-};
-
-// tbl: round 0 of the round-major table of this p (all p ranks per row, rows `stride` bytes
-// apart, any alignment; up to 15 bytes before a row's first and after its last needed byte are
-// read as well).  The tile is ranks r0..r0+n-1; stage: where its rank-major rows start.
-// kQ: q known at compile time (loops over the rounds unrolled), 0 = use the argument.
-template <int kQ, class Skips>
-__device__ __forceinline__ void transpose_tile(const Skips skip, uint32_t p, int q_arg,
-                                               const int8_t *__restrict__ tbl, uint64_t stride,
-                                               uint32_t r0, uint32_t n, bool rotate,
-                                               TransposeShared &ts, uint8_t *stage)
-{
-    const int q = kQ ? kQ : q_arg;
-    if (threadIdx.x == 0) ts.wraps = 0;
-    __syncthreads();
-    const int vecs = kTrPitch / 16;         // 18 vectors cover 256 bytes at any misalignment
-    for (int w = threadIdx.x; w < q * vecs; w += kTile) {
-        const int k = w / vecs, v = w - k * vecs;
-        const uint8_t *src_row = reinterpret_cast<const uint8_t *>(tbl) + (uint64_t)k * stride;
-        uint32_t start = r0 + (rotate ? skip(k) : 0u);
-        if (start >= p) start -= p;
-        const uint32_t mis = (uint32_t)(reinterpret_cast<uintptr_t>(src_row + start) & 15u);
-        const uint32_t run = p - start < n ? p - start : n;      // bytes before the wrap
-        if (v == 0) {
-            ts.lead[k] = mis;
-            if (run < n) atomicOr(&ts.wraps, 1u << k);
-        }
-        if ((uint32_t)v * 16u < mis + run)                        // the vector holds a needed byte
-            *reinterpret_cast<uint4 *>(ts.rounds + k * kTrPitch + v * 16) =
-                *reinterpret_cast<const uint4 *>(src_row + start - mis + v * 16);
-    }
-    __syncthreads();
-    for (uint32_t left = ts.wraps; left != 0; left &= left - 1u) {  // the part after the wrap, by bytes
-        const int k = __ffs(left) - 1;
-        uint32_t start = r0 + (rotate ? skip(k) : 0u);
-        if (start >= p) start -= p;
-        const uint32_t run = p - start;                           // < n for these rounds
-        const uint8_t *src_row = reinterpret_cast<const uint8_t *>(tbl) + (uint64_t)k * stride;
-        const uint32_t j = threadIdx.x;
-        if (j >= run && j < n) ts.rounds[k * kTrPitch + ts.lead[k] + j] = src_row[j - run];
-    }
-    if (ts.wraps) __syncthreads();
-    // lane l of warp w takes rank 128 * (w / 4) + 4 * l + (w % 4): the rows written by one
-    // warp start q * 4 bytes = q words apart, which is a different bank for every lane when q
-    // is odd, and the bytes it reads lie in 32 consecutive words.
-    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    const uint32_t mine = 128u * (warp >> 2) + 4u * lane + (warp & 3u);
-    if (mine < n) {
-        uint8_t *__restrict__ row = stage + mine * q;
-        const uint8_t *__restrict__ column = ts.rounds + mine;
-        const uint32_t *__restrict__ lead_k = ts.lead;
-        if (kQ) {
-#pragma unroll
-            for (int k = 0; k < (kQ ? kQ : 1); ++k) row[k] = column[k * kTrPitch + lead_k[k]];
-        } else {
-#pragma unroll 4
-            for (int k = 0; k < q; ++k) row[k] = column[k * kTrPitch + lead_k[k]];
-        }
-    }
-}
-
-// Single p, the same transposition on the copy unit and in registers.  recv_t holds all p ranks
-// of every round; the CTA's tile is ranks r0..r0+n-1 of the range r_begin..r_begin+count-1.
-// rotate: send rows; otherwise the receive rows themselves.
+// rotation 0).  A tile is up to 256 consecutive ranks of one p.
 //   * Thread k < q brings the (rotated) bytes of round k into shared memory with one bulk copy
 //     (cp.async.bulk global -> shared, completion counted on an mbarrier); the copy starts at the
 //     16-byte boundary at or before the first needed byte and ends at the one at or after the
-//     last.  A round whose bytes pass the end of the row (at most q tiles of a table) gets the
-//     part after the wrap by plain loads.
-//   * Thread j then takes the four ranks 4j..4j+3: one 32-bit word per round (two aligned words
-//     and a funnel shift, as the rotation puts the tile anywhere in the word), and its 4q output
-//     bytes -- q aligned words of the rank-major rows, since 4q bytes start at a multiple of 4 --
-//     are put together by byte permutations with selectors known at compile time.  Shared memory
-//     sees 3 word accesses per four entries instead of 8 byte accesses.
-//   * The rows are written over the round buffer (after a barrier) and leave as one bulk store.
-// 64 threads and 6 KB (q = 21) per 256 ranks: the whole grid of a million-rank table is resident
-// at once, and the many small CTAs per SM overlap one another's copies.
-constexpr int kTrThreads = kTile / 4;
+//     last (up to 15 bytes before and after the needed ones are read as well).  A round whose
+//     bytes pass the end of the row (at most q tiles of a table) gets the part after the wrap
+//     by plain loads.
+//   * Thread j < 64 then takes the four ranks 4j..4j+3: one 32-bit word per round (two aligned
+//     words and a funnel shift, as the rotation puts the tile anywhere in the word), and its 4q
+//     output bytes -- q words of the rank-major rows -- are put together by byte permutations
+//     with selectors known at compile time (one instantiation per q).  Shared memory sees 3 word
+//     accesses per four entries instead of 8 byte accesses.
+constexpr int kTrPitch = kTile + 32;        // bytes per round in shared memory: 256 + alignment slack
+constexpr int kTrThreads = kTile / 4;       // threads that gather
 constexpr uint32_t kWaitLimit = 1u << 22;   // polls of the mbarrier before a CTA gives up
 
 // CTAs whose bulk load did not complete within kWaitLimit polls (they leave their tile unwritten).
 __device__ unsigned long long g_wait_expired;
 
-template <int kQ>
-__global__ void __launch_bounds__(kTrThreads)
-send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restrict__ recv_t,
-                      uint64_t t_stride, int8_t *send_out, uint32_t r_begin, uint32_t count,
-                      bool rotate)
+template <int kRounds>
+struct RoundBuffer {
+    __align__(128) uint8_t rounds[kRounds * kTrPitch];
+    __align__(8) uint64_t bar;
+    uint32_t lead[kRounds];     // offset of the tile's first byte inside its pitch row
+    uint32_t wraps;             // rounds whose bytes pass the end of the row
+};
+
+// Skips from the kernel parameter (single p).
+struct TableSkips {
+    const PTable &tab;
+    __device__ __forceinline__ uint32_t operator()(int k) const { return tab.s[k]; }
+};
+
+// All threads of the CTA call.  tbl: round 0 of the round-major table of this p (rows `stride`
+// bytes apart, any alignment); the tile is ranks r0..r0+n-1 (r0 < p, n <= 256, n <= p).
+// Returns false, in all threads, if the copies did not arrive within the poll limit.
+template <class Skips, class Buffer>
+__device__ __forceinline__ bool load_rounds(const Skips skip, uint32_t p, int q,
+                                            const int8_t *__restrict__ tbl, uint64_t stride,
+                                            uint32_t r0, uint32_t n, bool rotate, Buffer &rb)
 {
-    __shared__ __align__(128) uint8_t rounds[kQ * kTrPitch];   // later the rank-major rows (256 q bytes)
-    __shared__ __align__(8) uint64_t bar;
-    __shared__ uint32_t lead[kQ];            // offset of the tile's first byte inside its pitch row
-    __shared__ uint32_t wraps;               // rounds whose bytes pass the end of the row
-    const uint32_t p = tab.p;
-    const uint32_t first = blockIdx.x * kTile;
-    const uint32_t n = count - first < (uint32_t)kTile ? count - first : (uint32_t)kTile;
-    const uint32_t r0 = r_begin + first;
-    const uint32_t bar_addr = (uint32_t)__cvta_generic_to_shared(&bar);
+    const uint32_t bar_addr = (uint32_t)__cvta_generic_to_shared(&rb.bar);
     if (threadIdx.x == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar_addr), "r"(kQ) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar_addr), "r"(q) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        wraps = 0;
+        rb.wraps = 0;
     }
     grid_launch_dependents();
     __syncthreads();
     grid_dependency_wait();                                    // the round-major copy is complete
-    if (threadIdx.x < kQ) {
+    if (threadIdx.x < (uint32_t)q) {
         const int k = threadIdx.x;
-        uint32_t start = r0 + (rotate ? tab.s[k] : 0u);
+        uint32_t start = r0 + (rotate ? skip(k) : 0u);
         if (start >= p) start -= p;
-        const uint32_t mis = start & 15u;                      // rows start 16-byte aligned
+        const uint64_t from = reinterpret_cast<uint64_t>(tbl) + (uint64_t)k * stride + start;
+        const uint32_t mis = (uint32_t)(from & 15u);
         const uint32_t run = p - start < n ? p - start : n;    // bytes before the wrap
         const uint32_t bytes = (mis + run + 15u) & ~15u;       // <= 272, inside the row's pitch
-        lead[k] = mis;
-        if (run < n) atomicOr(&wraps, 1u << k);
-        const uint64_t src = reinterpret_cast<uint64_t>(recv_t) + (uint64_t)k * t_stride + (start - mis);
-        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(rounds + k * kTrPitch);
+        rb.lead[k] = mis;
+        if (run < n) atomicOr(&rb.wraps, 1u << k);
+        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(rb.rounds + k * kTrPitch);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
                      :: "r"(bar_addr), "r"(bytes) : "memory");
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     :: "r"(dst), "l"(src), "r"(bytes), "r"(bar_addr) : "memory");
+                     :: "r"(dst), "l"(from - mis), "r"(bytes), "r"(bar_addr) : "memory");
     }
     uint32_t done = 0;
     for (uint32_t poll = 0; poll < kWaitLimit && !done; ++poll)
@@ -859,41 +794,71 @@ send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restri
                      : "=r"(done) : "r"(bar_addr) : "memory");
     if (__syncthreads_or(!done)) {                             // uniform: nobody touches the tile
         if (threadIdx.x == 0) atomicAdd(&g_wait_expired, 1ull);
-        return;
+        return false;
     }
-    if (wraps) {                                               // the part after the wrap, by bytes
-        for (uint32_t left = wraps; left != 0; left &= left - 1u) {
+    if (rb.wraps) {                                            // the part after the wrap, by bytes
+        for (uint32_t left = rb.wraps; left != 0; left &= left - 1u) {
             const int k = __ffs(left) - 1;
-            uint32_t start = r0 + (rotate ? tab.s[k] : 0u);
+            uint32_t start = r0 + (rotate ? skip(k) : 0u);
             if (start >= p) start -= p;
             const uint32_t run = p - start;                    // < n for these rounds
-            const uint8_t *src_row = reinterpret_cast<const uint8_t *>(recv_t) + (uint64_t)k * t_stride;
-            for (uint32_t j = run + threadIdx.x; j < n; j += kTrThreads)
-                rounds[k * kTrPitch + lead[k] + j] = src_row[j - run];
+            const uint8_t *src_row = reinterpret_cast<const uint8_t *>(tbl) + (uint64_t)k * stride;
+            for (uint32_t j = run + threadIdx.x; j < n; j += blockDim.x)
+                rb.rounds[k * kTrPitch + rb.lead[k] + j] = src_row[j - run];
         }
         __syncthreads();
     }
-    // W[k]: the entries of round k of this thread's four ranks
-    uint32_t W[kQ];
+    return true;
+}
+
+// W[k]: the entries of round k of the ranks 4j..4j+3 of the tile.
+template <int kQ, class Buffer>
+__device__ __forceinline__ void load_four_ranks(const Buffer &rb, uint32_t j, uint32_t (&W)[kQ])
+{
 #pragma unroll
     for (int k = 0; k < kQ; ++k) {
-        const uint32_t off = (uint32_t)k * kTrPitch + lead[k] + 4u * threadIdx.x;
-        const uint32_t *word = reinterpret_cast<const uint32_t *>(rounds + (off & ~3u));
+        const uint32_t off = (uint32_t)k * kTrPitch + rb.lead[k] + 4u * j;
+        const uint32_t *word = reinterpret_cast<const uint32_t *>(rb.rounds + (off & ~3u));
         W[k] = __funnelshift_r(word[0], word[1], (off & 3u) * 8u);
     }
+}
+
+// Word m of the 4q bytes of four consecutive rank-major rows: byte e is rank e / q, round e % q.
+template <int kQ>
+__device__ __forceinline__ uint32_t row_word(const uint32_t (&W)[kQ], int m)
+{
+    const int e = 4 * m;
+    const uint32_t lo = __byte_perm(W[e % kQ], W[(e + 1) % kQ],
+                                    (uint32_t)(e / kQ) | (uint32_t)(4 + (e + 1) / kQ) << 4);
+    const uint32_t hi = __byte_perm(W[(e + 2) % kQ], W[(e + 3) % kQ],
+                                    (uint32_t)((e + 2) / kQ) | (uint32_t)(4 + (e + 3) / kQ) << 4);
+    return __byte_perm(lo, hi, 0x5410u);
+}
+
+// Single p: recv_t holds all p ranks of every round (rows 16-byte aligned); the CTA's tile is
+// ranks r0..r0+n-1 of the range r_begin..r_begin+count-1.  rotate: send rows; otherwise the
+// receive rows themselves.  The rows are written over the round buffer (after a barrier) and
+// leave as one bulk store: 64 threads and 6 KB (q = 21) per 256 ranks, so the whole grid of a
+// million-rank table is resident at once, and the many small CTAs per SM overlap one another's
+// copies.
+template <int kQ>
+__global__ void __launch_bounds__(kTrThreads)
+send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restrict__ recv_t,
+                      uint64_t t_stride, int8_t *send_out, uint32_t r_begin, uint32_t count,
+                      bool rotate)
+{
+    __shared__ RoundBuffer<kQ> rb;
+    const uint32_t first = blockIdx.x * kTile;
+    const uint32_t n = count - first < (uint32_t)kTile ? count - first : (uint32_t)kTile;
+    if (!load_rounds(TableSkips{tab}, tab.p, kQ, recv_t, t_stride, r_begin + first, n, rotate, rb))
+        return;
+    uint32_t W[kQ];
+    load_four_ranks(rb, threadIdx.x, W);
     __syncthreads();                                       // everyone has read: the rows take the buffer over
-    uint8_t *stage = rounds;
-    // output word m holds bytes 4m..4m+3 of the four rows: byte e is rank e / q, round e % q
-    uint32_t *rows = reinterpret_cast<uint32_t *>(stage) + threadIdx.x * kQ;
+    uint8_t *stage = rb.rounds;
+    uint32_t *rows = reinterpret_cast<uint32_t *>(stage) + threadIdx.x * kQ;   // 4q bytes start at a multiple of 4
 #pragma unroll
-    for (int m = 0; m < kQ; ++m) {
-        const int e = 4 * m;
-        const uint32_t lo = __byte_perm(W[e % kQ], W[(e + 1) % kQ],
-                                        (uint32_t)(e / kQ) | (uint32_t)(4 + (e + 1) / kQ) << 4);
-        const uint32_t hi = __byte_perm(W[(e + 2) % kQ], W[(e + 3) % kQ],
-                                        (uint32_t)((e + 2) / kQ) | (uint32_t)(4 + (e + 3) / kQ) << 4);
-        rows[m] = __byte_perm(lo, hi, 0x5410u);
-    }
+    for (int m = 0; m < kQ; ++m) rows[m] = row_word<kQ>(W, m);
     const uint32_t len = n * (uint32_t)kQ;                 // starts at byte first * q: 16-byte aligned
     if ((len & 15u) == 0) {
         flush_span_bulk(stage, len, send_out, (uint64_t)first * (uint64_t)kQ);
@@ -902,6 +867,50 @@ send_transpose_kernel(const __grid_constant__ PTable tab, const int8_t *__restri
         flush_span(stage, 0, len, send_out, (uint64_t)first * (uint64_t)kQ);
     }
 }
+
+// Batch: the same for a tile whose rows start at any byte.  `out` is where the tile's first row
+// starts in the staging buffer; with sh = its address mod 4, word m of a thread's rows lies sh
+// bytes into an aligned word, so consecutive words are funnel-shifted together and the up to
+// three bytes at either end go out one by one.
+using BatchRoundBuffer = RoundBuffer<BCS_MAX_Q>;
+
+template <int kQ>
+__device__ __forceinline__ void gather_rows_unaligned(const BatchRoundBuffer &rb, uint8_t *out)
+{
+    uint32_t W[kQ];
+    load_four_ranks(rb, threadIdx.x, W);
+    uint8_t *mine = out + 4u * threadIdx.x * kQ;
+    const uint32_t sh = (uint32_t)(__cvta_generic_to_shared(mine) & 3u);
+    uint32_t *words = reinterpret_cast<uint32_t *>(mine - sh);
+    uint32_t prev = 0;
+#pragma unroll
+    for (int m = 0; m < kQ; ++m) {
+        const uint32_t cur = row_word<kQ>(W, m);
+        if (m == 0 && sh != 0) {
+            for (uint32_t e = 0; e + sh < 4u; ++e) mine[e] = (uint8_t)(cur >> (8u * e));
+        } else {
+            words[m] = __funnelshift_l(prev, cur, 8u * sh);
+        }
+        prev = cur;
+    }
+    for (uint32_t e = 0; e < sh; ++e)                         // the last sh bytes
+        mine[4u * kQ - sh + e] = (uint8_t)(prev >> (8u * (4u - sh + e)));
+}
+
+template <int kQ>
+struct GatherDispatch {
+    static __device__ __forceinline__ void run(int q, const BatchRoundBuffer &rb, uint8_t *out)
+    {
+        if (q == kQ)
+            gather_rows_unaligned<kQ>(rb, out);
+        else
+            GatherDispatch<kQ - 1>::run(q, rb, out);
+    }
+};
+template <>
+struct GatherDispatch<0> {
+    static __device__ __forceinline__ void run(int, const BatchRoundBuffer &, uint8_t *) {}
+};
 
 template <int kQ>
 struct TransposeLauncher {
@@ -933,11 +942,11 @@ inline void launch_transpose(const PTable &tab, const int8_t *recv_t, uint64_t t
 }
 
 // Batch: a CTA inside one p transposes; a CTA that straddles several p gathers byte by byte.
-__global__ void __launch_bounds__(kTile)
+__global__ void __launch_bounds__(kTile, 6)
 send_batch_kernel(BatchArgs ba, const int8_t *__restrict__ recv_t, int8_t *send_out)
 {
     __shared__ TileShared sh;
-    __shared__ TransposeShared ts;
+    __shared__ BatchRoundBuffer rb;
     PTable unused;
     RankCtx c = resolve_rank<true>(sh, unused, 0, 0, ba);
     const uint32_t shift = (uint32_t)(sh.span_begin & 15u);
@@ -945,9 +954,12 @@ send_batch_kernel(BatchArgs ba, const int8_t *__restrict__ recv_t, int8_t *send_
         const uint64_t g0 = (uint64_t)blockIdx.x * kTile;
         const uint32_t n = (uint32_t)(ba.total_ranks - g0 < (uint64_t)kTile ? ba.total_ranks - g0
                                                                              : (uint64_t)kTile);
-        if (c.q > 0)
-            transpose_tile<0>(SharedSkips{sh.skips[0]}, c.p, c.q, recv_t + ba.entry_off[c.pj],
-                           (uint64_t)c.p, (uint32_t)(g0 - c.rank0), n, true, ts, sh.stage + shift);
+        if (c.q > 0) {
+            if (!load_rounds(SharedSkips{sh.skips[0]}, c.p, c.q, recv_t + ba.entry_off[c.pj],
+                             (uint64_t)c.p, (uint32_t)(g0 - c.rank0), n, true, rb))
+                return;
+            if (threadIdx.x < kTrThreads) GatherDispatch<BCS_MAX_Q>::run(c.q, rb, sh.stage + shift);
+        }
     } else if (c.valid) {
         uint8_t *row = sh.stage + shift + (c.entry - sh.span_begin);
         const int8_t *tbl = recv_t + ba.entry_off[c.pj];
