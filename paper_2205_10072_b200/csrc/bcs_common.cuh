@@ -86,7 +86,9 @@ struct TileShared {
     uint32_t skips[kCachedRows][kRow];
     uint32_t full[kCachedRows][kRow];
     uint64_t span_begin, span_end;
+    uint64_t rank0_first, entry0_first;   // batch: rank and entry offset of the CTA's first p
     uint32_t j_first, j_last;
+    uint32_t p_first;
     __align__(16) uint8_t stage[kStageBytes];
 };
 
@@ -217,12 +219,15 @@ __device__ __forceinline__ RankCtx resolve_rank(TileShared &sh, const PTable &ta
         const uint32_t jf = find_segment_warp(ba.rank_off, ba.num_p, g0);
         const uint32_t jl = ba.rank_off[jf + 1] >= g1 ? jf : find_segment_warp(ba.rank_off, ba.num_p, g1 - 1);
         if (threadIdx.x == 0) {
-        sh.j_first = jf;
-        sh.j_last = jl;
-        int qf = ceil_log2_fast(ba.p_list[jf]);
-        int ql = ceil_log2_fast(ba.p_list[jl]);
-        sh.span_begin = ba.entry_off[jf] + (g0 - ba.rank_off[jf]) * (uint64_t)qf;
-        sh.span_end = ba.entry_off[jl] + (g1 - ba.rank_off[jl]) * (uint64_t)ql;
+            sh.j_first = jf;
+            sh.j_last = jl;
+            sh.p_first = ba.p_list[jf];
+            sh.rank0_first = ba.rank_off[jf];
+            sh.entry0_first = ba.entry_off[jf];
+            const int qf = ceil_log2_fast(sh.p_first);
+            const int ql = ceil_log2_fast(ba.p_list[jl]);
+            sh.span_begin = sh.entry0_first + (g0 - sh.rank0_first) * (uint64_t)qf;
+            sh.span_end = ba.entry_off[jl] + (g1 - ba.rank_off[jl]) * (uint64_t)ql;
         }
     }
     __syncthreads();
@@ -239,6 +244,17 @@ __device__ __forceinline__ RankCtx resolve_rank(TileShared &sh, const PTable &ta
     __syncthreads();
     const uint64_t g = g0 + threadIdx.x;
     c.valid = g < g1;
+    if (jf == jl) {                                  // the whole CTA inside one p: no per-thread lookups
+        c.s = sh.skips[0];
+        c.full = sh.full[0];
+        c.pj = jf;
+        c.p = sh.p_first;
+        c.q = ceil_log2_fast(c.p);
+        c.rank0 = sh.rank0_first;
+        c.r = (uint32_t)(g - c.rank0);
+        c.entry = sh.entry0_first + (uint64_t)c.r * (uint64_t)c.q;
+        return c;
+    }
     const uint32_t j = c.valid ? find_segment(ba.rank_off, jf, jl, g) : jf;
     const bool cached = j - jf < (uint32_t)kCachedRows;
     c.s = cached ? sh.skips[j - jf] : ba.skips_tab + (size_t)j * kRow;

@@ -658,7 +658,7 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, const __grid_constant
 // are large) runs the warp-cooperative tile with that p's table rows from shared memory; a CTA
 // that straddles several p, or a small p, runs the per-lane search.
 template <bool kColOut>
-__global__ void __launch_bounds__(kTile)
+__global__ void __launch_bounds__(kTile, 6)
 recv_codes_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t *recv_out,
                         int8_t *recv_t)
 {
