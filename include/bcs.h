@@ -220,7 +220,7 @@ bcs_status bcs_circulant_rounds(uint32_t p, uint64_t r_begin, uint64_t r_end, in
  * omits it and would then start with block x instead of block 0.  The to- and from-processors
  * of the round are those of bcs_expand.
  *   recv, send: device int8, the FULL [p][q] tables, 16-byte aligned; pack_out, unpack_out:
- *   device int32, (n-1+q) * p entries each, 4-byte aligned, either may be NULL.  n-1+q <= 65535 * 64. */
+ *   device int32, (n-1+q) * p entries each, 4-byte aligned, either may be NULL. */
 bcs_status bcs_allgather_tables(uint32_t p, uint32_t n, uint32_t r,
                                 const int8_t *recv, const int8_t *send,
                                 int32_t *pack_out, int32_t *unpack_out, void *cuda_stream);

@@ -7,56 +7,75 @@ namespace {
 
 // ---------------------------------------------------------------- Algorithm 6: round tables
 constexpr int kExpandThreads = 256;
-constexpr int kExpandRanks = 8;   // ranks per CTA
+constexpr uint32_t kExpandRecords = 8192;      // records (128 KB of output) that a CTA aims for
+constexpr uint32_t kExpandSharedBytes = 48 * 1024;
 
+// A CTA takes `ranks_per_cta` consecutive ranks.  Their records are one contiguous stretch of
+// the output, which the threads walk as a flat stream, thread t at the records t - shift,
+// t - shift + 256, ...: `shift` (0..7) is chosen so that a warp's 32 x 16 bytes are four whole
+// 128-byte lines of memory wherever the stretch starts (stores that cut lines or 32-byte sectors
+// cost up to a fifth of the write bandwidth), and short rows (few rounds) fill the threads as
+// well as long ones.  Rank, round, entry and phase of a thread's record are kept incrementally.
 __global__ void __launch_bounds__(kExpandThreads)
-expand_kernel(PTable tab, uint32_t n, uint64_t r_begin, uint64_t r_end,
+expand_kernel(PTable tab, uint32_t n, uint64_t r_begin, uint64_t r_end, uint32_t ranks_per_cta,
               const int8_t *__restrict__ recv, const int8_t *__restrict__ send,
               int4 *__restrict__ table_out)
 {
     // per rank of the CTA and per round k of a phase: {send entry - x, recv entry - x, to, from}.
     // Algorithm 6 adds q to an entry after each use and starts entries k < x at +q because
     // their first use is in the second phase; both are covered by adding q * floor(i / q).
-    __shared__ int4 base[kExpandRanks][32];
-    const int q = tab.q;
+    extern __shared__ int4 base[];             // [ranks_per_cta][q]
+    const uint32_t q = (uint32_t)tab.q;
     const uint32_t p = tab.p;
-    const uint32_t rounds = n - 1u + (uint32_t)q;
-    const int x = (int)(((uint32_t)q - rounds % (uint32_t)q) % (uint32_t)q);
-    const uint64_t j0 = (uint64_t)blockIdx.x * kExpandRanks;
+    const uint32_t rounds = n - 1u + q;
+    const uint32_t x = (q - rounds % q) % q;
+    const uint64_t j0 = (uint64_t)blockIdx.x * ranks_per_cta;
     const uint64_t count = r_end - r_begin;
+    const uint32_t ranks = (uint32_t)(count - j0 < (uint64_t)ranks_per_cta ? count - j0 : (uint64_t)ranks_per_cta);
     {
-        const int g = threadIdx.x / 32, k = threadIdx.x % 32;
-        if (g < kExpandRanks && k < q && j0 + g < count) {
-            const uint64_t row = (j0 + g) * (uint64_t)q;
+        const int8_t *srow = send + j0 * q, *rrow = recv + j0 * q;     // the CTA's rows are contiguous
+        for (uint32_t e = threadIdx.x; e < ranks * q; e += kExpandThreads) {
+            const uint32_t g = e / q, k = e - g * q;
             const uint32_t r = (uint32_t)(r_begin + j0 + g);
             const uint32_t sk = tab.s[k];
-            const int adj = -x;
             uint32_t to = r + sk;
             if (to >= p) to -= p;
-            uint32_t from = r >= sk ? r - sk : r + p - sk;
-            base[g][k] = make_int4((int)send[row + k] + adj, (int)recv[row + k] + adj, (int)to,
-                                   (int)from);
+            const uint32_t from = r >= sk ? r - sk : r + p - sk;
+            base[e] = make_int4((int)srow[e] - (int)x, (int)rrow[e] - (int)x, (int)to, (int)from);
         }
     }
     __syncthreads();
-    // round j uses i = j + x: entry k = i mod q of phase i / q.
-    const uint32_t step_k = kExpandThreads % (uint32_t)q, step_ph = kExpandThreads / (uint32_t)q;
+    const uint32_t total = ranks * rounds;                           // records of the CTA (ranks > 1 only when rounds < kExpandRecords)
+    const uint64_t first = j0 * rounds;                              // index of its first record
+    int4 *out = table_out + first;
+    const uint32_t shift = (uint32_t)((reinterpret_cast<uintptr_t>(table_out) >> 4) + first) & 7u;
+    uint32_t e = threadIdx.x >= shift ? threadIdx.x - shift : threadIdx.x + kExpandThreads - shift;
+    if (e >= total) return;
+    // record e is round j of the CTA's rank number gq / q; round j uses i = j + x: entry
+    // k = i mod q of phase floor(i / q), whose block numbers are the entries plus add = q * floor(i / q)
+    uint32_t j = e % rounds, gq = e / rounds * q;
+    int k = (int)((j + x) % q), add = (int)((j + x) / q * q);
+    const int step_k = kExpandThreads % q, step_add = kExpandThreads / q * q;
+    const int row_k = (int)(rounds % q), row_add = (int)(rounds / q * q);   // what a whole row adds to k and add
     const int last = (int)n - 1;
-    for (int g = 0; g < kExpandRanks; ++g) {
-        if (j0 + g >= count) break;
-        int4 *out = table_out + (j0 + g) * (uint64_t)rounds;
-        uint32_t i = threadIdx.x + (uint32_t)x;
-        uint32_t k = i % (uint32_t)q, ph = i / (uint32_t)q;
-        for (uint32_t j = threadIdx.x; j < rounds; j += kExpandThreads) {
-            int4 rec = base[g][k];
-            const int add = (int)(ph * (uint32_t)q);
-            int sb = rec.x + add, rb = rec.y + add;
-            sb = sb < 0 ? -1 : (sb > last ? last : sb);
-            rb = rb < 0 ? -1 : (rb > last ? last : rb);
-            __stcs(out + j, make_int4(sb, rb, rec.z, rec.w));
-            k += step_k;
-            ph += step_ph;
-            if (k >= (uint32_t)q) { k -= (uint32_t)q; ++ph; }
+    for (;;) {
+        const int4 rec = base[gq + (uint32_t)k];
+        int sb = rec.x + add, rb = rec.y + add;
+        sb = sb < 0 ? -1 : (sb > last ? last : sb);
+        rb = rb < 0 ? -1 : (rb > last ? last : rb);
+        __stcs(out + e, make_int4(sb, rb, rec.z, rec.w));
+        e += kExpandThreads;
+        if (e >= total) break;
+        j += kExpandThreads;
+        k += step_k;
+        add += step_add;
+        if (k >= (int)q) { k -= (int)q; add += (int)q; }
+        while (j >= rounds) {                                        // on to the next rank: i falls by `rounds`
+            j -= rounds;
+            gq += q;
+            k -= row_k;
+            add -= row_add;
+            if (k < 0) { k += (int)q; add -= (int)q; }
         }
     }
 }
@@ -112,9 +131,16 @@ bcs_status bcs_expand(uint32_t p, uint32_t n, uint64_t r_begin, uint64_t r_end,
     if (count == 0 || tab.q == 0) return BCS_OK;
     if (recv == nullptr || send == nullptr || table_out == nullptr) return BCS_ERR_ARG;
     if (!aligned16(table_out)) return BCS_ERR_ALIGN;
-    const unsigned blocks = (unsigned)((count + kExpandRanks - 1) / kExpandRanks);
-    expand_kernel<<<blocks, kExpandThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-        tab, n, r_begin, r_end, recv, send, reinterpret_cast<int4 *>(table_out));
+    // ranks per CTA: about kExpandRecords records, as far as the per-rank constants fit in shared memory
+    const uint32_t rounds = n - 1u + (uint32_t)tab.q;
+    uint32_t per_cta = (kExpandRecords + rounds - 1) / rounds;
+    const uint32_t fit = kExpandSharedBytes / (16u * (uint32_t)tab.q);
+    if (per_cta > fit) per_cta = fit;
+    const uint64_t blocks = (count + per_cta - 1) / per_cta;
+    if (blocks > 0x7fffffffull) return BCS_ERR_UNSUPPORTED;
+    expand_kernel<<<(unsigned)blocks, kExpandThreads, (size_t)per_cta * tab.q * 16u,
+                    static_cast<cudaStream_t>(cuda_stream)>>>(
+        tab, n, r_begin, r_end, per_cta, recv, send, reinterpret_cast<int4 *>(table_out));
     return launch_status();
 }
 
