@@ -465,8 +465,9 @@ def test_circulant_round_tables_match_oracle(bcs):
 def test_checksum_matches_oracle(bcs):
     rng = np.random.default_rng(11)
     out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    # (the word index passes 2^32, where the weights' high half changes, in the 2^34 - 40 case)
     for nbytes, first in ((0, 0), (1, 0), (3, 4), (4, 8), (1000, 16), (1003, 2**34 + 8),
-                          (5 * 2**20 + 1, 2**36)):
+                          (200003, 2**34 - 40), (5 * 2**20 + 1, 2**36)):
         host = rng.integers(-31, 31, nbytes).astype(np.int8)
         dev = torch.from_numpy(host).cuda() if nbytes else torch.zeros(4, dtype=torch.int8,
                                                                        device="cuda")
