@@ -654,6 +654,357 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, const __grid_constant
 }
 
 
+// Single p, p >= 64, four consecutive ranks per thread.  The work of a round that does not depend
+// on the rank -- the address of the codes at the window's lower end, the store into the
+// round-major copy -- is done once for four ranks: their four codes are four words at one
+// address, their four entries one aligned 32-bit word of the copy.  A thread whose four ranks
+// lie in the same homerange past the table rounds (all but a few dozen quads of a p) runs the
+// rounds for the four together, with the wrap decided per quad: before the home round h every
+// window bound is r - skip, after it r + p - skip.  A tile that holds any other quad (around a
+// skip, next to the root, at the end of the range: a few dozen tiles of a p) runs the general
+// code, home round and wrap tested per rank, for all its quads.
+//
+// The run table of the tile (see recv_warp_tile) is kept as four sub-tables by position mod 4:
+// entry x (x = -64 .. tile-1, counted from the tile's first rank) is word
+// ((x + 64) mod 4) * kQuadSub + (x + 64) / 4 of its level, so that the threads of a warp, whose
+// ranks are four apart, read consecutive words whatever the distance of the window.
+#ifndef QUAD_MIN_BLOCKS
+#define QUAD_MIN_BLOCKS 8
+#endif
+constexpr int kQuadThreads = 128;
+constexpr int kQuadTile = 4 * kQuadThreads;                 // ranks per CTA
+constexpr int kQuadSub = kQuadThreads + kRunBack / 4;       // words per sub-table
+constexpr int kQuadLevelWords = 4 * kQuadSub;               // words per level
+constexpr int kQuadTableRounds = 6;                         // at most six rounds have skips[i+1] <= 33
+
+struct QuadConsts {
+    // Table round i, word w (0, 1: the two runs that cover the first window; 2, 3: the second
+    // window, or the first again), rank j of the quad: byte offset of that word from the thread's
+    // word of sub-table 0, level 0.
+    int32_t word[kQuadTableRounds][4][4];
+    uint32_t len2[kRow];     // length of the second window of round i, or 0
+    int table_rounds;        // rounds 0 .. table_rounds-1 are decided from the run table
+    // tiles that (may) hold a quad for the general code: those of the ranks skips[k], the first
+    // and the last of the range; distinct, n_special <= 32 (missing one costs time, not correctness)
+    uint32_t special[kRow];
+    int n_special;
+};
+
+inline QuadConsts make_quad_consts(const PTable &tab, uint64_t r_begin, uint64_t r_end)
+{
+    QuadConsts qc = {};
+    {
+        const uint64_t count = r_end - r_begin;
+        auto add = [&](uint64_t tile) {
+            for (int m = 0; m < qc.n_special; ++m)
+                if (qc.special[m] == tile) return;
+            if (qc.n_special < kRow) qc.special[qc.n_special++] = (uint32_t)tile;
+        };
+        if (count) {
+            add(0);
+            for (int k = 1; k < tab.q; ++k)
+                if (tab.s[k] >= r_begin && tab.s[k] < r_end) add((tab.s[k] - r_begin) / kQuadTile);
+            add((count - 1) / kQuadTile);
+        }
+    }
+    RoundConsts rc = {};
+    for (int i = 0; i < tab.q; ++i) {
+        round_consts(tab.s, i, &rc);
+        qc.len2[i] = rc.len2[i];
+    }
+    int rounds = 0;
+    while (rounds < tab.q && rounds < kQuadTableRounds && tab.s[rounds + 1] <= 33u) ++rounds;
+    qc.table_rounds = rounds;
+    for (int i = 0; i < rounds; ++i) {
+        uint32_t sum = 0;
+        for (int j = 0; j <= i; ++j) sum += tab.s[j];
+        const uint32_t lo = tab.s[i], hi = tab.s[i + 1];
+        // the len >= 1 ranks that end d ranks below: runs of 2^l ranks, l = floor(log2 len),
+        // ending d and d + len - 2^l ranks below
+        int level[4];
+        uint32_t back[4];
+        int l1 = 0;
+        while ((2u << l1) <= hi - lo) ++l1;
+        level[0] = level[1] = l1;
+        back[0] = lo;
+        back[1] = hi - (1u << l1);
+        level[2] = level[3] = l1;
+        back[2] = back[0];
+        back[3] = back[1];
+        if (qc.len2[i]) {
+            int l2 = 0;
+            while ((2u << l2) <= qc.len2[i]) ++l2;
+            level[2] = level[3] = l2;
+            back[2] = hi;
+            back[3] = sum + 1u - (1u << l2);
+        }
+        for (int w = 0; w < 4; ++w)
+            for (int j = 0; j < 4; ++j) {
+                const int rel = j - (int)back[w];            // position relative to the quad's first rank
+                const int sub = rel & 3;
+                const int quad = (rel - sub) / 4;            // exact: rel - sub is a multiple of 4
+                qc.word[i][w][j] = 4 * (level[w] * kQuadLevelWords + sub * kQuadSub + kRunBack / 4 + quad);
+            }
+    }
+    return qc;
+}
+
+template <bool kRowOut, bool kColOut>
+__global__ void __launch_bounds__(kQuadThreads, QUAD_MIN_BLOCKS)
+recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant__ QuadConsts qc,
+                       uint64_t r_begin, uint64_t r_end, const uint32_t *__restrict__ codes,
+                       int8_t *recv_out, int8_t *recv_t, uint64_t t_stride)
+{
+    __shared__ __align__(16) uint8_t stage[kQuadTile * BCS_MAX_Q];
+    __shared__ uint32_t full_sh[kRow];
+    __shared__ uint32_t runs[kRunLevels][kQuadLevelWords];
+    grid_launch_dependents();
+    const uint32_t t = threadIdx.x;
+    if (t < kRow) full_sh[t] = tab.full[t];                    // read after the first barrier
+    const uint32_t p = tab.p;
+    const int q = tab.q;
+    const uint64_t count = r_end - r_begin;
+    // The first CTAs of the grid take the tiles that run the general code (listed by the host):
+    // they last longer, so they start first; the others skip a listed tile.
+    uint64_t tile = blockIdx.x;
+    if (blockIdx.x < (uint32_t)qc.n_special) {
+        tile = qc.special[blockIdx.x];
+    } else {
+        tile -= (uint32_t)qc.n_special;
+        if (__syncthreads_or(t < (uint32_t)qc.n_special && qc.special[t] == tile)) return;
+    }
+    grid_dependency_wait();                                    // the codes are complete from here on
+    {
+    const uint64_t g0 = tile * kQuadTile;
+    const uint32_t n = (uint32_t)(count - g0 < (uint64_t)kQuadTile ? count - g0 : (uint64_t)kQuadTile);
+    // ranks of the quad mod p (defined for every thread, also past the end of the range: the
+    // table entries of such ranks are never read for a rank of the range)
+    uint32_t r[4], c[4], B[4];
+    {
+        uint64_t wrapped = r_begin + g0 + 4u * t;
+        while (wrapped >= p) wrapped -= p;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            r[j] = (uint32_t)wrapped + j;
+            if (r[j] >= p) r[j] -= p;
+            c[j] = codes[r[j]];
+            B[j] = c[j] & (0u - c[j]);                         // baseblock as a bit, 0 for the root
+            runs[0][j * kQuadSub + kRunBack / 4 + t] = B[j];
+        }
+        if (t < kRunBack / 4) {                                // the 64 ranks before the tile, mod p (p >= 64)
+            uint64_t back = r_begin + g0 + 4u * t + p - kRunBack;
+            while (back >= p) back -= p;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                uint32_t x = (uint32_t)back + j;
+                if (x >= p) x -= p;
+                const uint32_t cx = codes[x];
+                runs[0][j * kQuadSub + t] = cx & (0u - cx);
+            }
+        }
+    }
+    __syncthreads();
+    // Runs of 2 and 4 from the single bits, then runs of 8 and 16 from the runs of 4; entry x of
+    // level l is complete from x = -64 + 2^l - 1 on, and nothing before x = -41 is ever read.
+    // `slot` is the thread's word in the sub-tables: its own quad, or a quad of the ranks before the tile.
+    auto build_narrow = [&](uint32_t slot, uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3) {
+        const uint32_t m1 = runs[0][3 * kQuadSub + slot - 1];  // the three ranks before the quad
+        const uint32_t m2 = runs[0][2 * kQuadSub + slot - 1];
+        const uint32_t m3 = runs[0][1 * kQuadSub + slot - 1];
+        runs[1][0 * kQuadSub + slot] = b0 | m1;
+        runs[1][1 * kQuadSub + slot] = b1 | b0;
+        runs[1][2 * kQuadSub + slot] = b2 | b1;
+        runs[1][3 * kQuadSub + slot] = b3 | b2;
+        runs[2][0 * kQuadSub + slot] = b0 | m1 | m2 | m3;
+        runs[2][1 * kQuadSub + slot] = b1 | b0 | m1 | m2;
+        runs[2][2 * kQuadSub + slot] = b2 | b1 | b0 | m1;
+        runs[2][3 * kQuadSub + slot] = b3 | b2 | b1 | b0;
+    };
+    build_narrow(kRunBack / 4 + t, B[0], B[1], B[2], B[3]);
+    if (t >= 1u && t < kRunBack / 4)
+        build_narrow(t, runs[0][t], runs[0][kQuadSub + t], runs[0][2 * kQuadSub + t], runs[0][3 * kQuadSub + t]);
+    __syncthreads();
+    auto build_wide = [&](uint32_t slot) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t *four = &runs[2][j * kQuadSub + slot];   // runs of 4 ending at x, x-4, x-8, x-12
+            const uint32_t eight = four[0] | four[-1];
+            runs[3][j * kQuadSub + slot] = eight;
+            runs[4][j * kQuadSub + slot] = eight | four[-2] | four[-3];
+        }
+    };
+    build_wide(kRunBack / 4 + t);
+    if (t >= 4u && t < kRunBack / 4) build_wide(t);
+    __syncthreads();
+    const char *mine = reinterpret_cast<const char *>(&runs[0][t]);
+    auto word = [&](int byte_offset) { return *reinterpret_cast<const uint32_t *>(mine + byte_offset); };
+    uint8_t *row0 = stage + 4u * t * (uint32_t)q;              // rows of the quad: row0 + j * q
+    int8_t *col0 = kColOut ? recv_t + g0 + 4u * t : nullptr;   // the quad's four bytes of round 0
+    const int first_lane_round = qc.table_rounds;
+    const int h0 = 31 - __clz(c[0]);                           // -1 for the root
+    const bool together = 4u * t + 4u <= n && r[0] != 0u && r[3] == r[0] + 3u &&
+                          h0 == 31 - __clz(c[3]) && h0 >= first_lane_round;
+    // One path for the whole tile (no divergence inside a warp): the general one if any of its
+    // quads needs it -- the first tile, the last, and the tiles in which a homerange starts.
+    const bool empty = 4u * t >= n;
+    if (__syncthreads_or(!empty && !together)) {
+        // Four ranks, each with its own homerange, wrap and validity: the table rounds with the
+        // home round tested per rank, then recv_round for every rank and round.
+        int h[4], bb[4];
+        RoundState st[4];
+        bool valid[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            valid[j] = 4u * t + j < n;
+            h[j] = -1;
+            bb[j] = 0;
+            st[j].B = 0;
+            if (r[j] > 0) {
+                h[j] = 31 - __clz(c[j]);
+                bb[j] = __ffs(c[j]) - 1;
+                st[j].B = B[j];
+            }
+        }
+        uint32_t sum = 0;
+        for (int i = 0; i < first_lane_round; ++i) {
+            sum += tab.s[i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t free_blocks = ~st[j].B;
+                uint32_t U = (word(qc.word[i][0][j]) | word(qc.word[i][1][j])) & free_blocks;
+                const uint32_t U2 = (word(qc.word[i][2][j]) | word(qc.word[i][3][j])) & free_blocks;
+                if (U == 0) U = U2;
+                const int lead = __clz(U);
+                uint32_t bit = U ? 0x80000000u >> lead : 0u;
+                int entry = U ? 31 - q - lead : BCS_BAD_ENTRY;
+                if (i == h[j]) {
+                    entry = bb[j];
+                    bit = 0;
+                }
+                st[j].B |= bit;
+                if (kRowOut) row0[j * q + i] = (uint8_t)entry;
+                if (kColOut && valid[j]) col0[(uint64_t)i * t_stride + j] = (int8_t)entry;
+            }
+        }
+        if (first_lane_round < q) {
+            const uint32_t edge = tab.s[first_lane_round];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                st[j].sum = sum;
+                st[j].lo_skip = edge;
+                st[j].upper = codes[r[j] - edge + (r[j] >= edge ? 0u : p)];
+            }
+            for (int i = first_lane_round; i < q; ++i) {
+                const uint32_t hi_skip = tab.s[i + 1];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int entry = recv_round(codes, full_sh, p, q, r[j], i, h[j], bb[j], hi_skip, st[j]);
+                    if (kRowOut) row0[j * q + i] = (uint8_t)entry;
+                    if (kColOut && valid[j]) col0[(uint64_t)i * t_stride + j] = (int8_t)entry;
+                }
+            }
+        }
+    } else if (!empty) {
+        // ---- the four ranks together: same homerange h0, no home round among the table rounds
+        uint32_t *col = reinterpret_cast<uint32_t *>(col0);    // g0 + 4t and t_stride are multiples of 4
+        const uint64_t col_step = t_stride / 4;
+        int i = 0;
+#pragma unroll
+        for (int unrolled = 0; unrolled < kQuadTableRounds; ++unrolled) {
+            if (unrolled >= first_lane_round) break;           // uniform over the grid
+            i = unrolled;
+            uint32_t packed = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t free_blocks = ~B[j];
+                uint32_t U = (word(qc.word[unrolled][0][j]) | word(qc.word[unrolled][1][j])) & free_blocks;
+                const uint32_t U2 = (word(qc.word[unrolled][2][j]) | word(qc.word[unrolled][3][j])) & free_blocks;
+                if (U == 0) U = U2;
+                const int lead = __clz(U);                     // 32 when U == 0
+                B[j] |= U ? 0x80000000u >> lead : 0u;
+                const int entry = U ? 31 - q - lead : BCS_BAD_ENTRY;
+                if (kRowOut) row0[j * q + unrolled] = (uint8_t)entry;
+                packed |= ((uint32_t)entry & 0xffu) << (8 * j);
+            }
+            if (kColOut) {
+                *col = packed;
+                col += col_step;
+            }
+            i = unrolled + 1;
+        }
+        // Per-lane rounds.  upper[j]: code of r[j] - skips[i]; lower[j]: code of r[j] - skips[i+1].
+        uint32_t upper[4], lower[4];
+        auto load4 = [&](uint32_t (&dst)[4], uint32_t index) {
+            const uint32_t *src = codes + index;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) dst[j] = src[j];
+        };
+        uint8_t *out = row0 + i;
+        auto store_round = [&](const int (&entry)[4]) {
+            if (kRowOut) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) out[j * q] = (uint8_t)entry[j];
+                ++out;
+            }
+            if (kColOut) {
+                *col = ((uint32_t)entry[0] & 0xffu) | (((uint32_t)entry[1] & 0xffu) << 8) |
+                       (((uint32_t)entry[2] & 0xffu) << 16) | ((uint32_t)entry[3] << 24);
+                col += col_step;
+            }
+        };
+        // rounds i .. end-1 with the window bounds at from - skip (from = r[0] or r[0] + p)
+        auto rounds_until = [&](int end, uint32_t from) {
+            if (i >= end) return;
+            uint32_t ahead[4];
+            load4(ahead, from - tab.s[i + 1]);
+#pragma unroll 2
+            for (; i < end; ++i) {
+                const uint32_t below = from - tab.s[i + 1];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) lower[j] = ahead[j];
+                if (i + 1 < end) load4(ahead, from - tab.s[i + 2]);
+                int entry[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t diff = lower[j] ^ upper[j];
+                    int blk = 31 - __clz(diff);                // first head; -1 for an empty window
+                    if (diff == 0 || ((B[j] >> blk) & 1u)) {
+                        blk = pick_rest(codes, full_sh, p, q, below + j, lower[j], upper[j], qc.len2[i], B[j]);
+                        entry[j] = blk < 0 ? BCS_BAD_ENTRY : blk - q;
+                        if (blk >= 0) B[j] |= 1u << blk;
+                    } else {
+                        B[j] |= 1u << blk;
+                        entry[j] = blk - q;
+                    }
+                    upper[j] = lower[j];
+                }
+                store_round(entry);
+            }
+        };
+        load4(upper, r[0] - tab.s[i]);                         // i <= h0: skips[i] <= r[0]
+        rounds_until(h0, r[0]);
+        {                                                      // home round: the baseblocks themselves
+            int entry[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) entry[j] = __ffs(c[j]) - 1;
+            store_round(entry);
+            load4(upper, r[0] + p - tab.s[h0 + 1]);            // r[3] < skips[h0+1]
+            i = h0 + 1;
+        }
+        rounds_until(q, r[0] + p);
+    }
+    if (kRowOut) {
+        const uint32_t len = n * (uint32_t)q;                  // the tile's rows start at byte g0 * q: 16-byte aligned
+        if ((len & 15u) == 0) {
+            flush_span_bulk(stage, len, recv_out, g0 * (uint64_t)q);
+        } else {                                               // ragged last tile
+            __syncthreads();
+            flush_span(stage, 0, len, recv_out, g0 * (uint64_t)q);
+        }
+    }
+    }
+}
+
 // Batch: a CTA whose 256 flattened ranks all belong to one p >= 64 (nearly all CTAs when the p
 // are large) runs the warp-cooperative tile with that p's table rows from shared memory; a CTA
 // that straddles several p, or a small p, runs the per-lane search.
@@ -1036,24 +1387,25 @@ bcs_status bcs_build(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_
         launch_codes(tab, ws.codes, stream);
         if ((st = launch_status()) != BCS_OK) return st;
         const bool warp_rounds = p >= 64;      // the table kernel needs 64 distinct ranks back
-        const RoundConsts rc = make_round_consts(tab);
+        const QuadConsts rc = make_quad_consts(tab, r_begin, r_end);
+        const unsigned qblocks = (unsigned)((count + kQuadTile - 1) / kQuadTile) + (unsigned)rc.n_special;
         if (recv_out != nullptr && send_out != nullptr) {
             if (warp_rounds)
-                launch_dependent(true, recv_codes_warp_kernel<true, true>, blocks, kTile, stream, tab, rc,
+                launch_dependent(true, recv_codes_quad_kernel<true, true>, qblocks, kQuadThreads, stream, tab, rc,
                                  r_begin, r_end, ws.codes, recv_out, ws.recv_t, ws.t_stride);
             else
                 recv_codes_kernel<true, true><<<blocks, kTile, 0, stream>>>(
                     tab, r_begin, r_end, ws.codes, recv_out, ws.recv_t, ws.t_stride);
         } else if (recv_out != nullptr) {
             if (warp_rounds)
-                launch_dependent(true, recv_codes_warp_kernel<true, false>, blocks, kTile, stream, tab, rc,
+                launch_dependent(true, recv_codes_quad_kernel<true, false>, qblocks, kQuadThreads, stream, tab, rc,
                                  r_begin, r_end, ws.codes, recv_out, nullptr, 0);
             else
                 recv_codes_kernel<true, false><<<blocks, kTile, 0, stream>>>(
                     tab, r_begin, r_end, ws.codes, recv_out, nullptr, 0);
         } else {
             if (warp_rounds)
-                launch_dependent(true, recv_codes_warp_kernel<false, true>, blocks, kTile, stream, tab, rc,
+                launch_dependent(true, recv_codes_quad_kernel<false, true>, qblocks, kQuadThreads, stream, tab, rc,
                                  r_begin, r_end, ws.codes, nullptr, ws.recv_t, ws.t_stride);
             else
                 recv_codes_kernel<false, true><<<blocks, kTile, 0, stream>>>(
@@ -1106,11 +1458,12 @@ bcs_status bcs_prepare(uint32_t p, void *workspace, size_t workspace_bytes, void
     const unsigned blocks = (unsigned)((p + kTile - 1) / kTile);
     launch_codes(tab, codes, stream);
     if ((st = launch_status()) != BCS_OK) return st;
-    if (p >= 64)
-        launch_dependent(true, recv_codes_warp_kernel<false, true>, blocks, kTile, stream, tab,
-                         make_round_consts(tab),
+    if (p >= 64) {
+        const QuadConsts qc = make_quad_consts(tab, 0, p);
+        launch_dependent(true, recv_codes_quad_kernel<false, true>,
+                         (p + kQuadTile - 1) / kQuadTile + (unsigned)qc.n_special, kQuadThreads, stream, tab, qc,
                          (uint64_t)0, (uint64_t)p, codes, nullptr, recv_t, t_stride);
-    else
+    } else
         recv_codes_kernel<false, true><<<blocks, kTile, 0, stream>>>(tab, 0, p, codes, nullptr,
                                                                      recv_t, t_stride);
     return launch_status();
