@@ -668,14 +668,19 @@ recv_codes_warp_kernel(const __grid_constant__ PTable tab, const __grid_constant
 // entry x (x = -64 .. tile-1, counted from the tile's first rank) is word
 // ((x + 64) mod 4) * kQuadSub + (x + 64) / 4 of its level, so that the threads of a warp, whose
 // ranks are four apart, read consecutive words whatever the distance of the window.
-#ifndef QUAD_MIN_BLOCKS
-#define QUAD_MIN_BLOCKS 8
-#endif
 constexpr int kQuadThreads = 128;
 constexpr int kQuadTile = 4 * kQuadThreads;                 // ranks per CTA
 constexpr int kQuadSub = kQuadThreads + kRunBack / 4;       // words per sub-table
 constexpr int kQuadLevelWords = 4 * kQuadSub;               // words per level
 constexpr int kQuadTableRounds = 6;                         // at most six rounds have skips[i+1] <= 33
+
+// 1 << k for k = 0..31, 0 for any other k (the hardware shift clamps its count).
+__device__ __forceinline__ uint32_t bit_or_none(int k)
+{
+    uint32_t bit;
+    asm("shl.b32 %0, 1, %1;" : "=r"(bit) : "r"(k));
+    return bit;
+}
 
 struct QuadConsts {
     // Table round i, word w (0, 1: the two runs that cover the first window; 2, 3: the second
@@ -750,7 +755,7 @@ inline QuadConsts make_quad_consts(const PTable &tab, uint64_t r_begin, uint64_t
 }
 
 template <bool kRowOut, bool kColOut>
-__global__ void __launch_bounds__(kQuadThreads, QUAD_MIN_BLOCKS)
+__global__ void __launch_bounds__(kQuadThreads, 8)
 recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant__ QuadConsts qc,
                        uint64_t r_begin, uint64_t r_end, const uint32_t *__restrict__ codes,
                        int8_t *recv_out, int8_t *recv_t, uint64_t t_stride)
@@ -963,19 +968,32 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
 #pragma unroll
                 for (int j = 0; j < 4; ++j) lower[j] = ahead[j];
                 if (i + 1 < end) load4(ahead, from - tab.s[i + 2]);
-                int entry[4];
+                // The first head of each of the four windows, then ONE test whether any of them is
+                // already taken (or its window empty): the four chains stay free of branches.
+                int blk[4];
+                bool taken = false;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const uint32_t diff = lower[j] ^ upper[j];
-                    int blk = 31 - __clz(diff);                // first head; -1 for an empty window
-                    if (diff == 0 || ((B[j] >> blk) & 1u)) {
-                        blk = pick_rest(codes, full_sh, p, q, below + j, lower[j], upper[j], qc.len2[i], B[j]);
-                        entry[j] = blk < 0 ? BCS_BAD_ENTRY : blk - q;
-                        if (blk >= 0) B[j] |= 1u << blk;
-                    } else {
-                        B[j] |= 1u << blk;
-                        entry[j] = blk - q;
+                    blk[j] = 31 - __clz(diff);                 // -1 for an empty window
+                    taken |= diff == 0 || ((B[j] >> blk[j]) & 1u);
+                }
+                if (taken) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t diff = lower[j] ^ upper[j];
+                        if (diff == 0 || ((B[j] >> blk[j]) & 1u)) {
+                            const int b = pick_rest(codes, full_sh, p, q, below + j, lower[j], upper[j],
+                                                    qc.len2[i], B[j]);
+                            blk[j] = b >= 0 ? b : BCS_BAD_ENTRY + q;   // entry BCS_BAD_ENTRY, no bit
+                        }
                     }
+                }
+                int entry[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    B[j] |= bit_or_none(blk[j]);
+                    entry[j] = blk[j] - q;
                     upper[j] = lower[j];
                 }
                 store_round(entry);
