@@ -983,8 +983,20 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
                     for (int j = 0; j < 4; ++j) {
                         const uint32_t diff = lower[j] ^ upper[j];
                         if (diff == 0 || ((B[j] >> blk[j]) & 1u)) {
-                            const int b = pick_rest(codes, full_sh, p, q, below + j, lower[j], upper[j],
-                                                    qc.len2[i], B[j]);
+                            // The usual case, decided here: the first head is taken and the search
+                            // of pick_block ends at its second step, with a new block in the run
+                            // of low blocks behind the head.  Everything else: the full search.
+                            const uint32_t below_head = (1u << (blk[j] & 31)) - 1u;
+                            const uint32_t rest = upper[j] & below_head;
+                            const uint32_t low = rest ? (2u << (31 - __clz(rest))) - 1u : 0u;
+                            const uint32_t diff2 = (lower[j] & below_head) ^ full_sh[blk[j] & 31];
+                            const uint32_t fresh = low & ~B[j];
+                            int b;
+                            if (diff != 0 && fresh != 0 && (diff2 == 0 || (0x80000000u >> __clz(diff2)) <= low))
+                                b = 31 - __clz(fresh);
+                            else
+                                b = pick_rest(codes, full_sh, p, q, below + j, lower[j], upper[j],
+                                              qc.len2[i], B[j]);
                             blk[j] = b >= 0 ? b : BCS_BAD_ENTRY + q;   // entry BCS_BAD_ENTRY, no bit
                         }
                     }
