@@ -5,7 +5,7 @@
 // Two constructions, bit-identical in their results:
 //
 //  * workspace path.  codes_single_kernel / codes_batch_kernel write the skip code (bcs_common.cuh) of every rank x of a p
-//    once.  The receive kernels (recv_codes_warp_kernel for one p >= 64, recv_codes_batch_kernel
+//    once.  The receive kernels (recv_codes_quad_kernel for one p >= 64, recv_codes_batch_kernel
 //    for a batch, recv_codes_kernel for tiny p) then read, per rank r and round i, the codes of
 //    the two ranks that bound the window of Algorithm 4 (r - skips[i+1], r - skips[i];
 //    consecutive threads read consecutive words) and find the largest new block of the window
@@ -398,7 +398,8 @@ recv_codes_kernel(PTable tab, uint64_t r_begin, uint64_t r_end,
     }
 }
 
-// Single p, p >= 64: the same rows with the first rounds decided from a table of the tile.  The
+// A tile of 256 ranks of one p >= 64, one rank per thread (the batch kernel's tiles; a single p
+// uses recv_codes_quad_kernel below): the first rounds are decided from a table of the tile.  The
 // windows of the rounds with skips[i+1] <= 33 (at most six rounds, i <= 5) reach only a few
 // ranks back: the first window ends skips[i+1] - 1 ranks below r, the second at
 // sum_{j<=i} skips[j] <= skips[i+1] + i <= 38 (every halving rounds up by at most one), and a run
@@ -412,21 +413,11 @@ recv_codes_kernel(PTable tab, uint64_t r_begin, uint64_t r_end,
 // only (RoundConsts).  These are the rounds in which
 // neighbouring ranks disagree about which path of the code search they take; the later rounds
 // run the code search per lane.
-// Where the skips of the tile's p are read from: the kernel parameter (single p: immediate /
-// constant-bank operands) or a table row in shared memory (batch).
+// Where the skips of the tile's p are read from: a table row in shared memory.
 struct RoundConsts;
 struct RunTable;
-struct ParamSkips {
-    const PTable &tab;
-    const RoundConsts &rc;
-    static constexpr bool kHostConsts = true;          // per-round constants come with the launch
-    __device__ __forceinline__ uint32_t operator()(int k) const { return tab.s[k]; }
-    __device__ __forceinline__ int4 window(int i, const RunTable &) const;
-    __device__ __forceinline__ uint32_t len2(int i, const RunTable &) const;
-};
 struct SharedSkips {
     const uint32_t *s;
-    static constexpr bool kHostConsts = false;         // the CTA computes them into its RunTable
     __device__ __forceinline__ uint32_t operator()(int k) const { return s[k]; }
     __device__ __forceinline__ int4 window(int i, const RunTable &runs) const;
     __device__ __forceinline__ uint32_t len2(int i, const RunTable &runs) const;
@@ -445,7 +436,7 @@ struct RoundConsts {
 };
 struct RunTable {
     uint32_t bits[kRunLevels][kRunPitch];
-    RoundConsts rc;          // used by the batch kernel only
+    RoundConsts rc;
 };
 
 // Constants of round i (host and device) from the skips of the p at hand.
@@ -476,17 +467,8 @@ __host__ __device__ inline void round_consts(const uint32_t *skips, int i, Round
     }
 }
 
-__device__ __forceinline__ int4 ParamSkips::window(int i, const RunTable &) const { return rc.window[i]; }
-__device__ __forceinline__ uint32_t ParamSkips::len2(int i, const RunTable &) const { return rc.len2[i]; }
 __device__ __forceinline__ int4 SharedSkips::window(int i, const RunTable &runs) const { return runs.rc.window[i]; }
 __device__ __forceinline__ uint32_t SharedSkips::len2(int i, const RunTable &runs) const { return runs.rc.len2[i]; }
-
-inline RoundConsts make_round_consts(const PTable &tab)
-{
-    RoundConsts rc = {};
-    for (int i = 0; i < tab.q; ++i) round_consts(tab.s, i, &rc);
-    return rc;
-}
 
 // The tile is the n ranks first..first+n-1 of a p (n <= 256, one per thread); `stage` is where
 // the tile's rank-major rows start in shared memory, `col` this thread's element of round 0 in
@@ -512,9 +494,7 @@ __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t 
         const uint32_t c = codes[(uint32_t)back];
         runs.bits[0][threadIdx.x] = c & (0u - c);
     }
-    if constexpr (!Skips::kHostConsts) {                  // per-round constants of this p
-        if (threadIdx.x < (uint32_t)q) round_consts(skip.s, threadIdx.x, &runs.rc);
-    }
+    if (threadIdx.x < (uint32_t)q) round_consts(skip.s, threadIdx.x, &runs.rc);   // per-round constants of this p
     int h = -1, bb = 0;
     RoundState st;
     st.B = 0;
@@ -623,36 +603,6 @@ __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t 
         rounds_until(q, r + p);
     }
 }
-
-template <bool kRowOut, bool kColOut>
-__global__ void __launch_bounds__(kTile, 8)
-recv_codes_warp_kernel(const __grid_constant__ PTable tab, const __grid_constant__ RoundConsts rc,
-                       uint64_t r_begin, uint64_t r_end, const uint32_t *__restrict__ codes,
-                       int8_t *recv_out, int8_t *recv_t, uint64_t t_stride)
-{
-    __shared__ __align__(16) uint8_t stage[kTile * 32];
-    __shared__ uint32_t full_sh[kRow];
-    __shared__ RunTable runs;
-    grid_launch_dependents();
-    if (threadIdx.x < kRow) full_sh[threadIdx.x] = tab.full[threadIdx.x];   // read after the tile's first barrier
-    const uint64_t count = r_end - r_begin;
-    const uint64_t g0 = (uint64_t)blockIdx.x * kTile;
-    const uint32_t n = (uint32_t)(count - g0 < (uint64_t)kTile ? count - g0 : (uint64_t)kTile);
-    grid_dependency_wait();                                // the codes are complete from here on
-    recv_warp_tile<kRowOut, kColOut>(ParamSkips{tab, rc}, full_sh, tab.p, tab.q, r_begin + g0, n, codes,
-                                     stage, kColOut ? recv_t + g0 + threadIdx.x : nullptr,
-                                     t_stride, runs);
-    if (kRowOut) {
-        const uint32_t len = n * (uint32_t)tab.q;          // the tile's rows start at byte g0 * q: 16-byte aligned
-        if ((len & 15u) == 0) {
-            flush_span_bulk(stage, len, recv_out, g0 * (uint64_t)tab.q);
-        } else {                                           // ragged last tile
-            __syncthreads();
-            flush_span(stage, 0, len, recv_out, g0 * (uint64_t)tab.q);
-        }
-    }
-}
-
 
 // Single p, p >= 64, four consecutive ranks per thread.  The work of a round that does not depend
 // on the rank -- the address of the codes at the window's lower end, the store into the
