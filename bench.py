@@ -191,8 +191,8 @@ def _bench_allgather(torch, bcs, workloads, flush, hbm_gbs, peak_src, steps):
     return {"workload": "p=100003, n=1000, processor 54607: pack+unpack int32 [1016][100003]",
             "ms": ms, "bytes": nbytes, "gbs": gbs,
             "roofline": {"bound": "hbm", "kernel": "allgather_kernel", "achieved": gbs,
-                         "peak": hbm_gbs, "unit": "GB/s", "frac": gbs / hbm_gbs, "traffic": None,
-                         "peak_source": peak_src}}
+                         "peak": hbm_gbs, "unit": "GB/s", "frac": gbs / hbm_gbs,
+                         "traffic": ALLGATHER_TRAFFIC_BYTES, "peak_source": peak_src}}
 
 
 def _bench_checksum(torch, bcs, flush, hbm_gbs, peak_src, table, steps):
@@ -371,7 +371,7 @@ def run_ours(args) -> None:
         model = ALU_MODEL[q]
         alu_peak = SM_COUNT * ALU_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12     # T int-op/s
         achieved = model * p / (recv_ms * 1e-3) / 1e12
-        roof = {"bound": "alu", "kernel": "codes_kernel+recv_codes_kernel", "achieved": achieved,
+        roof = {"bound": "alu", "kernel": "codes_single_kernel+recv_codes_quad_kernel", "achieved": achieved,
                 "peak": alu_peak, "unit": "Tint-op/s", "frac": achieved / alu_peak,
                 "traffic": RECV_TRAFFIC_BYTES, "ms": recv_ms, "model_int_ops_per_rank": model,
                 "peak_source": "148 SMs x 64 INT32 lanes x %.0f MHz (max SM clock)" % sm_max_mhz,
@@ -510,17 +510,23 @@ def run_ours(args) -> None:
 
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of the
 # current kernels); None until counters have been taken for the kernel as it stands.
-RECV_TRAFFIC_BYTES = 4218368 + 434944        # recv_codes_warp_kernel<true,true>, p = 2^20+1
-# thread instructions per rank that the codes and receive kernels execute on that workload
-# (smsp__thread_inst_executed.sum of the same capture / p): 111 + 1006
-EXECUTED_INST_PER_RANK = {21: 111 + 1006}
-EXPAND_TRAFFIC_BYTES = 1567312000 + 3457280   # expand_kernel, p = 100003, n = 1000
+RECV_TRAFFIC_BYTES = 4257536 + 238080        # recv_codes_quad_kernel<true,true>, p = 2^20+1
+# thread instructions per rank that the codes kernel and the receive-only variant of the receive
+# kernel (the one timed for the roofline line) execute on that workload
+# (smsp__thread_inst_executed.sum of the same capture / p): 91 + 477
+EXECUTED_INST_PER_RANK = {21: 91 + 477}
+EXPAND_TRAFFIC_BYTES = 1566649856 + 3409408   # expand_kernel, p = 100003, n = 1000
+ALLGATHER_TRAFFIC_BYTES = 753529344 + 3564800  # allgather_kernel, p = 100003, n = 1000
 
-# integer operations per rank of the receive-schedule construction that the kernels run, by q:
-# skip code (3 per level + 5) + per round 22 (address select, code load, one step of the head
-# search, set update, entry, two stores, loop) + the measured extra 0.66 search steps and 0.19
-# second windows per rank (CPU count of the same loops over sampled ranks of p = 2^20+1).
-ALU_MODEL = {21: (3 * 21 + 5) + 22 * 21 + 14}
+# Integer operations per rank of the receive-schedule construction as the kernels run it (four
+# ranks per thread share a round's address arithmetic), by q: skip code (3 per level + 5); the six
+# rounds read from the tile's run table 18 each (four words and their addresses 8, the two window
+# sets and the choice between them 4, leading block, its bit and the entry 3, set update, row
+# store, share of the column store); the other rounds 10 each (code load and share of its address
+# 1.5, xor, leading bit, taken-test 4, bit and set update 2, entry, row store, share of the packed
+# column store 1.5); plus 2 for the 0.23 % of the rounds whose first head is taken (CPU count over
+# sampled ranks of p = 2^20+1).
+ALU_MODEL = {21: (3 * 21 + 5) + 6 * 18 + (21 - 6) * 10 + 2}
 
 
 def main() -> None:
