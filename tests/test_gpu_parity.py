@@ -147,7 +147,9 @@ def test_sub_ranges_ragged_tails_and_single_outputs(bcs, fast):
     q = oracle.q_of(p)
     want_r, want_s = oracle.full_table(p)
     for r0, r1 in ((0, 1), (0, 255), (0, 257), (1, 258), (777, 1300), (p - 300, p), (p - 1, p),
-                   (50000, 50000 + 16 * 3 + 5), (99000, 100003)):
+                   (50000, 50000 + 16 * 3 + 5), (99000, 100003),
+                   # several 512-rank tiles of the four-ranks-per-thread kernel, odd starts and ends
+                   (12345, 14002), (3, 70003), (25001 - 700, 25001 + 700)):
         recv, send = _build(bcs, p, r0, r1, fast=fast)
         assert np.array_equal(recv, want_r[r0:r1]), (r0, r1)
         assert np.array_equal(send, want_s[r0:r1]), (r0, r1)      # partly looked up, partly recomputed
