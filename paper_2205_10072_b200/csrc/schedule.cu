@@ -645,6 +645,44 @@ struct QuadConsts {
     int n_special;
 };
 
+// Length of the second window of round i, sum_{j<=i} skips[j] - skips[i+1] + 1, or 0 if empty.
+__host__ __device__ inline uint32_t quad_len2(const uint32_t *skips, int i)
+{
+    uint32_t sum = 0;
+    for (int j = 0; j <= i; ++j) sum += skips[j];
+    return sum >= skips[i + 1] ? sum - skips[i + 1] + 1u : 0u;
+}
+
+// Rounds 0 .. result-1 have skips[i+1] <= 33 and are decided from the run table.
+__host__ __device__ inline int quad_table_rounds(const uint32_t *skips, int q)
+{
+    int rounds = 0;
+    while (rounds < q && rounds < kQuadTableRounds && skips[rounds + 1] <= 33u) ++rounds;
+    return rounds;
+}
+
+// QuadConsts::word[i][w][j] of a p with these skips.  The len >= 1 ranks that end d ranks below a
+// rank are covered by two runs of 2^l ranks, l = floor(log2 len), ending d and d + len - 2^l
+// ranks below: words 0, 1 for the first window (d = skips[i], len = skips[i+1] - skips[i]),
+// words 2, 3 for the second (d = skips[i+1], len = quad_len2), or the first again if it is empty.
+__host__ __device__ inline int32_t quad_word_offset(const uint32_t *skips, int i, int w, int j)
+{
+    const uint32_t lo = skips[i], hi = skips[i + 1];
+    uint32_t d = lo, len = hi - lo;
+    const uint32_t len2 = quad_len2(skips, i);
+    if (w >= 2 && len2) {
+        d = hi;
+        len = len2;
+    }
+    int level = 0;
+    while ((2u << level) <= len) ++level;
+    const uint32_t back = (w & 1) ? d + len - (1u << level) : d;
+    const int rel = j - (int)back;                 // position relative to the quad's first rank
+    const int sub = rel & 3;
+    const int quad = (rel - sub) / 4;              // exact: rel - sub is a multiple of 4
+    return 4 * (level * kQuadLevelWords + sub * kQuadSub + kRunBack / 4 + quad);
+}
+
 inline QuadConsts make_quad_consts(const PTable &tab, uint64_t r_begin, uint64_t r_end)
 {
     QuadConsts qc = {};
@@ -662,81 +700,53 @@ inline QuadConsts make_quad_consts(const PTable &tab, uint64_t r_begin, uint64_t
             add((count - 1) / kQuadTile);
         }
     }
-    RoundConsts rc = {};
-    for (int i = 0; i < tab.q; ++i) {
-        round_consts(tab.s, i, &rc);
-        qc.len2[i] = rc.len2[i];
-    }
-    int rounds = 0;
-    while (rounds < tab.q && rounds < kQuadTableRounds && tab.s[rounds + 1] <= 33u) ++rounds;
-    qc.table_rounds = rounds;
-    for (int i = 0; i < rounds; ++i) {
-        uint32_t sum = 0;
-        for (int j = 0; j <= i; ++j) sum += tab.s[j];
-        const uint32_t lo = tab.s[i], hi = tab.s[i + 1];
-        // the len >= 1 ranks that end d ranks below: runs of 2^l ranks, l = floor(log2 len),
-        // ending d and d + len - 2^l ranks below
-        int level[4];
-        uint32_t back[4];
-        int l1 = 0;
-        while ((2u << l1) <= hi - lo) ++l1;
-        level[0] = level[1] = l1;
-        back[0] = lo;
-        back[1] = hi - (1u << l1);
-        level[2] = level[3] = l1;
-        back[2] = back[0];
-        back[3] = back[1];
-        if (qc.len2[i]) {
-            int l2 = 0;
-            while ((2u << l2) <= qc.len2[i]) ++l2;
-            level[2] = level[3] = l2;
-            back[2] = hi;
-            back[3] = sum + 1u - (1u << l2);
-        }
+    for (int i = 0; i < tab.q; ++i) qc.len2[i] = quad_len2(tab.s, i);
+    qc.table_rounds = quad_table_rounds(tab.s, tab.q);
+    for (int i = 0; i < qc.table_rounds; ++i)
         for (int w = 0; w < 4; ++w)
-            for (int j = 0; j < 4; ++j) {
-                const int rel = j - (int)back[w];            // position relative to the quad's first rank
-                const int sub = rel & 3;
-                const int quad = (rel - sub) / 4;            // exact: rel - sub is a multiple of 4
-                qc.word[i][w][j] = 4 * (level[w] * kQuadLevelWords + sub * kQuadSub + kRunBack / 4 + quad);
-            }
-    }
+            for (int j = 0; j < 4; ++j) qc.word[i][w][j] = quad_word_offset(tab.s, i, w, j);
     return qc;
 }
 
-template <bool kRowOut, bool kColOut>
-__global__ void __launch_bounds__(kQuadThreads, 8)
-recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant__ QuadConsts qc,
-                       uint64_t r_begin, uint64_t r_end, const uint32_t *__restrict__ codes,
-                       int8_t *recv_out, int8_t *recv_t, uint64_t t_stride)
+// Where a quad tile reads the constants of its p from: the kernel parameters (single p:
+// constant-bank operands) ...
+struct ParamEnv {
+    const PTable &tab;
+    const QuadConsts &qc;
+    __device__ __forceinline__ uint32_t skip(int k) const { return tab.s[k]; }
+    __device__ __forceinline__ int word(int i, int w, int j) const { return qc.word[i][w][j]; }
+    __device__ __forceinline__ uint32_t len2(int i) const { return qc.len2[i]; }
+    __device__ __forceinline__ int table_rounds() const { return qc.table_rounds; }
+};
+// ... or shared memory (batch: the CTA computes them for the p of its tile).
+struct SharedEnv {
+    const uint32_t *s;
+    const QuadConsts *qc;
+    __device__ __forceinline__ uint32_t skip(int k) const { return s[k]; }
+    __device__ __forceinline__ int word(int i, int w, int j) const { return qc->word[i][w][j]; }
+    __device__ __forceinline__ uint32_t len2(int i) const { return qc->len2[i]; }
+    __device__ __forceinline__ int table_rounds() const { return qc->table_rounds; }
+};
+
+// One tile: the n <= 512 ranks first .. first+n-1 of a p >= 64 (first may exceed p for the
+// threads past the end of a range: taken mod p), four per thread; all 128 threads must call.
+// codes: skip codes of this p; stage: where the tile's rank-major rows start in shared memory;
+// col_tile: byte of the tile's first rank in round 0 of the round-major copy, rounds t_stride
+// bytes apart (kPackedCol: both multiples of 4, so that the four entries of a quad and round are
+// stored as one word).
+template <bool kRowOut, bool kColOut, bool kPackedCol, class Env>
+__device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh, uint32_t p, int q,
+                                          uint64_t first, uint32_t n,
+                                          const uint32_t *__restrict__ codes, uint8_t *stage,
+                                          int8_t *col_tile, uint64_t t_stride,
+                                          uint32_t (&runs)[kRunLevels][kQuadLevelWords])
 {
-    __shared__ __align__(16) uint8_t stage[kQuadTile * BCS_MAX_Q];
-    __shared__ uint32_t full_sh[kRow];
-    __shared__ uint32_t runs[kRunLevels][kQuadLevelWords];
-    grid_launch_dependents();
     const uint32_t t = threadIdx.x;
-    if (t < kRow) full_sh[t] = tab.full[t];                    // read after the first barrier
-    const uint32_t p = tab.p;
-    const int q = tab.q;
-    const uint64_t count = r_end - r_begin;
-    // The first CTAs of the grid take the tiles that run the general code (listed by the host):
-    // they last longer, so they start first; the others skip a listed tile.
-    uint64_t tile = blockIdx.x;
-    if (blockIdx.x < (uint32_t)qc.n_special) {
-        tile = qc.special[blockIdx.x];
-    } else {
-        tile -= (uint32_t)qc.n_special;
-        if (__syncthreads_or(t < (uint32_t)qc.n_special && qc.special[t] == tile)) return;
-    }
-    grid_dependency_wait();                                    // the codes are complete from here on
-    {
-    const uint64_t g0 = tile * kQuadTile;
-    const uint32_t n = (uint32_t)(count - g0 < (uint64_t)kQuadTile ? count - g0 : (uint64_t)kQuadTile);
     // ranks of the quad mod p (defined for every thread, also past the end of the range: the
     // table entries of such ranks are never read for a rank of the range)
     uint32_t r[4], c[4], B[4];
     {
-        uint64_t wrapped = r_begin + g0 + 4u * t;
+        uint64_t wrapped = first + 4u * t;
         while (wrapped >= p) wrapped -= p;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -747,7 +757,7 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
             runs[0][j * kQuadSub + kRunBack / 4 + t] = B[j];
         }
         if (t < kRunBack / 4) {                                // the 64 ranks before the tile, mod p (p >= 64)
-            uint64_t back = r_begin + g0 + 4u * t + p - kRunBack;
+            uint64_t back = first + 4u * t + p - kRunBack;
             while (back >= p) back -= p;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -794,8 +804,8 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
     const char *mine = reinterpret_cast<const char *>(&runs[0][t]);
     auto word = [&](int byte_offset) { return *reinterpret_cast<const uint32_t *>(mine + byte_offset); };
     uint8_t *row0 = stage + 4u * t * (uint32_t)q;              // rows of the quad: row0 + j * q
-    int8_t *col0 = kColOut ? recv_t + g0 + 4u * t : nullptr;   // the quad's four bytes of round 0
-    const int first_lane_round = qc.table_rounds;
+    int8_t *col0 = kColOut ? col_tile + 4u * t : nullptr;      // the quad's four bytes of round 0
+    const int first_lane_round = env.table_rounds();
     const int h0 = 31 - __clz(c[0]);                           // -1 for the root
     const bool together = 4u * t + 4u <= n && r[0] != 0u && r[3] == r[0] + 3u &&
                           h0 == 31 - __clz(c[3]) && h0 >= first_lane_round;
@@ -822,12 +832,12 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
         }
         uint32_t sum = 0;
         for (int i = 0; i < first_lane_round; ++i) {
-            sum += tab.s[i];
+            sum += env.skip(i);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const uint32_t free_blocks = ~st[j].B;
-                uint32_t U = (word(qc.word[i][0][j]) | word(qc.word[i][1][j])) & free_blocks;
-                const uint32_t U2 = (word(qc.word[i][2][j]) | word(qc.word[i][3][j])) & free_blocks;
+                uint32_t U = (word(env.word(i, 0, j)) | word(env.word(i, 1, j))) & free_blocks;
+                const uint32_t U2 = (word(env.word(i, 2, j)) | word(env.word(i, 3, j))) & free_blocks;
                 if (U == 0) U = U2;
                 const int lead = __clz(U);
                 uint32_t bit = U ? 0x80000000u >> lead : 0u;
@@ -842,7 +852,7 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
             }
         }
         if (first_lane_round < q) {
-            const uint32_t edge = tab.s[first_lane_round];
+            const uint32_t edge = env.skip(first_lane_round);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 st[j].sum = sum;
@@ -850,7 +860,7 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
                 st[j].upper = codes[r[j] - edge + (r[j] >= edge ? 0u : p)];
             }
             for (int i = first_lane_round; i < q; ++i) {
-                const uint32_t hi_skip = tab.s[i + 1];
+                const uint32_t hi_skip = env.skip(i + 1);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int entry = recv_round(codes, full_sh, p, q, r[j], i, h[j], bb[j], hi_skip, st[j]);
@@ -861,8 +871,8 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
         }
     } else if (!empty) {
         // ---- the four ranks together: same homerange h0, no home round among the table rounds
-        uint32_t *col = reinterpret_cast<uint32_t *>(col0);    // g0 + 4t and t_stride are multiples of 4
-        const uint64_t col_step = t_stride / 4;
+        // kPackedCol: col_tile and t_stride are multiples of 4, the four entries of a round are one word
+        int8_t *col = col0;
         int i = 0;
 #pragma unroll
         for (int unrolled = 0; unrolled < kQuadTableRounds; ++unrolled) {
@@ -872,8 +882,8 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const uint32_t free_blocks = ~B[j];
-                uint32_t U = (word(qc.word[unrolled][0][j]) | word(qc.word[unrolled][1][j])) & free_blocks;
-                const uint32_t U2 = (word(qc.word[unrolled][2][j]) | word(qc.word[unrolled][3][j])) & free_blocks;
+                uint32_t U = (word(env.word(unrolled, 0, j)) | word(env.word(unrolled, 1, j))) & free_blocks;
+                const uint32_t U2 = (word(env.word(unrolled, 2, j)) | word(env.word(unrolled, 3, j))) & free_blocks;
                 if (U == 0) U = U2;
                 const int lead = __clz(U);                     // 32 when U == 0
                 B[j] |= U ? 0x80000000u >> lead : 0u;
@@ -882,8 +892,13 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
                 packed |= ((uint32_t)entry & 0xffu) << (8 * j);
             }
             if (kColOut) {
-                *col = packed;
-                col += col_step;
+                if (kPackedCol) {
+                    *reinterpret_cast<uint32_t *>(col) = packed;
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) col[j] = (int8_t)(packed >> (8 * j));
+                }
+                col += t_stride;
             }
             i = unrolled + 1;
         }
@@ -902,22 +917,28 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
                 ++out;
             }
             if (kColOut) {
-                *col = ((uint32_t)entry[0] & 0xffu) | (((uint32_t)entry[1] & 0xffu) << 8) |
-                       (((uint32_t)entry[2] & 0xffu) << 16) | ((uint32_t)entry[3] << 24);
-                col += col_step;
+                if (kPackedCol) {
+                    *reinterpret_cast<uint32_t *>(col) =
+                        ((uint32_t)entry[0] & 0xffu) | (((uint32_t)entry[1] & 0xffu) << 8) |
+                        (((uint32_t)entry[2] & 0xffu) << 16) | ((uint32_t)entry[3] << 24);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) col[j] = (int8_t)entry[j];
+                }
+                col += t_stride;
             }
         };
         // rounds i .. end-1 with the window bounds at from - skip (from = r[0] or r[0] + p)
         auto rounds_until = [&](int end, uint32_t from) {
             if (i >= end) return;
             uint32_t ahead[4];
-            load4(ahead, from - tab.s[i + 1]);
+            load4(ahead, from - env.skip(i + 1));
 #pragma unroll 2
             for (; i < end; ++i) {
-                const uint32_t below = from - tab.s[i + 1];
+                const uint32_t below = from - env.skip(i + 1);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) lower[j] = ahead[j];
-                if (i + 1 < end) load4(ahead, from - tab.s[i + 2]);
+                if (i + 1 < end) load4(ahead, from - env.skip(i + 2));
                 // The first head of each of the four windows, then ONE test whether any of them is
                 // already taken (or its window empty): the four chains stay free of branches.
                 int blk[4];
@@ -946,7 +967,7 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
                                 b = 31 - __clz(fresh);
                             else
                                 b = pick_rest(codes, full_sh, p, q, below + j, lower[j], upper[j],
-                                              qc.len2[i], B[j]);
+                                              env.len2(i), B[j]);
                             blk[j] = b >= 0 ? b : BCS_BAD_ENTRY + q;   // entry BCS_BAD_ENTRY, no bit
                         }
                     }
@@ -961,18 +982,50 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
                 store_round(entry);
             }
         };
-        load4(upper, r[0] - tab.s[i]);                         // i <= h0: skips[i] <= r[0]
+        load4(upper, r[0] - env.skip(i));                         // i <= h0: skips[i] <= r[0]
         rounds_until(h0, r[0]);
         {                                                      // home round: the baseblocks themselves
             int entry[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) entry[j] = __ffs(c[j]) - 1;
             store_round(entry);
-            load4(upper, r[0] + p - tab.s[h0 + 1]);            // r[3] < skips[h0+1]
+            load4(upper, r[0] + p - env.skip(h0 + 1));            // r[3] < skips[h0+1]
             i = h0 + 1;
         }
         rounds_until(q, r[0] + p);
     }
+}
+
+template <bool kRowOut, bool kColOut>
+__global__ void __launch_bounds__(kQuadThreads, 8)
+recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant__ QuadConsts qc,
+                       uint64_t r_begin, uint64_t r_end, const uint32_t *__restrict__ codes,
+                       int8_t *recv_out, int8_t *recv_t, uint64_t t_stride)
+{
+    __shared__ __align__(16) uint8_t stage[kQuadTile * BCS_MAX_Q];
+    __shared__ uint32_t full_sh[kRow];
+    __shared__ uint32_t runs[kRunLevels][kQuadLevelWords];
+    grid_launch_dependents();
+    const uint32_t t = threadIdx.x;
+    if (t < kRow) full_sh[t] = tab.full[t];                    // read after the first barrier
+    const uint32_t p = tab.p;
+    const int q = tab.q;
+    const uint64_t count = r_end - r_begin;
+    // The first CTAs of the grid take the tiles that run the general code (listed by the host):
+    // they last longer, so they start first; the others skip a listed tile.
+    uint64_t tile = blockIdx.x;
+    if (blockIdx.x < (uint32_t)qc.n_special) {
+        tile = qc.special[blockIdx.x];
+    } else {
+        tile -= (uint32_t)qc.n_special;
+        if (__syncthreads_or(t < (uint32_t)qc.n_special && qc.special[t] == tile)) return;
+    }
+    grid_dependency_wait();                                    // the codes are complete from here on
+    const uint64_t g0 = tile * kQuadTile;
+    const uint32_t n = (uint32_t)(count - g0 < (uint64_t)kQuadTile ? count - g0 : (uint64_t)kQuadTile);
+    // g0 and t_stride are multiples of 4 and recv_t is 16-byte aligned: packed column stores
+    quad_tile<kRowOut, kColOut, true>(ParamEnv{tab, qc}, full_sh, p, q, r_begin + g0, n, codes, stage,
+                                      kColOut ? recv_t + g0 : nullptr, t_stride, runs);
     if (kRowOut) {
         const uint32_t len = n * (uint32_t)q;                  // the tile's rows start at byte g0 * q: 16-byte aligned
         if ((len & 15u) == 0) {
@@ -982,7 +1035,85 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
             flush_span(stage, 0, len, recv_out, g0 * (uint64_t)q);
         }
     }
+}
+
+// Batch: 512 flattened ranks per CTA.  A CTA whose ranks all belong to one p >= 64 (nearly all
+// CTAs when the p are large) runs the quad tile with that p's constants computed into shared
+// memory; a CTA that straddles several p, or a small p, runs the per-lane search rank by rank.
+// The tile's rows start at any byte of the output (staged shifted by that byte's offset in its
+// 16-byte group), and a round of the round-major copy is p bytes long: no packed column stores.
+struct QuadBatchShared {
+    uint32_t skips[kRow], full[kRow];
+    QuadConsts qc;
+    uint64_t span_begin, span_end;          // bytes of the output that the CTA writes
+    uint64_t rank0, entry0;                 // flattened rank and byte offset of rank 0 of the first p
+    uint32_t j_first, j_last, p_first;
+    __align__(16) uint8_t stage[kQuadTile * BCS_MAX_Q + 16];
+    uint32_t runs[kRunLevels][kQuadLevelWords];
+};
+
+template <bool kColOut>
+__global__ void __launch_bounds__(kQuadThreads, 8)
+recv_quad_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t *recv_out,
+                       int8_t *recv_t)
+{
+    __shared__ QuadBatchShared sh;
+    const uint32_t t = threadIdx.x;
+    const uint64_t g0 = (uint64_t)blockIdx.x * kQuadTile;
+    const uint64_t g1 = g0 + kQuadTile < ba.total_ranks ? g0 + kQuadTile : ba.total_ranks;
+    if (t < 32) {
+        const uint32_t jf = find_segment_warp(ba.rank_off, ba.num_p, g0);
+        const uint32_t jl = ba.rank_off[jf + 1] >= g1 ? jf : find_segment_warp(ba.rank_off, ba.num_p, g1 - 1);
+        if (t == 0) {
+            sh.j_first = jf;
+            sh.j_last = jl;
+            sh.p_first = ba.p_list[jf];
+            sh.rank0 = ba.rank_off[jf];
+            sh.entry0 = ba.entry_off[jf];
+            const int qf = ceil_log2_fast(sh.p_first);
+            const int ql = ceil_log2_fast(ba.p_list[jl]);
+            sh.span_begin = sh.entry0 + (g0 - sh.rank0) * (uint64_t)qf;
+            sh.span_end = ba.entry_off[jl] + (g1 - ba.rank_off[jl]) * (uint64_t)ql;
+        }
     }
+    __syncthreads();
+    const uint32_t jf = sh.j_first, jl = sh.j_last;
+    const uint32_t shift = (uint32_t)(sh.span_begin & 15u);
+    if (jf == jl && sh.p_first >= 64u) {                           // uniform over the CTA
+        const uint32_t p = sh.p_first;
+        const int q = ceil_log2_fast(p);
+        const uint32_t *skips = ba.skips_tab + (size_t)jf * kRow;  // the constants of this p
+        if (t < kRow) {
+            sh.skips[t] = skips[t];
+            sh.full[t] = ba.full_tab[(size_t)jf * kRow + t];
+            if (t < (uint32_t)q) sh.qc.len2[t] = quad_len2(skips, (int)t);
+            if (t == 0) sh.qc.table_rounds = quad_table_rounds(skips, q);
+        } else if (t < kRow + kQuadTableRounds * 16 && (int)((t - kRow) >> 4) < q) {
+            const uint32_t e = t - kRow;                           // round e / 16, word (e / 4) % 4, rank e % 4
+            sh.qc.word[e >> 4][(e >> 2) & 3u][e & 3u] = quad_word_offset(skips, (int)(e >> 4), (int)((e >> 2) & 3u), (int)(e & 3u));
+        }
+        // (the tile's first barrier comes before anything here is read)
+        const uint64_t first = g0 - sh.rank0;
+        quad_tile<true, kColOut, false>(SharedEnv{sh.skips, &sh.qc}, sh.full, p, q, first, (uint32_t)(g1 - g0),
+                                        codes + sh.rank0, sh.stage + shift,
+                                        kColOut ? recv_t + sh.entry0 + first : nullptr, (uint64_t)p, sh.runs);
+    } else {
+        for (uint64_t g = g0 + t; g < g1; g += kQuadThreads) {
+            const uint32_t j = find_segment(ba.rank_off, jf, jl, g);
+            const uint32_t p = ba.p_list[j];
+            const int q = ceil_log2_fast(p);
+            if (q == 0) continue;
+            const uint64_t rank0 = ba.rank_off[j], entry0 = ba.entry_off[j];
+            const uint32_t r = (uint32_t)(g - rank0);
+            uint8_t *row = sh.stage + shift + (entry0 + (uint64_t)r * (uint64_t)q - sh.span_begin);
+            int8_t *col = kColOut ? recv_t + entry0 + r : nullptr;
+            recv_rounds_codes<true, kColOut>(codes + rank0, ba.skips_tab + (size_t)j * kRow,
+                                             ba.full_tab + (size_t)j * kRow, p, q, r, q - 1, row, col,
+                                             (uint64_t)p);
+        }
+    }
+    __syncthreads();
+    flush_span(sh.stage, shift, (uint32_t)(sh.span_end - sh.span_begin), recv_out, sh.span_begin);
 }
 
 // Batch: a CTA whose 256 flattened ranks all belong to one p >= 64 (nearly all CTAs when the p
@@ -1613,10 +1744,11 @@ bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_
         int8_t *recv_t = static_cast<int8_t *>(workspace) + align_up(4ull * total_ranks, 256);
         codes_batch_kernel<<<blocks, kTile, 0, stream>>>(ba, codes);
         if ((st = launch_status()) != BCS_OK) return st;
+        const unsigned qblocks = (unsigned)((total_ranks + kQuadTile - 1) / kQuadTile);
         if (send_out != nullptr)
-            recv_codes_batch_kernel<true><<<blocks, kTile, 0, stream>>>(ba, codes, recv_out, recv_t);
+            recv_quad_batch_kernel<true><<<qblocks, kQuadThreads, 0, stream>>>(ba, codes, recv_out, recv_t);
         else
-            recv_codes_batch_kernel<false><<<blocks, kTile, 0, stream>>>(ba, codes, recv_out, nullptr);
+            recv_quad_batch_kernel<false><<<qblocks, kQuadThreads, 0, stream>>>(ba, codes, recv_out, nullptr);
         if ((st = launch_status()) != BCS_OK) return st;
         if (send_out != nullptr) {
             send_batch_kernel<<<blocks, kTile, 0, stream>>>(ba, recv_t, send_out);
