@@ -237,14 +237,63 @@ inline void launch_codes(const PTable &tab, uint32_t *codes, cudaStream_t stream
                                      stream);
 }
 
-// Batch: codes[g] for the flattened rank g.
+// Batch: codes[g] for the flattened rank g, 1024 flattened ranks per CTA.  A CTA inside one p
+// (nearly all when the p are large) scans four consecutive ranks per thread, one shared-memory
+// load of the skip per level for the four, and stores their codes as one 16-byte vector; a CTA
+// that straddles several p finds the p of every rank.
+constexpr int kCodesTile = 4 * kTile;
 __global__ void __launch_bounds__(kTile)
 codes_batch_kernel(BatchArgs ba, uint32_t *__restrict__ codes)
 {
-    __shared__ TileShared sh;
-    PTable unused;
-    RankCtx c = resolve_rank<true>(sh, unused, 0, 0, ba);
-    if (c.valid) codes[c.rank0 + c.r] = skip_code(c.s, c.q, c.r);
+    __shared__ uint32_t skips_sh[kRow];
+    __shared__ uint32_t seg[3];                  // first and last p of the CTA, the first p itself
+    __shared__ uint64_t rank0_sh;
+    const uint64_t g0 = (uint64_t)blockIdx.x * kCodesTile;
+    const uint64_t g1 = g0 + kCodesTile < ba.total_ranks ? g0 + kCodesTile : ba.total_ranks;
+    if (threadIdx.x < 32) {
+        const uint32_t jf = find_segment_warp(ba.rank_off, ba.num_p, g0);
+        const uint32_t jl = ba.rank_off[jf + 1] >= g1 ? jf : find_segment_warp(ba.rank_off, ba.num_p, g1 - 1);
+        skips_sh[threadIdx.x] = ba.skips_tab[(size_t)jf * kRow + threadIdx.x];
+        if (threadIdx.x == 0) {
+            seg[0] = jf;
+            seg[1] = jl;
+            seg[2] = ba.p_list[jf];
+            rank0_sh = ba.rank_off[jf];
+        }
+    }
+    __syncthreads();
+    const uint32_t jf = seg[0], jl = seg[1];
+    if (jf == jl) {
+        const uint64_t g = g0 + 4u * threadIdx.x;
+        if (g >= g1) return;
+        const int q = ceil_log2_fast(seg[2]);
+        uint32_t x[4], code[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) x[e] = (uint32_t)(g - rank0_sh) + e;   // ranks >= p give unused codes
+        for (int k = q - 1; k >= 0; --k) {
+            const uint32_t skip = skips_sh[k];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                if (x[e] >= skip) {
+                    x[e] -= skip;
+                    code[e] |= 1u << k;
+                }
+            }
+        }
+        if (g + 4 <= g1) {
+            *reinterpret_cast<uint4 *>(codes + g) = make_uint4(code[0], code[1], code[2], code[3]);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (g + e < g1) codes[g + e] = code[e];
+        }
+    } else {
+        for (uint64_t g = g0 + threadIdx.x; g < g1; g += kTile) {
+            const uint32_t j = find_segment(ba.rank_off, jf, jl, g);
+            const uint32_t p = ba.p_list[j];
+            codes[g] = skip_code(ba.skips_tab + (size_t)j * kRow, ceil_log2_fast(p), (uint32_t)(g - ba.rank_off[j]));
+        }
+    }
 }
 
 // Largest block among the baseblocks of the ranks x+1..y that is not in B, or -1; X and F
@@ -1403,32 +1452,67 @@ inline void launch_transpose(const PTable &tab, const int8_t *recv_t, uint64_t t
                                          dependent, stream);
 }
 
-// Batch: a CTA inside one p transposes; a CTA that straddles several p gathers byte by byte.
-__global__ void __launch_bounds__(kTile, 6)
+// Batch: 256 flattened ranks and 64 threads per CTA, as in the single-p kernel.  A CTA inside one
+// p transposes; a CTA that straddles several p gathers byte by byte.
+struct SendBatchShared {
+    uint32_t skips[kRow];
+    uint64_t span_begin, span_end;          // bytes of the output that the CTA writes
+    uint64_t rank0, entry0;                 // flattened rank and byte offset of rank 0 of the first p
+    uint32_t j_first, j_last, p_first;
+    __align__(16) uint8_t stage[kStageBytes];
+};
+
+__global__ void __launch_bounds__(kTrThreads)
 send_batch_kernel(BatchArgs ba, const int8_t *__restrict__ recv_t, int8_t *send_out)
 {
-    __shared__ TileShared sh;
+    __shared__ SendBatchShared sh;
     __shared__ BatchRoundBuffer rb;
-    PTable unused;
-    RankCtx c = resolve_rank<true>(sh, unused, 0, 0, ba);
-    const uint32_t shift = (uint32_t)(sh.span_begin & 15u);
-    if (sh.j_first == sh.j_last) {                            // uniform over the CTA
-        const uint64_t g0 = (uint64_t)blockIdx.x * kTile;
-        const uint32_t n = (uint32_t)(ba.total_ranks - g0 < (uint64_t)kTile ? ba.total_ranks - g0
-                                                                             : (uint64_t)kTile);
-        if (c.q > 0) {
-            if (!load_rounds(SharedSkips{sh.skips[0]}, c.p, c.q, recv_t + ba.entry_off[c.pj],
-                             (uint64_t)c.p, (uint32_t)(g0 - c.rank0), n, true, rb))
-                return;
-            if (threadIdx.x < kTrThreads) GatherDispatch<BCS_MAX_Q>::run(c.q, rb, sh.stage + shift);
+    const uint32_t t = threadIdx.x;
+    const uint64_t g0 = (uint64_t)blockIdx.x * kTile;
+    const uint64_t g1 = g0 + kTile < ba.total_ranks ? g0 + kTile : ba.total_ranks;
+    if (t < 32) {
+        const uint32_t jf = find_segment_warp(ba.rank_off, ba.num_p, g0);
+        const uint32_t jl = ba.rank_off[jf + 1] >= g1 ? jf : find_segment_warp(ba.rank_off, ba.num_p, g1 - 1);
+        sh.skips[t] = ba.skips_tab[(size_t)jf * kRow + t];
+        if (t == 0) {
+            sh.j_first = jf;
+            sh.j_last = jl;
+            sh.p_first = ba.p_list[jf];
+            sh.rank0 = ba.rank_off[jf];
+            sh.entry0 = ba.entry_off[jf];
+            const int qf = ceil_log2_fast(sh.p_first);
+            const int ql = ceil_log2_fast(ba.p_list[jl]);
+            sh.span_begin = sh.entry0 + (g0 - sh.rank0) * (uint64_t)qf;
+            sh.span_end = ba.entry_off[jl] + (g1 - ba.rank_off[jl]) * (uint64_t)ql;
         }
-    } else if (c.valid) {
-        uint8_t *row = sh.stage + shift + (c.entry - sh.span_begin);
-        const int8_t *tbl = recv_t + ba.entry_off[c.pj];
-        for (int k = 0; k < c.q; ++k) {
-            uint32_t t = c.r + c.s[k];
-            if (t >= c.p) t -= c.p;
-            row[k] = (uint8_t)tbl[(uint64_t)k * c.p + t];
+    }
+    __syncthreads();
+    const uint32_t jf = sh.j_first, jl = sh.j_last;
+    const uint32_t shift = (uint32_t)(sh.span_begin & 15u);
+    if (jf == jl) {                                            // uniform over the CTA
+        const uint32_t p = sh.p_first;
+        const int q = ceil_log2_fast(p);
+        if (q > 0) {
+            if (!load_rounds(SharedSkips{sh.skips}, p, q, recv_t + sh.entry0, (uint64_t)p,
+                             (uint32_t)(g0 - sh.rank0), (uint32_t)(g1 - g0), true, rb))
+                return;
+            GatherDispatch<BCS_MAX_Q>::run(q, rb, sh.stage + shift);
+        }
+    } else {
+        for (uint64_t g = g0 + t; g < g1; g += kTrThreads) {
+            const uint32_t j = find_segment(ba.rank_off, jf, jl, g);
+            const uint32_t p = ba.p_list[j];
+            const int q = ceil_log2_fast(p);
+            const uint64_t entry0 = ba.entry_off[j];
+            const uint32_t r = (uint32_t)(g - ba.rank_off[j]);
+            const uint32_t *skips = ba.skips_tab + (size_t)j * kRow;
+            uint8_t *row = sh.stage + shift + (entry0 + (uint64_t)r * (uint64_t)q - sh.span_begin);
+            const int8_t *tbl = recv_t + entry0;
+            for (int k = 0; k < q; ++k) {
+                uint32_t to = r + skips[k];
+                if (to >= p) to -= p;
+                row[k] = (uint8_t)tbl[(uint64_t)k * p + to];
+            }
         }
     }
     __syncthreads();
@@ -1742,7 +1826,7 @@ bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_
         workspace_bytes >= bcs_build_batch_workspace_bytes(total_ranks, total_entries)) {
         uint32_t *codes = static_cast<uint32_t *>(workspace);
         int8_t *recv_t = static_cast<int8_t *>(workspace) + align_up(4ull * total_ranks, 256);
-        codes_batch_kernel<<<blocks, kTile, 0, stream>>>(ba, codes);
+        codes_batch_kernel<<<(unsigned)((total_ranks + kCodesTile - 1) / kCodesTile), kTile, 0, stream>>>(ba, codes);
         if ((st = launch_status()) != BCS_OK) return st;
         const unsigned qblocks = (unsigned)((total_ranks + kQuadTile - 1) / kQuadTile);
         if (send_out != nullptr)
@@ -1751,7 +1835,7 @@ bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_
             recv_quad_batch_kernel<false><<<qblocks, kQuadThreads, 0, stream>>>(ba, codes, recv_out, nullptr);
         if ((st = launch_status()) != BCS_OK) return st;
         if (send_out != nullptr) {
-            send_batch_kernel<<<blocks, kTile, 0, stream>>>(ba, recv_t, send_out);
+            send_batch_kernel<<<blocks, kTrThreads, 0, stream>>>(ba, recv_t, send_out);
             if ((st = launch_status()) != BCS_OK) return st;
         }
         return BCS_OK;
