@@ -5,7 +5,7 @@
 // Two constructions, bit-identical in their results:
 //
 //  * workspace path.  codes_single_kernel / codes_batch_kernel write the skip code (bcs_common.cuh) of every rank x of a p
-//    once.  The receive kernels (recv_codes_quad_kernel for one p >= 64, recv_codes_batch_kernel
+//    once.  The receive kernels (recv_codes_quad_kernel for one p >= 64, recv_quad_batch_kernel
 //    for a batch, recv_codes_kernel for tiny p) then read, per rank r and round i, the codes of
 //    the two ranks that bound the window of Algorithm 4 (r - skips[i+1], r - skips[i];
 //    consecutive threads read consecutive words) and find the largest new block of the window
@@ -447,213 +447,28 @@ recv_codes_kernel(PTable tab, uint64_t r_begin, uint64_t r_end,
     }
 }
 
-// A tile of 256 ranks of one p >= 64, one rank per thread (the batch kernel's tiles; a single p
-// uses recv_codes_quad_kernel below): the first rounds are decided from a table of the tile.  The
-// windows of the rounds with skips[i+1] <= 33 (at most six rounds, i <= 5) reach only a few
-// ranks back: the first window ends skips[i+1] - 1 ranks below r, the second at
+// The run table.  The windows of the rounds with skips[i+1] <= 33 (at most six rounds, i <= 5)
+// reach only a few ranks back: the first window ends skips[i+1] - 1 ranks below r, the second at
 // sum_{j<=i} skips[j] <= skips[i+1] + i <= 38 (every halving rounds up by at most one), and a run
 // of the table adds at most 3 more to the second and none beyond skips[i+1] - 1 to the first.  So
 // every baseblock those windows can contain is the lowest code bit of one of the tile's ranks or
-// of the 64 ranks before the tile.  The tile keeps, for x = every one of those 320 ranks and
-// j = 0..4, the baseblock bits OR-ed over the 2^j ranks that end at x (runs of 2 and 4 from the
+// of the 64 ranks before the tile.  The tile keeps, for x = every one of those ranks and
+// l = 0..4, the baseblock bits OR-ed over the 2^l ranks that end at x (runs of 2 and 4 from the
 // single bits, runs of 8 and 16 from the runs of 4: two barriers after the one that publishes the
 // bits); a window of L ranks is the union of two such runs of 2^floor(log2 L) ranks: two
 // shared-memory words per window, whatever its length, at offsets that depend on p and the round
-// only (RoundConsts).  These are the rounds in which
-// neighbouring ranks disagree about which path of the code search they take; the later rounds
-// run the code search per lane.
-// Where the skips of the tile's p are read from: a table row in shared memory.
-struct RoundConsts;
-struct RunTable;
+// only.  These are the rounds in which neighbouring ranks disagree about which path of the code
+// search they take; the later rounds run the code search per lane.
+constexpr int kRunBack = 64;                   // ranks before the tile that the run table covers
+constexpr int kRunLevels = 5;                  // runs of 1, 2, 4, 8, 16 ranks
+
+// Skips of a p from a table row in shared memory.
 struct SharedSkips {
     const uint32_t *s;
     __device__ __forceinline__ uint32_t operator()(int k) const { return s[k]; }
-    __device__ __forceinline__ int4 window(int i, const RunTable &runs) const;
-    __device__ __forceinline__ uint32_t len2(int i, const RunTable &runs) const;
 };
 
-constexpr int kRunBack = 64;                   // ranks before the tile that the run table covers
-constexpr int kRunLevels = 5;                  // runs of 1, 2, 4, 8, 16 ranks
-constexpr int kRunPitch = kTile + kRunBack;    // words per level
-// Per-round constants of one p.
-struct RoundConsts {
-    // Round i of the table rounds reads the four words at these byte offsets from a thread's own
-    // level-0 entry: .x | .y is its first window, .z | .w its second (a repeat of the first when
-    // the round has no second window).
-    int4 window[8];
-    uint32_t len2[kRow];     // length of the second window of round i: sum_{j<=i} skips[j] - skips[i+1] + 1, or 0
-};
-struct RunTable {
-    uint32_t bits[kRunLevels][kRunPitch];
-    RoundConsts rc;
-};
-
-// Constants of round i (host and device) from the skips of the p at hand.
-__host__ __device__ inline void round_consts(const uint32_t *skips, int i, RoundConsts *rc)
-{
-    uint32_t sum = 0;
-    for (int j = 0; j <= i; ++j) sum += skips[j];
-    const uint32_t lo = skips[i], hi = skips[i + 1];
-    const uint32_t len2 = sum >= hi ? sum - hi + 1u : 0u;
-    rc->len2[i] = len2;
-    if (hi <= 33u) {
-        // the len >= 1 ranks that end d ranks below: runs of 2^j ranks, j = floor(log2 len),
-        // ending d and d + len - 2^j ranks below
-        int j1 = 0;
-        while ((2u << j1) <= hi - lo) ++j1;
-        int4 w;
-        w.x = 4 * (j1 * kRunPitch - (int)lo);
-        w.y = 4 * (j1 * kRunPitch - (int)(hi - (1u << j1)));
-        w.z = w.x;
-        w.w = w.y;
-        if (len2) {
-            int j2 = 0;
-            while ((2u << j2) <= len2) ++j2;
-            w.z = 4 * (j2 * kRunPitch - (int)hi);
-            w.w = 4 * (j2 * kRunPitch - (int)(sum + 1u - (1u << j2)));
-        }
-        rc->window[i] = w;
-    }
-}
-
-__device__ __forceinline__ int4 SharedSkips::window(int i, const RunTable &runs) const { return runs.rc.window[i]; }
-__device__ __forceinline__ uint32_t SharedSkips::len2(int i, const RunTable &runs) const { return runs.rc.len2[i]; }
-
-// The tile is the n ranks first..first+n-1 of a p (n <= 256, one per thread); `stage` is where
-// the tile's rank-major rows start in shared memory, `col` this thread's element of round 0 in
-// the round-major copy.  All 256 threads must call (the table is built by all of them).
-template <bool kRowOut, bool kColOut, class Skips>
-__device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t *full_sh,
-                                               uint32_t p, int q, uint64_t first, uint32_t n,
-                                               const uint32_t *__restrict__ codes, uint8_t *stage,
-                                               int8_t *col, uint64_t t_stride, RunTable &runs)
-{
-    const bool valid = threadIdx.x < n;
-    // rank of this thread mod p (defined for every thread, also past the end of the range: the
-    // table entries of such ranks are never read by a valid thread)
-    uint64_t wrapped = first + threadIdx.x;
-    while (wrapped >= p) wrapped -= p;
-    const uint32_t r = (uint32_t)wrapped;
-    const uint32_t own = codes[r];
-    const uint32_t own_bit = own & (0u - own);            // baseblock of r as a bit, 0 for the root
-    runs.bits[0][kRunBack + threadIdx.x] = own_bit;
-    if (threadIdx.x < kRunBack) {                         // the 64 ranks before the tile, mod p (p >= 64)
-        uint64_t back = first + threadIdx.x + p - kRunBack;
-        while (back >= p) back -= p;
-        const uint32_t c = codes[(uint32_t)back];
-        runs.bits[0][threadIdx.x] = c & (0u - c);
-    }
-    if (threadIdx.x < (uint32_t)q) round_consts(skip.s, threadIdx.x, &runs.rc);   // per-round constants of this p
-    int h = -1, bb = 0;
-    RoundState st;
-    st.B = 0;
-    if (r > 0) {
-        h = 31 - __clz(own);
-        bb = __ffs(own) - 1;
-        st.B = own_bit;
-    }
-    uint8_t *row = stage + threadIdx.x * q;
-    __syncthreads();
-    // levels 1 and 2 from level 0, then levels 3 and 4 from level 2: entry x of level j is
-    // complete from x = 2^j - 1 on, and nothing below x = 23 is ever read
-    auto build = [&](int x) {
-        const uint32_t *b = &runs.bits[0][x];
-        const uint32_t pair = b[0] | b[-1];
-        runs.bits[1][x] = pair;
-        runs.bits[2][x] = pair | b[-2] | b[-3];
-    };
-    build(kRunBack + threadIdx.x);
-    if (threadIdx.x < kRunBack && threadIdx.x >= 3u) build(threadIdx.x);
-    __syncthreads();
-    auto build_wide = [&](int x) {
-        const uint32_t *b = &runs.bits[2][x];
-        const uint32_t eight = b[0] | b[-4];
-        runs.bits[3][x] = eight;
-        runs.bits[4][x] = eight | b[-8] | b[-12];
-    };
-    build_wide(kRunBack + threadIdx.x);
-    if (threadIdx.x < kRunBack && threadIdx.x >= 15u) build_wide(threadIdx.x);
-    __syncthreads();
-    const char *mine = reinterpret_cast<const char *>(&runs.bits[0][kRunBack + threadIdx.x]);
-    auto word = [&](int byte_offset) { return *reinterpret_cast<const uint32_t *>(mine + byte_offset); };
-    int i = 0;
-#pragma unroll
-    for (int unrolled = 0; unrolled < 6; ++unrolled) {    // at most six such rounds; uniform over the grid
-        if (!(unrolled < q && skip(unrolled + 1) <= 33u)) break;
-        i = unrolled;
-        const int4 w = skip.window(i, runs);
-        const uint32_t free_blocks = ~st.B;
-        uint32_t U = (word(w.x) | word(w.y)) & free_blocks;       // ranks r - d, d = skips[i]..skips[i+1]-1
-        const uint32_t U2 = (word(w.z) | word(w.w)) & free_blocks; // d = skips[i+1]..sum_{j<=i} skips[j]
-        if (U == 0) U = U2;
-        // largest block of U; the home round takes the baseblock and leaves B alone
-        const int lead = __clz(U);                                 // 32 when U == 0
-        uint32_t bit = U ? 0x80000000u >> lead : 0u;
-        int entry = U ? 31 - q - lead : BCS_BAD_ENTRY;
-        if (i == h) {
-            entry = bb;
-            bit = 0;
-        }
-        st.B |= bit;
-        if (kRowOut) row[i] = (uint8_t)entry;
-        if (kColOut && valid) *col = (int8_t)entry;
-        if (kColOut) col += t_stride;
-        i = unrolled + 1;
-    }
-    if (valid && i < q) {
-        // Per-lane rounds.  Before the home round h both window bounds are r - skip, after it
-        // both are r + p - skip: two loops with the wrap decided once, the home round between.
-        const uint32_t edge = skip(i);
-        st.upper = codes[r - edge + (r >= edge ? 0u : p)];  // code of r - skips[i]
-        uint8_t *out = row + i;
-        // lower = code of the rank at the lower end of the window, from - skips[ii+1]
-        auto round = [&](int ii, uint32_t from, uint32_t lower) {
-            const uint32_t diff = lower ^ st.upper;
-            int blk = 31 - __clz(diff);                      // first head; -1 for an empty window
-            int entry;
-            if (diff == 0 || ((st.B >> blk) & 1u)) {
-                blk = pick_rest(codes, full_sh, p, q, from - skip(ii + 1), lower, st.upper,
-                                skip.len2(ii, runs), st.B);
-                entry = blk < 0 ? BCS_BAD_ENTRY : blk - q;
-                if (blk >= 0) st.B |= 1u << blk;
-            } else {
-                st.B |= 1u << blk;
-                entry = blk - q;
-            }
-            st.upper = lower;
-            if (kRowOut) *out++ = (uint8_t)entry;
-            if (kColOut) {
-                *col = (int8_t)entry;
-                col += t_stride;
-            }
-        };
-        // The code a round needs depends on the rank and the round only, not on the rounds
-        // before: it is loaded one round ahead, so its latency overlaps the round in between.
-        auto rounds_until = [&](int end, uint32_t from) {    // from = r or r + p
-            if (i >= end) return;
-            uint32_t ahead = codes[from - skip(i + 1)];
-#pragma unroll 2
-            for (; i < end; ++i) {
-                const uint32_t lower = ahead;
-                if (i + 1 < end) ahead = codes[from - skip(i + 2)];
-                round(i, from, lower);
-            }
-        };
-        rounds_until(h < q ? h : q, r);
-        if (i == h) {                                        // home round: the baseblock itself
-            st.upper = codes[r + p - skip(i + 1)];
-            if (kRowOut) *out++ = (uint8_t)bb;
-            if (kColOut) {
-                *col = (int8_t)bb;
-                col += t_stride;
-            }
-            ++i;
-        }
-        rounds_until(q, r + p);
-    }
-}
-
-// Single p, p >= 64, four consecutive ranks per thread.  The work of a round that does not depend
+// A tile of one p >= 64, four consecutive ranks per thread.  The work of a round that does not depend
 // on the rank -- the address of the codes at the window's lower end, the store into the
 // round-major copy -- is done once for four ranks: their four codes are four words at one
 // address, their four entries one aligned 32-bit word of the copy.  A thread whose four ranks
@@ -663,7 +478,7 @@ __device__ __forceinline__ void recv_warp_tile(const Skips skip, const uint32_t 
 // skip, next to the root, at the end of the range: a few dozen tiles of a p) runs the general
 // code, home round and wrap tested per rank, for all its quads.
 //
-// The run table of the tile (see recv_warp_tile) is kept as four sub-tables by position mod 4:
+// The run table of the tile is kept as four sub-tables by position mod 4:
 // entry x (x = -64 .. tile-1, counted from the tile's first rank) is word
 // ((x + 64) mod 4) * kQuadSub + (x + 64) / 4 of its level, so that the threads of a warp, whose
 // ranks are four apart, read consecutive words whatever the distance of the window.
@@ -1160,37 +975,6 @@ recv_quad_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t 
                                              ba.full_tab + (size_t)j * kRow, p, q, r, q - 1, row, col,
                                              (uint64_t)p);
         }
-    }
-    __syncthreads();
-    flush_span(sh.stage, shift, (uint32_t)(sh.span_end - sh.span_begin), recv_out, sh.span_begin);
-}
-
-// Batch: a CTA whose 256 flattened ranks all belong to one p >= 64 (nearly all CTAs when the p
-// are large) runs the warp-cooperative tile with that p's table rows from shared memory; a CTA
-// that straddles several p, or a small p, runs the per-lane search.
-template <bool kColOut>
-__global__ void __launch_bounds__(kTile, 6)
-recv_codes_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t *recv_out,
-                        int8_t *recv_t)
-{
-    __shared__ TileShared sh;
-    __shared__ RunTable runs;
-    PTable unused;
-    RankCtx c = resolve_rank<true>(sh, unused, 0, 0, ba);
-    const uint32_t shift = (uint32_t)(sh.span_begin & 15u);
-    if (sh.j_first == sh.j_last && c.p >= 64u) {             // uniform over the CTA
-        const uint64_t g0 = (uint64_t)blockIdx.x * kTile;
-        const uint32_t n = (uint32_t)(ba.total_ranks - g0 < (uint64_t)kTile ? ba.total_ranks - g0
-                                                                             : (uint64_t)kTile);
-        const uint64_t first = g0 - c.rank0;
-        int8_t *col = kColOut ? recv_t + ba.entry_off[c.pj] + first + threadIdx.x : nullptr;
-        recv_warp_tile<true, kColOut>(SharedSkips{sh.skips[0]}, sh.full[0], c.p, c.q, first, n,
-                                      codes + c.rank0, sh.stage + shift, col, (uint64_t)c.p, runs);
-    } else if (c.valid && c.q > 0) {
-        int8_t *col = kColOut ? recv_t + ba.entry_off[c.pj] + c.r : nullptr;
-        uint8_t *row = sh.stage + shift + (c.entry - sh.span_begin);
-        recv_rounds_codes<true, kColOut>(codes + c.rank0, c.s, c.full, c.p, c.q, c.r, c.q - 1, row,
-                                         col, (uint64_t)c.p);
     }
     __syncthreads();
     flush_span(sh.stage, shift, (uint32_t)(sh.span_end - sh.span_begin), recv_out, sh.span_begin);
