@@ -202,7 +202,8 @@ def _bench_checksum(torch, bcs, flush, hbm_gbs, peak_src, table, steps):
     gbs = tb.numel() / ms / 1e6
     return {"workload": "%.2f GB buffer" % (tb.numel() / 1e9), "ms": ms, "gbs": gbs,
             "roofline": {"bound": "hbm", "kernel": "checksum_kernel", "achieved": gbs,
-                         "peak": hbm_gbs, "unit": "GB/s", "frac": gbs / hbm_gbs, "traffic": None,
+                         "peak": hbm_gbs, "unit": "GB/s", "frac": gbs / hbm_gbs,
+                         "traffic": CHECKSUM_TRAFFIC_BYTES if tb.numel() == 1625648768 else None,
                          "peak_source": peak_src}}
 
 
@@ -517,6 +518,7 @@ RECV_TRAFFIC_BYTES = 4257536 + 238080        # recv_codes_quad_kernel<true,true>
 EXECUTED_INST_PER_RANK = {21: 91 + 477}
 EXPAND_TRAFFIC_BYTES = 1566649856 + 3409408   # expand_kernel, p = 100003, n = 1000
 ALLGATHER_TRAFFIC_BYTES = 753529344 + 3564800  # allgather_kernel, p = 100003, n = 1000
+CHECKSUM_TRAFFIC_BYTES = 1625745664 + 3475200  # checksum_kernel over the 1 625 648 768 B round tables
 
 # Integer operations per rank of the receive-schedule construction as the kernels run it (four
 # ranks per thread share a round's address arithmetic), by q: skip code (3 per level + 5); the six
