@@ -917,7 +917,7 @@ struct QuadBatchShared {
 };
 
 template <bool kColOut>
-__global__ void __launch_bounds__(kQuadThreads, 8)
+__global__ void __launch_bounds__(kQuadThreads, 7)
 recv_quad_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t *recv_out,
                        int8_t *recv_t)
 {
@@ -1246,7 +1246,7 @@ struct SendBatchShared {
     __align__(16) uint8_t stage[kStageBytes];
 };
 
-__global__ void __launch_bounds__(kTrThreads)
+__global__ void __launch_bounds__(kTrThreads, 16)
 send_batch_kernel(BatchArgs ba, const int8_t *__restrict__ recv_t, int8_t *send_out)
 {
     __shared__ SendBatchShared sh;
