@@ -160,6 +160,42 @@ def test_sub_ranges_ragged_tails_and_single_outputs(bcs, fast):
     assert q == 17
 
 
+def test_seeded_p_sweep_full_tables_sub_ranges_and_one_batch(bcs):
+    """About 170 values of p between 64 and 300 000 -- the neighbours of the powers of two, values
+    whose skips contain 33 (six instead of five rounds read from the run table), and 150 seeded
+    log-uniform draws: the full tables, one seeded sub-range each, and all of them in one batch."""
+    rng = np.random.default_rng(20240)
+    edge = [64, 65, 127, 128, 129, 511, 512, 513, 1023, 1025, 2047, 2049, 4095, 4097, 33 * 64, 33 * 64 - 1,
+            33 * 128, 33 * 2048, 33 * 2048 - 5, 65535, 65536, 65537, 131071, 131073, 262143, 262145]
+    draws = np.exp(rng.uniform(np.log(64), np.log(300000), 150)).astype(np.int64)
+    ps = sorted(set(edge + [int(x) for x in draws]))
+    tables = {}
+    for p in ps:
+        want_r, want_s = tables[p] = oracle.full_table(p)
+        recv, send = _build(bcs, p, 0, p)
+        assert np.array_equal(recv, want_r) and np.array_equal(send, want_s), p
+        a = int(rng.integers(0, p - 1))
+        b = int(rng.integers(a + 1, p + 1))
+        recv, send = _build(bcs, p, a, b)
+        assert np.array_equal(recv, want_r[a:b]) and np.array_equal(send, want_s[a:b]), (p, a, b)
+    plan = bcs.bcs_batch_plan(ps)
+    dplan = plan.to("cuda")
+    raw_r, recv = _guarded(plan.total_entries)
+    raw_s, send = _guarded(plan.total_entries)
+    raw_w, ws = _guarded(bcs.bcs_build_batch_workspace_bytes(plan.total_ranks, plan.total_entries))
+    bcs.bcs_build_batch(dplan, plan.total_ranks, plan.total_entries, recv, send, ws)
+    torch.cuda.synchronize()
+    assert bcs.bcs_wait_expired() == 0
+    assert _guards_intact(raw_r, plan.total_entries) and _guards_intact(raw_s, plan.total_entries)
+    assert _guards_intact(raw_w, ws.numel())
+    got_r, got_s = recv.cpu().numpy(), send.cpu().numpy()
+    eo = plan.entry_off.tolist()
+    for j, p in enumerate(ps):
+        want_r, want_s = tables[p]
+        assert np.array_equal(got_r[eo[j]:eo[j + 1]].reshape(p, -1), want_r), p
+        assert np.array_equal(got_s[eo[j]:eo[j + 1]].reshape(p, -1), want_s), p
+
+
 def test_prepare_then_build_ranges(bcs):
     """bcs_prepare once, then receive and send rows of arbitrary ranges by bcs_build_prepared."""
     for p in (2, 3, 33, 63, 64, 1000, 4097, 100003):
