@@ -19,8 +19,11 @@
  *     (scratch memory is passed in by the caller as a `workspace`).
  *   - Schedule tables are int8, rank-major and unpadded: the row of rank r of a
  *     call for ranks r_begin..r_end-1 starts at byte (r - r_begin) * q.
- *   - Errors are return codes.  When a code other than BCS_OK is returned nothing
- *     was enqueued and no output byte was written.
+ *   - Errors are return codes.  Arguments are checked before the first CUDA call: when
+ *     BCS_ERR_ARG, BCS_ERR_RANGE, BCS_ERR_ALIGN or BCS_ERR_UNSUPPORTED is returned nothing
+ *     was enqueued and no output byte was written.  BCS_ERR_CUDA means that the runtime
+ *     refused a launch or a copy in the middle of a call: kernels enqueued before that point
+ *     still run, and the outputs of that call are to be discarded.
  *   - Supported: 1 <= p <= 2^31 - 1 (block sets are 32-bit masks).  p == 1 has
  *     q == 0: every call succeeds and writes nothing.
  *   - An entry that the construction could not determine (Algorithm 4 finding no
@@ -114,8 +117,11 @@ bcs_status bcs_build_prepared(uint32_t p, uint64_t r_begin, uint64_t r_end,
  *   otherwise BCS_ERR_UNSUPPORTED is returned and nothing is written.  Use bcs_build with
  *   your own workspace, or with NULL, beyond that.
  *   First use: the first call on each device asks the CUDA runtime for the array's device
- *   address (with that device current) and remembers it.  Make that first call outside any
- *   stream capture.
+ *   address (with that device current) and remembers it for the life of the process, so do
+ *   not use this entry point across a cudaDeviceReset.  Where the runtime loads the library's
+ *   device code lazily, that first call is also what sets the 8 MiB aside: make it early --
+ *   before other code has claimed the rest of the device memory -- and outside any stream
+ *   capture.  Later calls touch no allocator at all.
  *   Sharing: all calls on a device use the same array.  Two calls whose kernels can overlap
  *   on the GPU (different streams, or several host threads) race on it and produce garbage;
  *   order them on one stream or with events.  The array keeps whatever the last call left
@@ -189,7 +195,14 @@ bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_
  *   x = (q - (n-1+q) mod q) mod q, i = j + x, k = i mod q,
  *   block = sched[k] - x + q * floor(i / q); below 0 -> -1 (nothing is sent or
  *   received), above n-1 -> n-1; to = (r+skips[k]) mod p, from = (r-skips[k]+p) mod p.
- *   recv, send: device int8 rows of exactly these ranks as bcs_build writes them.
+ *   recv, send: device int8 rows of exactly these ranks as bcs_build writes them (the rows
+ *   of the range, not the full [p][q] tables, so that a chunk can be built and expanded
+ *   without the rest), or both NULL: the kernel then computes the rows of its ranks itself,
+ *   as Algorithm 6 does by calling recvsched and sendsched -- each entry by the paper's
+ *   per-rank construction (Algorithm 4 up to that round; the send entry as the receive entry
+ *   of the to-processor, Algorithm 5), O(log^3 p) per rank, without scratch memory.  Meant
+ *   for a few ranks or many rounds; for whole tables build the schedules once with bcs_build.
+ *   One of the two NULL and the other not: BCS_ERR_ARG.
  *   table_out: device, (r_end-r_begin) * (n-1+q) records of 16 bytes, 16-byte
  *   aligned; record of (r, j) at index (r-r_begin)*(n-1+q) + j. */
 bcs_status bcs_expand(uint32_t p, uint32_t n, uint64_t r_begin, uint64_t r_end,
@@ -262,12 +275,16 @@ bcs_status bcs_validate(uint32_t p, uint64_t r_begin, uint64_t r_end,
 bcs_status bcs_simulate(uint32_t p, uint32_t n, const int8_t *recv, const int8_t *send,
                         uint64_t *state_dev, uint64_t *counts_dev, void *cuda_stream);
 
-/* Bounded waits (no counterpart in the paper).  The transposition kernel of bcs_build and
- * bcs_build_prepared waits for its bulk copies on a shared-memory barrier with a poll limit; a
- * CTA whose copies did not arrive within the limit leaves its 256 ranks of the output unwritten
- * and counts itself in a device-wide counter that is never reset.  This call synchronises the
- * device and stores the counter of the current device in *count_host (host): 0 means that
- * every output written so far is complete. */
+/* Bounded waits (no counterpart in the paper).  The transposition kernels of bcs_build,
+ * bcs_build_prepared and bcs_build_batch wait for their bulk copies on a shared-memory barrier
+ * with a poll limit; a CTA whose copies did not arrive within the limit gives up, leaves its
+ * ranks of the output unwritten and counts itself in a device-wide counter that is never
+ * reset.  The build call that enqueued the kernel has long returned BCS_OK by then, so this
+ * poll is the only report.  The call waits for all work of the current device
+ * (cudaDeviceSynchronize, whatever streams it was enqueued on) and then stores the counter in
+ * *count_host (host).  0: every table written so far is complete.  Any increase since the last
+ * reading: discard EVERY table built in between, not only the counted tiles -- a copy that
+ * arrives after its CTA has gone may land in the shared memory of another CTA. */
 bcs_status bcs_wait_expired(uint64_t *count_host);
 
 /* Position-weighted 64-bit checksum of a stretch of schedule entries, additive

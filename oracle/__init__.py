@@ -201,6 +201,22 @@ def expand(p: int, n: int, recv: np.ndarray, send: np.ndarray, r_begin: int = 0,
     return out
 
 
+def expand_rows(p: int, n: int, r_begin: int, recv_rows: np.ndarray, send_rows: np.ndarray) -> np.ndarray:
+    """Algorithm 6 for the processors r_begin, r_begin+1, ... given only THEIR schedule rows
+    ([count][q] each): int32 [count][n-1+q][4], one call of the literal per-processor loop each."""
+    q = q_of(p)
+    recv_rows = np.ascontiguousarray(recv_rows, dtype=np.int8)
+    send_rows = np.ascontiguousarray(send_rows, dtype=np.int8)
+    count = recv_rows.shape[0]
+    assert recv_rows.shape == (count, q) and send_rows.shape == (count, q)
+    out = np.zeros((count, n - 1 + q, 4), dtype=np.int32)
+    fn = _load().bcso_expand_rank
+    for j in range(count):
+        fn(p, n, r_begin + j, _i8(recv_rows[j]), _i8(send_rows[j]),
+           out[j].ctypes.data_as(ctypes.POINTER(ctypes.c_int32)))
+    return out
+
+
 def checksum(buf: np.ndarray, first_index: int = 0) -> int:
     """Order-independent 64-bit checksum of int8 entries (not from the paper)."""
     buf = np.ascontiguousarray(buf, dtype=np.int8).reshape(-1)

@@ -24,7 +24,6 @@ from .binding import (  # noqa: F401
     bcs_circulant_rounds,
     bcs_expand,
     bcs_prepare,
-    bcs_probe_int_rate,
     bcs_prepare_workspace_bytes,
     bcs_q,
     bcs_simulate,

@@ -74,9 +74,6 @@ def lib():
         L.bcs_allgather_tables.restype = i32
         L.bcs_simulate.argtypes = [u32, u32, vp, vp, vp, vp, vp]
         L.bcs_simulate.restype = i32
-        L.bcs_probe_int_rate.argtypes = [i32, u32, vp, _c.POINTER(_c.c_double),
-                                         _c.POINTER(_c.c_float), vp]
-        L.bcs_probe_int_rate.restype = i32
         L.bcs_build_rooted_workspace_bytes.argtypes = [u32, u32, u64, u64]
         L.bcs_build_rooted_workspace_bytes.restype = _c.c_size_t
         L.bcs_build_rooted.argtypes = [u32, u32, u64, u64, vp, vp, vp, _c.c_size_t, vp]
@@ -285,17 +282,6 @@ def bcs_wait_expired() -> int:
     v = _c.c_uint64(0)
     _check(lib().bcs_wait_expired(_c.byref(v)), "bcs_wait_expired")
     return v.value
-
-
-def bcs_probe_int_rate(mix: int, iters: int = 4096, stream=None) -> float:
-    """Measured thread-level integer instructions per second of the current device
-    (mix 0: logic only; 1: logic and multiply-add alternating; 2: logic and addition
-    alternating).  Benchmark helper."""
-    sink = torch.zeros(1, dtype=torch.int32, device="cuda")
-    ops, ms = _c.c_double(0), _c.c_float(0)
-    _check(lib().bcs_probe_int_rate(mix, iters, sink.data_ptr(), _c.byref(ops), _c.byref(ms),
-                                    _stream(stream)), "bcs_probe_int_rate")
-    return ops.value / (ms.value * 1e-3)
 
 
 def bcs_checksum(buf, first_entry_index: int, sum_out, stream=None, n_entries: int | None = None) -> None:

@@ -1,6 +1,7 @@
 // Round tables of the n-block broadcast (arXiv 2205.10072, Algorithm 6 without the
 // Send||Recv): a pure store stream, one 16-byte record per (rank, round).
 #include "bcs_common.cuh"
+#include "paper_path.cuh"
 
 namespace bcs {
 namespace {
@@ -16,6 +17,11 @@ constexpr uint32_t kExpandSharedBytes = 48 * 1024;
 // 128-byte lines of memory wherever the stretch starts (stores that cut lines or 32-byte sectors
 // cost up to a fifth of the write bandwidth), and short rows (few rounds) fill the threads as
 // well as long ones.  Rank, round, entry and phase of a thread's record are kept incrementally.
+// kBuildRows: the caller gave no schedule tables, so the CTA computes the rows of its ranks as
+// Algorithm 6 itself does: the receive entry of round k by running Algorithm 4 up to round k,
+// the send entry as the receive entry of the to-processor (Algorithm 5) -- one (rank, round)
+// pair per thread, the paper's own per-rank construction, no table and no scratch memory.
+template <bool kBuildRows>
 __global__ void __launch_bounds__(kExpandThreads)
 expand_kernel(PTable tab, uint32_t n, uint64_t r_begin, uint64_t r_end, uint32_t ranks_per_cta,
               const int8_t *__restrict__ recv, const int8_t *__restrict__ send,
@@ -24,7 +30,12 @@ expand_kernel(PTable tab, uint32_t n, uint64_t r_begin, uint64_t r_end, uint32_t
     // per rank of the CTA and per round k of a phase: {send entry - x, recv entry - x, to, from}.
     // Algorithm 6 adds q to an entry after each use and starts entries k < x at +q because
     // their first use is in the second phase; both are covered by adding q * floor(i / q).
-    extern __shared__ int4 base[];             // [ranks_per_cta][q]
+    extern __shared__ int4 base[];             // [ranks_per_cta][q], then (kBuildRows) the skips
+    uint32_t *skips_sh = reinterpret_cast<uint32_t *>(base + (size_t)ranks_per_cta * tab.q);
+    if (kBuildRows) {
+        if (threadIdx.x < kRow) skips_sh[threadIdx.x] = tab.s[threadIdx.x];
+        __syncthreads();
+    }
     const uint32_t q = (uint32_t)tab.q;
     const uint32_t p = tab.p;
     const uint32_t rounds = n - 1u + q;
@@ -33,7 +44,8 @@ expand_kernel(PTable tab, uint32_t n, uint64_t r_begin, uint64_t r_end, uint32_t
     const uint64_t count = r_end - r_begin;
     const uint32_t ranks = (uint32_t)(count - j0 < (uint64_t)ranks_per_cta ? count - j0 : (uint64_t)ranks_per_cta);
     {
-        const int8_t *srow = send + j0 * q, *rrow = recv + j0 * q;     // the CTA's rows are contiguous
+        const int8_t *srow = kBuildRows ? nullptr : send + j0 * q;     // the CTA's rows are contiguous
+        const int8_t *rrow = kBuildRows ? nullptr : recv + j0 * q;
         for (uint32_t e = threadIdx.x; e < ranks * q; e += kExpandThreads) {
             const uint32_t g = e / q, k = e - g * q;
             const uint32_t r = (uint32_t)(r_begin + j0 + g);
@@ -41,7 +53,15 @@ expand_kernel(PTable tab, uint32_t n, uint64_t r_begin, uint64_t r_end, uint32_t
             uint32_t to = r + sk;
             if (to >= p) to -= p;
             const uint32_t from = r >= sk ? r - sk : r + p - sk;
-            base[e] = make_int4((int)srow[e] - (int)x, (int)rrow[e] - (int)x, (int)to, (int)from);
+            int sent, received;
+            if (kBuildRows) {
+                received = (int8_t)recv_rounds(skips_sh, p, (int)q, r, (int)k, nullptr);
+                sent = (int8_t)recv_rounds(skips_sh, p, (int)q, to, (int)k, nullptr);
+            } else {
+                sent = srow[e];
+                received = rrow[e];
+            }
+            base[e] = make_int4(sent - (int)x, received - (int)x, (int)to, (int)from);
         }
     }
     __syncthreads();
@@ -129,18 +149,24 @@ bcs_status bcs_expand(uint32_t p, uint32_t n, uint64_t r_begin, uint64_t r_end,
     make_table(p, &tab);
     const uint64_t count = r_end - r_begin;
     if (count == 0 || tab.q == 0) return BCS_OK;
-    if (recv == nullptr || send == nullptr || table_out == nullptr) return BCS_ERR_ARG;
+    if (table_out == nullptr || (recv == nullptr) != (send == nullptr)) return BCS_ERR_ARG;
     if (!aligned16(table_out)) return BCS_ERR_ALIGN;
     // ranks per CTA: about kExpandRecords records, as far as the per-rank constants fit in shared memory
     const uint32_t rounds = n - 1u + (uint32_t)tab.q;
     uint32_t per_cta = (kExpandRecords + rounds - 1) / rounds;
-    const uint32_t fit = kExpandSharedBytes / (16u * (uint32_t)tab.q);
+    const uint32_t extra = recv == nullptr ? kRow * 4u : 0u;     // room for the skips when the rows are built here
+    const uint32_t fit = (kExpandSharedBytes - extra) / (16u * (uint32_t)tab.q);
     if (per_cta > fit) per_cta = fit;
     const uint64_t blocks = (count + per_cta - 1) / per_cta;
     if (blocks > 0x7fffffffull) return BCS_ERR_UNSUPPORTED;
-    expand_kernel<<<(unsigned)blocks, kExpandThreads, (size_t)per_cta * tab.q * 16u,
-                    static_cast<cudaStream_t>(cuda_stream)>>>(
-        tab, n, r_begin, r_end, per_cta, recv, send, reinterpret_cast<int4 *>(table_out));
+    if (recv == nullptr)                               // no tables: the kernel builds the rows it needs
+        expand_kernel<true><<<(unsigned)blocks, kExpandThreads, (size_t)per_cta * tab.q * 16u + kRow * 4u,
+                              static_cast<cudaStream_t>(cuda_stream)>>>(
+            tab, n, r_begin, r_end, per_cta, nullptr, nullptr, reinterpret_cast<int4 *>(table_out));
+    else
+        expand_kernel<false><<<(unsigned)blocks, kExpandThreads, (size_t)per_cta * tab.q * 16u,
+                               static_cast<cudaStream_t>(cuda_stream)>>>(
+            tab, n, r_begin, r_end, per_cta, recv, send, reinterpret_cast<int4 *>(table_out));
     return launch_status();
 }
 

@@ -1,4 +1,4 @@
-// Integer instruction rate probe (measurement helper of the benchmark; see include/bcs_probe.h).
+// Integer instruction rate probe (measurement helper of the benchmark; see bcs_probe.h; built into a library of its own).
 #include "bcs_common.cuh"
 #include "bcs_probe.h"
 

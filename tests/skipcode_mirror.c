@@ -1,0 +1,298 @@
+/*
+ * skipcode_mirror.c -- CPU restatement, with operation counters, of the construction that the
+ * fast CUDA kernels run (TEST INFRASTRUCTURE; shares no code with the kernels or the oracle).
+ *
+ * The kernels do not descend the homeranges as Algorithm 3 of arXiv 2205.10072 does.  They give
+ * every rank x a "skip code": x is written as a sum of distinct skips, largest first (the sums
+ * that Algorithm 2 walks down), and bit k of code(x) says whether skips[k] is a term.  The
+ * lowest set bit is the baseblock of x, the highest its homerange, and codes order like ranks.
+ * The largest baseblock among the ranks x+1..y is then the highest bit in which code(x) and
+ * code(y) differ; everything Algorithm 4 needs per round (the largest block of a window that is
+ * not in B yet) follows from the two codes that bound the window.
+ *
+ * This file computes receive and send rows that way, one rank at a time, in plain C, and counts
+ * the integer operations an ideal translation of each step needs (no address arithmetic beyond
+ * what the step itself requires, no loop overhead).  The tests compare its rows with the
+ * oracle's; the benchmark takes its operation counts as the model numerator of the integer
+ * roofline.  Operations shared by the four consecutive ranks that a GPU thread handles are
+ * counted as a quarter each: all counters are in QUARTER operations.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define SKM_MAX_Q 31
+#define Q4(n) ((uint64_t)(4 * (n)))     /* n whole operations, in quarter operations */
+
+enum {
+    SKM_RANKS = 0,          /* ranks whose receive row was built                                */
+    SKM_CODE_OPS,           /* skip code of the rank itself: compare, subtract, set bit per level */
+    SKM_TABLE_OPS,          /* rounds decided from the window's exact block set (short windows)  */
+    SKM_HEAD_OPS,           /* rounds decided by the first head                                  */
+    SKM_STEP2_OPS,          /* extra work when the first head was taken and the second step decides */
+    SKM_REST_OPS,           /* extra work of the full search and of the second window            */
+    SKM_HOME_OPS,           /* the home round                                                    */
+    SKM_STORE_OPS,          /* row byte and the share of the packed column word, per entry       */
+    SKM_SEND_OPS,           /* send row by lookup in the round-major receive table               */
+    SKM_ROUNDS_TABLE, SKM_ROUNDS_HEAD, SKM_ROUNDS_STEP2, SKM_ROUNDS_REST, SKM_ROUNDS_SECOND,
+    SKM_ROUNDS_HOME,
+    SKM_NCOUNT
+};
+
+typedef struct {
+    uint32_t p;
+    int q;
+    uint32_t s[SKM_MAX_Q + 2];       /* skips[0..q] */
+    uint32_t full[SKM_MAX_Q + 2];    /* full[d] = code(skips[d] - 1) */
+    uint32_t len2[SKM_MAX_Q + 1];    /* ranks in the second window of round i */
+    int table_rounds;                /* rounds 0..table_rounds-1 have windows within 41 ranks */
+    const uint32_t *codes;           /* codes of all ranks when the caller has them, else NULL */
+} skm_ctx;
+
+/* Which rounds are decided from exact window sets: 0 = as the GPU kernels do (the rounds with
+ * skips[i+1] <= 33 when p >= 64), 1 = none (every round by the code search), 2 = those rounds
+ * for every p.  All three must give the same rows. */
+static int g_table_mode = 0;
+void skm_set_table_mode(int mode) { g_table_mode = mode; }
+
+static int top_bit(uint32_t v) { return v ? 31 - __builtin_clz(v) : -1; }
+
+/* Greedy decomposition of x into skips, largest first. */
+static uint32_t code_of(const skm_ctx *c, uint32_t x)
+{
+    if (c->codes) return c->codes[x];
+    uint32_t code = 0;
+    for (int k = c->q - 1; k >= 0; --k)
+        if (x >= c->s[k]) { x -= c->s[k]; code |= 1u << k; }
+    return code;
+}
+
+static void ctx_init(skm_ctx *c, uint32_t p)
+{
+    memset(c, 0, sizeof *c);
+    c->p = p;
+    int q = 0;
+    while (((uint64_t)1 << q) < p) ++q;
+    c->q = q;
+    uint32_t v = p;
+    for (int k = q; k >= 0; --k) { c->s[k] = v; v = (v + 1) / 2; }
+    for (int d = 0; d <= q; ++d) c->full[d] = code_of(c, c->s[d] - 1);
+    uint64_t sum = 0;
+    for (int i = 0; i < q; ++i) {
+        sum += c->s[i];
+        c->len2[i] = sum >= c->s[i + 1] ? (uint32_t)(sum - c->s[i + 1] + 1) : 0;
+    }
+    if (g_table_mode == 2 || (g_table_mode == 0 && p >= 64))
+        while (c->table_rounds < q && c->table_rounds < 6 && c->s[c->table_rounds + 1] <= 33)
+            ++c->table_rounds;
+}
+
+/* Largest block not in B among the baseblocks of the ranks x+1..y, given X = code(x) and
+ * F = code(y), x <= y; -1 if there is none.  *ops is charged with the operations of every
+ * step taken. */
+static int search_codes(const skm_ctx *c, uint32_t X, uint32_t F, uint32_t B, uint64_t *ops)
+{
+    uint32_t low = 0;                       /* blocks 0..m known to be in the range, as a mask */
+    for (;;) {
+        uint32_t diff = X ^ F;              *ops += Q4(2);   /* xor, test */
+        if (diff == 0) break;
+        int d = top_bit(diff);
+        uint32_t bit = 1u << d;             *ops += Q4(3);   /* leading bit, shift, compare with low */
+        if (bit <= low) break;              /* this head and all later ones are already in `low` */
+        *ops += Q4(2);                      /* and, test */
+        if (!(B & bit)) return d;
+        /* behind the head: a copy of the ranks 1..rest(y), which hold the blocks 0..top(rest) */
+        uint32_t rest = F & (bit - 1);      *ops += Q4(2);
+        if (rest) { low |= (2u << top_bit(rest)) - 1; *ops += Q4(4); }
+        /* before the head: rest(x)+1 .. skips[d]-1 inside a copy of 1..skips[d]-1 */
+        X &= bit - 1;
+        F = c->full[d];                     *ops += Q4(2);
+    }
+    uint32_t U = low & ~B;                  *ops += Q4(3);
+    return top_bit(U);
+}
+
+/* The same for the `len` ranks that end at rank e (mod p); the root holds no block. */
+static int search_cyclic(const skm_ctx *c, uint32_t e, uint32_t len, uint32_t B, uint64_t *ops)
+{
+    const uint32_t p = c->p;
+    *ops += Q4(2);
+    if (len == 0) return -1;
+    if (len >= p) return top_bit(((c->q >= 32) ? 0xffffffffu : ((1u << c->q) - 1)) & ~B);
+    if (e >= len) {                          /* ranks e-len+1 .. e, all at least 1 */
+        *ops += Q4(2);                       /* one more code: the rank just before the window */
+        return search_codes(c, code_of(c, e - len), code_of(c, e), B, ops);
+    }
+    /* the window reaches the root: ranks p-(len-e)+1 .. p-1 (if any), then 1 .. e (if any) */
+    uint32_t over = len - e;                 /* ranks at or before the root, root included */
+    int b1 = -1, b2 = -1;
+    *ops += Q4(4);
+    if (over >= 2) b1 = search_codes(c, code_of(c, p - over), c->full[c->q], B, ops);
+    if (e >= 1) b2 = search_codes(c, 0, code_of(c, e), B, ops);
+    return b1 > b2 ? b1 : b2;
+}
+
+/* Exact set of the baseblocks of the `len` ranks ending `back` ranks below r (mod p), root
+ * excluded: what the tile's table of OR-ed baseblock bits delivers for a short window. */
+static uint32_t window_set(const skm_ctx *c, uint32_t r, uint32_t back, uint32_t len)
+{
+    uint32_t set = 0;
+    for (uint32_t j = 0; j < len; ++j) {
+        uint64_t x = ((uint64_t)r + c->p - (back + j) % c->p) % c->p;
+        uint32_t cx = code_of(c, (uint32_t)x);
+        set |= cx & (0u - cx);               /* lowest set bit; 0 for the root */
+    }
+    return set;
+}
+
+/* Receive entries of rounds 0..last of rank r (Algorithm 4 on skip codes). */
+static void recv_row(const skm_ctx *c, uint32_t r, int last, int8_t *row, uint64_t *cnt)
+{
+    const uint32_t p = c->p;
+    const int q = c->q;
+    uint32_t own = code_of(c, r);
+    int h = top_bit(own);                     /* homerange; -1 for the root */
+    int bb = own ? __builtin_ctz(own) : 0;    /* baseblock */
+    uint32_t B = own ? 1u << bb : 0;
+    if (cnt) {
+        cnt[SKM_RANKS] += 1;
+        cnt[SKM_CODE_OPS] += Q4(3 * q + 3);   /* per level compare, subtract, or; then h, bb, B */
+    }
+    uint64_t dummy[SKM_NCOUNT];
+    if (!cnt) { memset(dummy, 0, sizeof dummy); cnt = dummy; }
+    for (int i = 0; i <= last; ++i) {
+        const uint32_t lo = c->s[i], hi = c->s[i + 1];
+        int entry;
+        if (i == h) {
+            entry = bb;                                            /* the baseblock itself */
+            cnt[SKM_HOME_OPS] += Q4(1);
+            cnt[SKM_ROUNDS_HOME] += 1;
+        } else if (i < c->table_rounds) {
+            /* Short windows: both windows as exact block sets (on the GPU four words of the
+             * tile's run table: 4 loads, 2 or, 2 and-not), first window unless it is empty of
+             * new blocks (1 select), then leading bit, its mask, entry, set update. */
+            uint32_t U = window_set(c, r, lo, hi - lo) & ~B;
+            if (U == 0 && c->len2[i]) U = window_set(c, r, hi, c->len2[i]) & ~B;
+            cnt[SKM_TABLE_OPS] += Q4(4 + 2 + 2 + 1 + 4);
+            cnt[SKM_ROUNDS_TABLE] += 1;
+            int blk = top_bit(U);
+            if (blk >= 0) B |= 1u << blk;
+            entry = blk >= 0 ? blk - q : 127;
+        } else {
+            /* window of round i: the ranks below+1 .. above with below = r - skips[i+1],
+             * above = r - skips[i] (both mod p; both wrapped past the home round, neither before) */
+            const uint32_t below = (uint32_t)(((uint64_t)r + p - hi) % p);
+            const uint32_t above = (uint32_t)(((uint64_t)r + p - lo) % p);
+            const uint32_t lower = code_of(c, below), upper = code_of(c, above);
+            /* address of the lower code: shared by the four ranks of a thread (1/4); its load;
+             * the upper code is last round's lower one */
+            cnt[SKM_HEAD_OPS] += 1 + Q4(1);
+            const uint32_t diff = lower ^ upper;
+            const int d = top_bit(diff);
+            const uint32_t bit = d >= 0 ? 1u << d : 0;
+            const uint32_t fresh = bit & ~B;
+            cnt[SKM_HEAD_OPS] += Q4(5 + 2);      /* xor, leading bit, shift, and-not, test; or into B, entry */
+            int blk;
+            if (fresh) {
+                blk = d;
+                cnt[SKM_ROUNDS_HEAD] += 1;
+            } else {
+                /* second step of the search, decided without a loop when it ends there: the
+                 * head is taken, the run of low blocks behind it has a new block, and the next
+                 * head (before the first one) is not above that run */
+                blk = -1;
+                int decided = 0;
+                if (diff != 0) {
+                    const uint32_t below_head = bit - 1;
+                    const uint32_t rest = upper & below_head;
+                    const uint32_t low = rest ? (2u << top_bit(rest)) - 1 : 0;
+                    const uint32_t diff2 = (lower & below_head) ^ c->full[d];
+                    const uint32_t news = low & ~B;
+                    cnt[SKM_STEP2_OPS] += Q4(12);
+                    if (news != 0 && (diff2 == 0 || (1u << top_bit(diff2)) <= low)) {
+                        blk = top_bit(news);
+                        decided = 1;
+                        cnt[SKM_ROUNDS_STEP2] += 1;
+                    }
+                }
+                if (!decided) {
+                    cnt[SKM_ROUNDS_REST] += 1;
+                    blk = diff ? search_codes(c, lower, upper, B, &cnt[SKM_REST_OPS]) : -1;
+                    if (blk < 0) {
+                        cnt[SKM_ROUNDS_SECOND] += 1;
+                        blk = search_cyclic(c, below, c->len2[i], B, &cnt[SKM_REST_OPS]);
+                    }
+                }
+            }
+            if (blk >= 0) B |= 1u << blk;
+            entry = blk >= 0 ? blk - q : 127;
+        }
+        /* the entry's byte in the rank-major row, and its share of the round's packed word of
+         * four ranks in the round-major copy (3 byte merges and 1 store per four entries) */
+        cnt[SKM_STORE_OPS] += Q4(1) + 4;
+        if (row) row[i] = (int8_t)entry;
+    }
+}
+
+/* ------------------------------------------------------------------------------------ API */
+int skm_q(uint32_t p)
+{
+    skm_ctx c;
+    ctx_init(&c, p);
+    return c.q;
+}
+
+/* Receive and send rows of the listed ranks.  recv, send: n * q bytes, rank-major; either may
+ * be NULL.  A send entry is the receive entry of the to-processor in that round; the counters
+ * charge it as the GPU obtains it -- a lookup in the round-major receive table (per four
+ * entries two word loads, a funnel shift, three byte merges and a store: 7/4 per entry). */
+int skm_rows(uint32_t p, const uint64_t *ranks, uint64_t n, int8_t *recv, int8_t *send,
+             uint64_t *counters /* SKM_NCOUNT, accumulated */)
+{
+    if (p == 0 || p > 0x7fffffffu) return -1;
+    skm_ctx c;
+    ctx_init(&c, p);
+    const int q = c.q;
+    int8_t tmp[SKM_MAX_Q + 1];
+    for (uint64_t m = 0; m < n; ++m) {
+        const uint32_t r = (uint32_t)ranks[m];
+        if (r >= p) return -2;
+        if (recv) recv_row(&c, r, q - 1, recv + m * (uint64_t)q, counters);
+        else recv_row(&c, r, q - 1, tmp, counters);
+        if (send) {
+            for (int k = 0; k < q; ++k) {
+                const uint32_t to = (uint32_t)(((uint64_t)r + c.s[k]) % p);
+                recv_row(&c, to, k, tmp, NULL);
+                send[m * (uint64_t)q + k] = tmp[k];
+                if (counters) counters[SKM_SEND_OPS] += 7;
+            }
+        }
+    }
+    return 0;
+}
+
+/* All ranks of p: recv and send are p * q bytes each (send may be NULL). */
+int skm_full(uint32_t p, int8_t *recv, int8_t *send, uint64_t *counters)
+{
+    if (p == 0 || p > 0x7fffffffu || recv == NULL) return -1;
+    skm_ctx c;
+    ctx_init(&c, p);
+    const int q = c.q;
+    uint32_t *codes = (uint32_t *)malloc((size_t)p * sizeof(uint32_t));
+    if (codes == NULL) return -3;
+    for (uint32_t x = 0; x < p; ++x) codes[x] = code_of(&c, x);
+    c.codes = codes;
+    for (uint32_t r = 0; r < p; ++r) recv_row(&c, r, q - 1, recv + (uint64_t)r * q, counters);
+    free(codes);
+    if (send) {
+        for (uint32_t r = 0; r < p; ++r)
+            for (int k = 0; k < q; ++k) {
+                const uint32_t to = (uint32_t)(((uint64_t)r + c.s[k]) % p);
+                send[(uint64_t)r * q + k] = recv[(uint64_t)to * q + k];
+            }
+        if (counters) counters[SKM_SEND_OPS] += 7ull * p * q;
+    }
+    return 0;
+}
+
+int skm_ncount(void) { return SKM_NCOUNT; }

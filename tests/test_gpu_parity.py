@@ -365,8 +365,13 @@ def test_build_to_host_matches(bcs):
 
 
 def test_batched_irregular_sweep_full_size(bcs):
-    """4096 octave-uniform p in [2^10, 2^20): the launch the benchmark uses.  Full tables are
-    compared for a spread of p, seeded sample ranks for every p."""
+    """4096 octave-uniform p in [2^10, 2^20): the launch the benchmark uses, 639 M ranks and
+    24 GB of tables.  EVERY table is compared byte for byte with the oracle's array form (about
+    a minute and a half of host time); for every p >= 2^16, 10^4 seeded ranks plus the ranks
+    skips[k]-2 .. skips[k]+2 of every k (where the receive kernel switches to its general tile
+    code), the root's neighbours and the last ranks are compared with the oracle's per-rank form
+    as well, which shares nothing with the array form but Algorithms 1 and 2; and the library's
+    property checker runs over every rank of every p."""
     plist = workloads.batch_p_list()
     plan = bcs.bcs_batch_plan(plist)
     assert plan.total_ranks == 639466253
@@ -377,25 +382,39 @@ def test_batched_irregular_sweep_full_size(bcs):
                      dtype=torch.int8, device="cuda")
     bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, send, ws)
     torch.cuda.synchronize()
+    assert bcs.bcs_wait_expired() == 0
     del ws
     eo = plan.entry_off.tolist()
-    order = sorted(range(len(plist)), key=lambda j: plist[j])
-    full = set(order[:24] + order[-3:] + order[::300] + list(range(6)))
-    for j in sorted(full):
-        p, q = plist[j], oracle.q_of(plist[j])
-        want_r, want_s = oracle.full_table(p)
-        assert np.array_equal(recv[eo[j]:eo[j + 1]].cpu().numpy().reshape(p, q), want_r), p
-        assert np.array_equal(send[eo[j]:eo[j + 1]].cpu().numpy().reshape(p, q), want_s), p
+    viol = torch.zeros(3, dtype=torch.int64, device="cuda")
+    total_viol = torch.zeros(3, dtype=torch.int64, device="cuda")
     rng = np.random.default_rng(220510072)
+    cache = {}
     for j, p in enumerate(plist):
-        if j in full:
-            continue
         q = oracle.q_of(p)
-        ranks = np.unique(np.concatenate([rng.integers(0, p, 48), [0, 1, p - 1]]))
-        want_r, want_s = oracle.build_ranks(p, ranks)
-        idx = (torch.from_numpy(ranks)[:, None] * q + torch.arange(q)[None, :] + eo[j]).cuda()
-        assert np.array_equal(recv[idx].cpu().numpy(), want_r), p
-        assert np.array_equal(send[idx].cpu().numpy(), want_s), p
+        got_r, got_s = recv[eo[j]:eo[j + 1]], send[eo[j]:eo[j + 1]]
+        if p not in cache:                       # duplicates of p are allowed in the list
+            want_r, want_s = oracle.full_table(p)
+            cache[p] = (torch.from_numpy(want_r).cuda().view(-1), torch.from_numpy(want_s).cuda().view(-1))
+        assert torch.equal(got_r, cache[p][0]), (j, p)
+        assert torch.equal(got_s, cache[p][1]), (j, p)
+        if p < 2**16:
+            del cache[p]                         # keep only what a duplicate could ask for again
+        else:
+            sk = oracle.skips(p)
+            near = np.concatenate([sk[k] + np.arange(-2, 3) for k in range(q + 1)] + [[0, 1, 2]]) % p
+            ranks = np.unique(np.concatenate([rng.integers(0, p, 10000), near]))
+            want_r, want_s = oracle.build_ranks(p, ranks)
+            idx = (torch.from_numpy(ranks)[:, None] * q + torch.arange(q)[None, :]).cuda()
+            assert np.array_equal(got_r[idx].cpu().numpy(), want_r), p
+            assert np.array_equal(got_s[idx].cpu().numpy(), want_s), p
+            if len(cache) > 64:
+                cache.clear()
+        # bcs_validate wants 16-byte aligned tables; a table of the batch starts at any byte
+        if eo[j] % 16 != 0:
+            got_r, got_s = got_r.clone(), got_s.clone()
+        bcs.bcs_validate(p, 0, p, got_r, got_s, viol)
+        total_viol += viol
+    assert total_viol.cpu().tolist() == [0, 0, 0]
 
 
 def test_expansion_full_size(bcs):
@@ -437,6 +456,34 @@ def test_expansion_small_cases_and_simulation(bcs):
             assert np.array_equal(got, oracle.expand(p, n, want_r, want_s)), (p, n)
             if n <= 40:
                 assert bcast_sim.simulate(p, n, got) is None
+
+
+def test_expansion_builds_its_rows_when_given_no_tables(bcs):
+    """bcs_expand with both tables NULL computes the rows of its ranks itself (Algorithm 6 calls
+    recvsched and sendsched): same records as the oracle's literal loop, for whole small p, for
+    sub-ranges around the root and the skips of larger p, and for the expansion workload's p."""
+    for p in (2, 3, 9, 20, 33, 257, 1000):
+        q = oracle.q_of(p)
+        want_r, want_s = oracle.full_table(p)
+        for n in (1, 5, q + 3, 3 * q + 2):
+            raw = torch.full((p * (n - 1 + q) * 4 + 128,), -77, dtype=torch.int32, device="cuda")
+            tab = raw[64:64 + p * (n - 1 + q) * 4].view(p, n - 1 + q, 4)
+            bcs.bcs_expand(p, n, 0, p, None, None, tab)
+            torch.cuda.synchronize()
+            assert bool((raw[:64] == -77).all()) and bool((raw[-64:] == -77).all())
+            assert np.array_equal(tab.cpu().numpy(), oracle.expand(p, n, want_r, want_s)), (p, n)
+    for p, n, r0, r1 in ((workloads.P_EXPAND, workloads.N_EXPAND, 50000, 50100),
+                         (workloads.P_EXPAND, 7, 0, 3000), (workloads.P_EXPAND, 40, 99000, 100003),
+                         (workloads.P_SINGLE, 30, 2**19 - 50, 2**19 + 200),
+                         (workloads.P_LARGE, 12, 2**29 - 20, 2**29 + 20), (2**31 - 1, 3, 0, 40)):
+        q = oracle.q_of(p)
+        want_r, want_s = oracle.build_range(p, r0, r1)
+        tab = torch.empty((r1 - r0, n - 1 + q, 4), dtype=torch.int32, device="cuda")
+        bcs.bcs_expand(p, n, r0, r1, None, None, tab)
+        torch.cuda.synchronize()
+        assert np.array_equal(tab.cpu().numpy(), oracle.expand_rows(p, n, r0, want_r, want_s)), (p, n, r0)
+    L = bcs.lib()
+    assert L.bcs_expand(10, 4, 0, 10, None, tab.data_ptr(), tab.data_ptr(), None) == 1   # one table only
 
 
 def test_allgather_tables_match_oracle(bcs):

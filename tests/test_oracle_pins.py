@@ -395,6 +395,34 @@ def test_validator_accepts_valid_and_counts_planted_mistakes():
     assert oracle.validate(p, 20, 21, recv[20:21], bad[20:21]) == (0, 1, 0)  # to-processor outside
 
 
+def test_validator_agrees_with_the_independent_set_based_checker():
+    """oracle.validate (C, bit masks) against tests/schedule_props.py (Python sets, written from
+    the sentences after Theorem 1, own skips and baseblock list): identical counts on valid tables
+    and on several hundred randomly corrupted ones, whole tables and sub-ranges, with both
+    tables or one."""
+    from tests import schedule_props
+    rng = np.random.default_rng(31)
+    right = load(SECOND_P9)
+    assert schedule_props.count_violations(9, 0, 9, right["recv"], right["send"]) == (0, 0, 0)
+    compared = 0
+    for p, r0, r1 in ((2, 0, 2), (3, 0, 3), (9, 0, 9), (20, 0, 20), (31, 0, 31), (32, 0, 32),
+                      (33, 0, 33), (100, 0, 100), (257, 0, 257), (1000, 0, 1000),
+                      (1000, 100, 900), (4097, 4000, 4097), (4097, 0, 300)):
+        q = oracle.q_of(p)
+        full_recv, full_send = oracle.full_table(p)
+        assert schedule_props.count_violations(p, 0, p, full_recv, full_send) == (0, 0, 0), p
+        for _ in range(24):
+            recv, send = full_recv[r0:r1].copy(), full_send[r0:r1].copy()
+            for _ in range(rng.integers(1, 12)):
+                tbl = recv if rng.integers(2) else send
+                tbl[rng.integers(r1 - r0), rng.integers(q)] = rng.integers(-q - 1, q + 1)
+            for a, b in ((recv, send), (recv, None), (None, send)):
+                assert oracle.validate(p, r0, r1, a, b) == \
+                    schedule_props.count_violations(p, r0, r1, a, b), (p, r0, r1)
+                compared += 1
+    assert compared > 900
+
+
 def test_oracle_simulator_agrees_with_the_numpy_simulation():
     """oracle.simulate (C, counts) against tests/bcast_sim.py (numpy, independent skips and round
     semantics): zero counts exactly when the numpy simulation accepts, on valid and on corrupted

@@ -1,13 +1,16 @@
 """bcs_build_static: the entry point for callers that can neither allocate device memory nor
 pass a workspace (it uses an 8 MiB scratch array that is part of the library).  Its tables must
-be byte-identical to those of bcs_build, call after call, although every call reuses the same
-scratch and finds the previous call's leftovers in it.
+be byte-identical to those of bcs_build and to the CPU oracle's, call after call, although every
+call reuses the same scratch and finds the previous call's leftovers in it.
 
 This file sorts last on purpose: a run that stops at the first failure has then already gone
 through every other test.  It does not depend on them: it also passes alone in a fresh process.
 """
+import numpy as np
 import pytest
 import torch
+
+import oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -32,6 +35,18 @@ def _reference(bcs, p, r0, r1):
     return recv, send
 
 
+_oracle_tables = {}
+
+
+def _oracle_rows(p, r0, r1):
+    """Rows r0..r1-1 of the oracle's tables (array form), as flat int8 CUDA tensors."""
+    if p not in _oracle_tables:
+        _oracle_tables[p] = oracle.full_table(p)
+    recv, send = _oracle_tables[p]
+    return (torch.from_numpy(np.ascontiguousarray(recv[r0:r1])).cuda().view(-1),
+            torch.from_numpy(np.ascontiguousarray(send[r0:r1])).cuda().view(-1))
+
+
 def test_static_scratch_matches_bcs_build_on_consecutive_calls(bcs):
     L = bcs.lib()
     limit = 8 << 20
@@ -50,12 +65,17 @@ def test_static_scratch_matches_bcs_build_on_consecutive_calls(bcs):
         torch.cuda.synchronize()
         assert torch.equal(recv, want_recv), (p, r0, r1)     # integer tables: bit-exact
         assert torch.equal(send, want_send), (p, r0, r1)
+        oracle_recv, oracle_send = _oracle_rows(p, r0, r1)   # and against the CPU oracle
+        assert torch.equal(recv, oracle_recv), (p, r0, r1)
+        assert torch.equal(send, oracle_send), (p, r0, r1)
     # one output only
     want_recv, want_send = _reference(bcs, 100003, 5, 7000)
     send = torch.empty_like(want_send)
     bcs.bcs_build_static(100003, 5, 7000, None, send)
     torch.cuda.synchronize()
     assert torch.equal(send, want_send)
+    assert torch.equal(send, _oracle_rows(100003, 5, 7000)[1])
+    _oracle_tables.clear()
 
 
 def test_static_scratch_rejects_what_does_not_fit(bcs):
