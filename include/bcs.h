@@ -99,6 +99,20 @@ bcs_status bcs_build(uint32_t p, uint64_t r_begin, uint64_t r_end,
  * as for bcs_build; a workspace that is NULL or too small is BCS_ERR_ARG. */
 size_t bcs_prepare_workspace_bytes(uint32_t p);
 bcs_status bcs_prepare(uint32_t p, void *workspace, size_t workspace_bytes, void *cuda_stream);
+/* bcs_prepare in two steps, for callers that want the rank-major receive rows of a chunk straight
+ * from the construction instead of from a transposition afterwards:
+ *   bcs_prepare_codes writes the skip codes of ALL ranks of p into the workspace;
+ *   bcs_prepare_rows then runs Algorithm 4 for the ranks r_begin..r_end-1: their entries go into
+ *   the round-major copy in the workspace and, if recv_out is not NULL, their rank-major rows to
+ *   recv_out (device, (r_end-r_begin)*q bytes, 16-byte aligned).  r_begin must be a multiple of
+ *   16 (BCS_ERR_ALIGN).  Chunks may be prepared in any order; once every rank of p has been
+ *   through bcs_prepare_rows the workspace is what bcs_prepare leaves, and bcs_build_prepared
+ *   gives the send rows of any range (sendsched[r][k] = recvsched[(r+skips[k]) mod p][k] reaches
+ *   into other chunks, hence only then).
+ * bcs_prepare(p, ...) is bcs_prepare_codes followed by bcs_prepare_rows(p, 0, p, NULL, ...). */
+bcs_status bcs_prepare_codes(uint32_t p, void *workspace, size_t workspace_bytes, void *cuda_stream);
+bcs_status bcs_prepare_rows(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_out,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream);
 bcs_status bcs_build_prepared(uint32_t p, uint64_t r_begin, uint64_t r_end,
                               int8_t *recv_out, int8_t *send_out,
                               const void *workspace, size_t workspace_bytes, void *cuda_stream);

@@ -24,6 +24,8 @@ from .binding import (  # noqa: F401
     bcs_circulant_rounds,
     bcs_expand,
     bcs_prepare,
+    bcs_prepare_codes,
+    bcs_prepare_rows,
     bcs_prepare_workspace_bytes,
     bcs_q,
     bcs_simulate,

@@ -52,6 +52,10 @@ def lib():
         L.bcs_prepare_workspace_bytes.restype = _c.c_size_t
         L.bcs_prepare.argtypes = [u32, vp, _c.c_size_t, vp]
         L.bcs_prepare.restype = i32
+        L.bcs_prepare_codes.argtypes = [u32, vp, _c.c_size_t, vp]
+        L.bcs_prepare_codes.restype = i32
+        L.bcs_prepare_rows.argtypes = [u32, u64, u64, vp, vp, _c.c_size_t, vp]
+        L.bcs_prepare_rows.restype = i32
         L.bcs_build_prepared.argtypes = [u32, u64, u64, vp, vp, vp, _c.c_size_t, vp]
         L.bcs_build_prepared.restype = i32
         L.bcs_build_static.argtypes = [u32, u64, u64, vp, vp, vp]
@@ -152,6 +156,19 @@ def bcs_prepare(p: int, workspace, stream=None) -> None:
     """Runs the construction once for all ranks of p into `workspace` (CUDA tensor of
     bcs_prepare_workspace_bytes(p) bytes) for later bcs_build_prepared calls."""
     _check(lib().bcs_prepare(p, _ptr(workspace), _nbytes(workspace), _stream(stream)), "bcs_prepare")
+
+
+def bcs_prepare_codes(p: int, workspace, stream=None) -> None:
+    """First half of bcs_prepare: the skip codes of all ranks of p into `workspace`."""
+    _check(lib().bcs_prepare_codes(p, _ptr(workspace), _nbytes(workspace), _stream(stream)),
+           "bcs_prepare_codes")
+
+
+def bcs_prepare_rows(p: int, r_begin: int, r_end: int, recv_out, workspace, stream=None) -> None:
+    """Second half, for one range (r_begin a multiple of 16): its entries into the round-major copy
+    in `workspace` and, if recv_out is not None, its rank-major receive rows into recv_out."""
+    _check(lib().bcs_prepare_rows(p, r_begin, r_end, _ptr(recv_out), _ptr(workspace),
+                                  _nbytes(workspace), _stream(stream)), "bcs_prepare_rows")
 
 
 def bcs_build_prepared(p: int, r_begin: int, r_end: int, recv_out, send_out, workspace,

@@ -1322,30 +1322,69 @@ size_t bcs_prepare_workspace_bytes(uint32_t p)
     return (size_t)(align_up(4ull * p, 256) + (uint64_t)q * align_up(p, 16));
 }
 
-bcs_status bcs_prepare(uint32_t p, void *workspace, size_t workspace_bytes, void *cuda_stream)
+// The two halves of bcs_prepare.  Layout of the workspace: skip codes of all p ranks, then the
+// round-major copy recv_t[k * align16(p) + r].
+static bcs_status prepare_check(uint32_t p, PTable *tab, const void *workspace, size_t workspace_bytes)
 {
-    PTable tab;
-    bcs_status st = make_table(p, &tab);
+    bcs_status st = make_table(p, tab);
     if (st != BCS_OK) return st;
-    if (tab.q == 0) return BCS_OK;
+    if (tab->q == 0) return BCS_OK;
     if (workspace == nullptr || workspace_bytes < bcs_prepare_workspace_bytes(p)) return BCS_ERR_ARG;
     if (!aligned16(workspace)) return BCS_ERR_ALIGN;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    uint32_t *codes = static_cast<uint32_t *>(workspace);
-    int8_t *recv_t = static_cast<int8_t *>(workspace) + align_up(4ull * p, 256);
-    const uint64_t t_stride = align_up(p, 16);
-    const unsigned blocks = (unsigned)((p + kTile - 1) / kTile);
-    launch_codes(tab, codes, stream);
-    if ((st = launch_status()) != BCS_OK) return st;
-    if (p >= 64) {
-        const QuadConsts qc = make_quad_consts(tab, 0, p);
-        launch_dependent(true, recv_codes_quad_kernel<false, true>,
-                         (p + kQuadTile - 1) / kQuadTile + (unsigned)qc.n_special, kQuadThreads, stream, tab, qc,
-                         (uint64_t)0, (uint64_t)p, codes, nullptr, recv_t, t_stride);
-    } else
-        recv_codes_kernel<false, true><<<blocks, kTile, 0, stream>>>(tab, 0, p, codes, nullptr,
-                                                                     recv_t, t_stride);
+    return BCS_OK;
+}
+
+bcs_status bcs_prepare_codes(uint32_t p, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    PTable tab;
+    bcs_status st = prepare_check(p, &tab, workspace, workspace_bytes);
+    if (st != BCS_OK || tab.q == 0) return st;
+    launch_codes(tab, static_cast<uint32_t *>(workspace), static_cast<cudaStream_t>(cuda_stream));
     return launch_status();
+}
+
+bcs_status bcs_prepare_rows(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_out,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    bcs_status st = check_range(p, r_begin, r_end);
+    if (st != BCS_OK) return st;
+    PTable tab;
+    st = prepare_check(p, &tab, workspace, workspace_bytes);
+    if (st != BCS_OK || tab.q == 0 || r_begin == r_end) return st;
+    if ((r_begin & 15u) != 0 || !aligned16(recv_out)) return BCS_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const uint32_t *codes = static_cast<const uint32_t *>(workspace);
+    const uint64_t t_stride = align_up(p, 16);
+    // round k of rank r_begin + j goes to recv_t[k * t_stride + r_begin + j]
+    int8_t *recv_t = static_cast<int8_t *>(workspace) + align_up(4ull * p, 256) + r_begin;
+    const uint64_t count = r_end - r_begin;
+    if (p >= 64) {
+        const QuadConsts qc = make_quad_consts(tab, r_begin, r_end);
+        const unsigned grid = (unsigned)((count + kQuadTile - 1) / kQuadTile) + (unsigned)qc.n_special;
+        // (dependent launch: harmless when the kernel before it on the stream is not the codes kernel)
+        if (recv_out != nullptr)
+            launch_dependent(true, recv_codes_quad_kernel<true, true>, grid, kQuadThreads, stream, tab, qc, r_begin,
+                             r_end, codes, recv_out, recv_t, t_stride);
+        else
+            launch_dependent(true, recv_codes_quad_kernel<false, true>, grid, kQuadThreads, stream, tab, qc, r_begin,
+                             r_end, codes, nullptr, recv_t, t_stride);
+    } else {
+        const unsigned blocks = (unsigned)((count + kTile - 1) / kTile);
+        if (recv_out != nullptr)
+            recv_codes_kernel<true, true><<<blocks, kTile, 0, stream>>>(tab, r_begin, r_end, codes, recv_out, recv_t,
+                                                                        t_stride);
+        else
+            recv_codes_kernel<false, true><<<blocks, kTile, 0, stream>>>(tab, r_begin, r_end, codes, nullptr, recv_t,
+                                                                         t_stride);
+    }
+    return launch_status();
+}
+
+bcs_status bcs_prepare(uint32_t p, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    bcs_status st = bcs_prepare_codes(p, workspace, workspace_bytes, cuda_stream);
+    if (st != BCS_OK) return st;
+    return bcs_prepare_rows(p, 0, p, nullptr, workspace, workspace_bytes, cuda_stream);
 }
 
 bcs_status bcs_build_prepared(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_out,

@@ -32,7 +32,7 @@ def test_every_declared_symbol_is_exported(lib):
     assert {"bcs_build", "bcs_build_batch", "bcs_expand", "bcs_checksum", "bcs_skips", "bcs_q",
             "bcs_batch_plan", "bcs_status_str", "bcs_build_to_host", "bcs_build_workspace_bytes",
             "bcs_build_batch_workspace_bytes", "bcs_validate", "bcs_build_static", "bcs_simulate", "bcs_prepare",
-            "bcs_build_prepared", "bcs_prepare_workspace_bytes", "bcs_allgather_tables", "bcs_circulant_rounds"} <= set(names)
+            "bcs_build_prepared", "bcs_prepare_workspace_bytes", "bcs_prepare_codes", "bcs_prepare_rows", "bcs_allgather_tables", "bcs_circulant_rounds"} <= set(names)
     dll = ctypes.CDLL(lib.lib_path())
     for n in names:
         assert hasattr(dll, n), n

@@ -226,6 +226,47 @@ def test_prepare_then_build_ranges(bcs):
     assert bcs.bcs_prepare_workspace_bytes(20) == 256 + 5 * 32
 
 
+def test_prepare_in_two_steps_chunk_by_chunk(bcs):
+    """bcs_prepare_codes, then bcs_prepare_rows chunk by chunk (in a shuffled order, chunk
+    boundaries at multiples of 16 that are not multiples of the kernels' tiles), each chunk's
+    receive rows taken straight from the construction; then the send rows of every chunk by
+    bcs_build_prepared, and the receive rows once more by transposition: all equal the oracle's."""
+    rng = np.random.default_rng(5)
+    for p, step in ((33, 16), (63, 32), (64, 16), (1000, 304), (4097, 1008), (100003, 30000),
+                    (workloads.P_SINGLE, 333328)):
+        q = oracle.q_of(p)
+        want_r, want_s = oracle.full_table(p)
+        raw_w, ws = _guarded(bcs.bcs_prepare_workspace_bytes(p))
+        bcs.bcs_prepare_codes(p, ws)
+        chunks = [(a, min(p, a + step)) for a in range(0, p, step)]
+        for c in rng.permutation(len(chunks)):
+            r0, r1 = chunks[c]
+            raw_r, recv = _guarded((r1 - r0) * q)
+            if c % 3 == 2:
+                bcs.bcs_prepare_rows(p, r0, r1, None, ws)        # round-major copy only
+            else:
+                bcs.bcs_prepare_rows(p, r0, r1, recv, ws)
+                torch.cuda.synchronize()
+                assert _guards_intact(raw_r, (r1 - r0) * q)
+                assert np.array_equal(recv.cpu().numpy().reshape(-1, q), want_r[r0:r1]), (p, r0, r1)
+        for r0, r1 in chunks:
+            raw_s, send = _guarded((r1 - r0) * q)
+            raw_r, recv = _guarded((r1 - r0) * q)
+            bcs.bcs_build_prepared(p, r0, r1, recv, send, ws)
+            torch.cuda.synchronize()
+            assert _guards_intact(raw_s, (r1 - r0) * q) and _guards_intact(raw_w, ws.numel())
+            assert np.array_equal(send.cpu().numpy().reshape(-1, q), want_s[r0:r1]), (p, r0, r1)
+            assert np.array_equal(recv.cpu().numpy().reshape(-1, q), want_r[r0:r1]), (p, r0, r1)
+    assert bcs.bcs_wait_expired() == 0
+    L = bcs.lib()
+    small = torch.zeros(4096, dtype=torch.int8, device="cuda")
+    assert L.bcs_prepare_rows(1000, 8, 100, small.data_ptr(), ws.data_ptr(), ws.numel(), None) == 3   # r_begin % 16
+    assert L.bcs_prepare_rows(1000, 16, 1001, small.data_ptr(), ws.data_ptr(), ws.numel(), None) == 2
+    assert L.bcs_prepare_rows(1000, 16, 100, small.data_ptr(), small.data_ptr(), 64, None) == 1        # too small
+    assert L.bcs_prepare_codes(1000, small.data_ptr(), 64, None) == 1
+    assert L.bcs_prepare_codes(1, None, 0, None) == 0
+
+
 def test_rooted_builds_are_the_renumbered_schedule(bcs):
     """Section 2: a broadcast from root rho uses the rank-0-rooted rows of virtual rank
     (r - rho) mod p.  Full and partial ranges, runs that pass virtual rank p-1 on and off a
