@@ -1,16 +1,21 @@
 #!/usr/bin/env python
 """Benchmark of the schedule construction on one B200 (or N independent replicas).
 
-A step = one bcs_build call for every rank of p = 2^20 + 1 (q = 21): the receive and the send
-schedule, 2 * 21 int8 entries per rank.  The metric is schedule ranks built per second.
+Headline workload: the large single p = 2^30 - 1 (q = 30), all ranks, receive and send schedule
+(64.4 GB of int8 tables), built in 8 rank chunks through one reused chunk buffer.  A step =
+bcs_prepare_codes + 8 x bcs_prepare_rows + 8 x bcs_build_prepared.  The metric is schedule ranks
+built per second.  The other workloads (single p = 2^20+1, the two batched sweeps, the round-table
+expansion) are timed beside it, each with its roofline block and the oracle's time on the host.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--only PART]
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on the host cores.
+`--only PART` runs one small part alone (the profiler-friendly runs that profiles/ cites).
 """
 from __future__ import annotations
 
 import argparse
+import ctypes
 import json
 import os
 import statistics
@@ -24,13 +29,12 @@ if ROOT not in sys.path:
 
 METRIC = "schedule ranks built/sec (int8 recv+send, q entries)"
 UNIT = "ranks/s"
-
-# Peak of the integer pipes that the schedule kernels are measured against: INT32 lanes per SM per
-# clock x number of SMs x SM clock.
-ALU_LANES_PER_SM = 64          # INT32 lanes per SM per clock
 SM_COUNT = 148
+ISSUE_PER_SM = 4 * 32          # thread instructions per clock: 4 schedulers x 32 lanes
+ALU_LANES_PER_SM = 64          # INT32 lanes per SM per clock (one pipe)
 
 
+# ------------------------------------------------------------------------------------ inputs
 def _peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -38,6 +42,28 @@ def _peaks():
             d = json.load(f)
         return float(d["hbm_gbs"]), float(d.get("sm_max_mhz", 1965.0)), "measured"
     return 6650.0, 1965.0, "fallback"
+
+
+def _executed_counts():
+    """profiles/executed_instructions.txt: thread instructions per rank that each kernel executes
+    (smsp__thread_inst_executed.sum / ranks of an ncu capture) and the DRAM bytes of that launch."""
+    out = {}
+    path = os.path.join(ROOT, "profiles", "executed_instructions.txt")
+    with open(path) as f:
+        for ln in f:
+            ln = ln.split("#")[0].split()
+            if len(ln) >= 4:
+                out[ln[0]] = {"thread_inst_per_rank": float(ln[1]),
+                              "dram_bytes": None if ln[2] == "-" else float(ln[2]),
+                              "ranks_captured": float(ln[3])}
+    return out
+
+
+def _model_ops():
+    """tests/skipcode_model_ops.json, written by `python -m tests.skipcode_mirror --write`: integer
+    operations per rank that the counted CPU restatement of the construction needs."""
+    with open(os.path.join(ROOT, "tests", "skipcode_model_ops.json")) as f:
+        return json.load(f)
 
 
 class ClockSampler:
@@ -96,38 +122,68 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+class Probe:
+    """libbcs_probe.so: the integer instruction rate of this GPU (benchmark helper, not product)."""
+
+    def __init__(self, torch):
+        from paper_2205_10072_b200 import build_ext
+        self.torch = torch
+        self.lib = ctypes.CDLL(build_ext.build_probe())
+        self.lib.bcs_probe_int_rate.argtypes = [ctypes.c_int, ctypes.c_uint32, ctypes.c_void_p,
+                                                ctypes.POINTER(ctypes.c_double),
+                                                ctypes.POINTER(ctypes.c_float), ctypes.c_void_p]
+        self.sink = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def rate(self, mix: int, iters: int = 4096) -> float:
+        ops, ms = ctypes.c_double(0), ctypes.c_float(0)
+        st = self.lib.bcs_probe_int_rate(mix, iters, self.sink.data_ptr(), ctypes.byref(ops),
+                                         ctypes.byref(ms), self.torch.cuda.current_stream().cuda_stream or None)
+        if st != 0:
+            raise RuntimeError("bcs_probe_int_rate: status %d" % st)
+        return ops.value / (ms.value * 1e-3)
+
+    def all(self):
+        names = ("logic_only", "logic_imad_mix", "logic_add_mix")
+        out = {nm: max(self.rate(mix) for _ in range(3)) / 1e12 for mix, nm in enumerate(names)}
+        out["unit"] = "Tint-op/s"
+        return out
+
+
+# ------------------------------------------------------------------------------------ reference arm
 def run_reference(args) -> None:
-    """CPU oracle (per-rank form: Algorithms 4 and 5 for every rank) on the host cores."""
+    """CPU oracle (per-rank form: Algorithms 4 and 5 for every rank) on the host cores, on a bounded
+    sample of the headline workload per step."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     import oracle
     from paper_2205_10072_b200 import workloads
-    p = workloads.P_SINGLE
-    sample = 32768                       # ranks per step: a bounded slice of the same workload
-    lo = (p // 2) - sample // 2
+    p = workloads.P_LARGE
+    sample = 16384                       # ranks per step: seeded spot ranks of the same p
+    ranks = workloads.spot_ranks(p, sample)
     for _ in range(args.warmup):
-        oracle.build_range(p, lo, lo + sample)
+        oracle.build_ranks(p, ranks)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle.build_range(p, lo, lo + sample)
+        oracle.build_ranks(p, ranks)
     dt = time.perf_counter() - t0
     value = args.steps * sample / dt
     cores = oracle.num_threads()
-    sample_txt = "ranks %d..%d of p=2^20+1 per step (per-rank form, Algorithms 4+5)" % (lo, lo + sample - 1)
+    sample_txt = ("%d seeded ranks (next() %% p, splitmix64 seed %d) of p=2^30-1 per step, per-rank "
+                  "form (Algorithms 4+5)" % (sample, workloads.SEED_SPOT))
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8/int32",
         "data": "synthetic",
-        "config": {"workload": "single p=2^20+1 (q=21), all ranks, recv+send int8", "p": p,
-                   "sample": sample_txt},
+        "config": {"workload": WORKLOAD_LARGE, "p": p, "sample": sample_txt},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": sample_txt},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
 
+# ------------------------------------------------------------------------------------ timing helpers
 def _event_ms(torch, fn, flush, steps, warmup):
     """Device time of `steps` calls of fn, each preceded by an (untimed) L2 flush."""
     for _ in range(warmup):
@@ -146,7 +202,195 @@ def _event_ms(torch, fn, flush, steps, warmup):
     return [a.elapsed_time(b) for a, b in pairs]
 
 
-def _bench_expand(torch, bcs, workloads, flush, hbm_gbs, peak_src, steps):
+def _no_flush():
+    pass
+
+
+def _alu_roofline(kernels, ranks, ms, out_bytes, hbm_gbs, sm_max_mhz, counts, model, measured):
+    """Roofline block of a construction step (integer-issue bound).
+    kernels: keys of profiles/executed_instructions.txt whose kernels ran in the `ms` that were timed;
+    model: integer operations per rank of the counted CPU restatement, or None."""
+    issue_peak = SM_COUNT * ISSUE_PER_SM * sm_max_mhz * 1e6 / 1e12           # T thread-inst/s
+    one_pipe = SM_COUNT * ALU_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12
+    per_rank = sum(counts[k]["thread_inst_per_rank"] for k in kernels)
+    achieved = per_rank * ranks / (ms * 1e-3) / 1e12
+    t_int_ms = per_rank * ranks / (issue_peak * 1e12) * 1e3
+    t_hbm_ms = out_bytes / (hbm_gbs * 1e9) * 1e3
+    roof = {"bound": "alu", "kernel": "+".join(kernels), "achieved": achieved, "peak": issue_peak,
+            "unit": "Tthread-inst/s", "frac": achieved / issue_peak, "ms": ms,
+            "executed_thread_inst_per_rank": per_rank,
+            "executed_source": "profiles/executed_instructions.txt (ncu smsp__thread_inst_executed.sum / ranks)",
+            "peak_source": "issue limit: 148 SMs x 4 schedulers x 32 lanes x %.0f MHz (max SM clock)" % sm_max_mhz,
+            "t_int_ms": t_int_ms, "t_hbm_ms": t_hbm_ms, "roofline_ms": max(t_int_ms, t_hbm_ms),
+            "frac_of_max_t_int_t_hbm": max(t_int_ms, t_hbm_ms) / ms,
+            "hbm_peak_gbs": hbm_gbs}
+    if measured:
+        two_pipe = max(measured["logic_imad_mix"], measured["logic_add_mix"])
+        roof["peak_measured"] = measured
+        roof["frac_of_measured_two_pipe_mix"] = achieved / two_pipe
+    if model is not None:
+        m_ach = model * ranks / (ms * 1e-3) / 1e12
+        roof["model"] = {"int_ops_per_rank": model, "achieved": m_ach, "unit": "Tint-op/s",
+                         "source": "tests/skipcode_model_ops.json (tests/skipcode_mirror.py --write)",
+                         "frac_of_issue_limit": m_ach / issue_peak,
+                         "frac_of_one_pipe_%.1fT" % one_pipe: m_ach / one_pipe}
+        if measured:
+            roof["model"]["frac_of_measured_two_pipe_mix"] = m_ach / max(measured["logic_imad_mix"],
+                                                                         measured["logic_add_mix"])
+    return roof
+
+
+WORKLOAD_LARGE = ("large single p=2^30-1 (q=30), all ranks, recv+send int8 (64.4 GB), 8 rank chunks "
+                  "through one reused chunk buffer")
+
+
+class LargeP:
+    """p = 2^30 - 1 in 8 rank chunks through one buffer pair (never all 64 GB resident)."""
+
+    def __init__(self, torch, bcs, workloads):
+        self.torch, self.bcs = torch, bcs
+        self.p = workloads.P_LARGE
+        self.q = bcs.bcs_q(self.p)
+        self.chunks = workloads.large_chunks()
+        cap = max(r1 - r0 for r0, r1 in self.chunks)
+        self.recv = torch.empty(cap * self.q, dtype=torch.int8, device="cuda")
+        self.send = torch.empty(cap * self.q, dtype=torch.int8, device="cuda")
+        self.ws = torch.empty(bcs.bcs_prepare_workspace_bytes(self.p), dtype=torch.int8, device="cuda")
+        self.launches_per_step = 1 + 2 * len(self.chunks)
+
+    def step(self):
+        bcs, p, ws = self.bcs, self.p, self.ws
+        bcs.bcs_prepare_codes(p, ws)
+        for r0, r1 in self.chunks:                   # receive rows of the chunk, round-major copy
+            bcs.bcs_prepare_rows(p, r0, r1, self.recv, ws)
+        for r0, r1 in self.chunks:                   # send rows of the chunk (Algorithm 9's lookup)
+            bcs.bcs_build_prepared(p, r0, r1, None, self.send, ws)
+
+    def parts_ms(self, reps=3):
+        """codes / receive rows / send rows of a step, by CUDA events."""
+        torch, bcs, p, ws = self.torch, self.bcs, self.p, self.ws
+        acc = [0.0, 0.0, 0.0]
+        for _ in range(reps):
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            ev[0].record()
+            bcs.bcs_prepare_codes(p, ws)
+            ev[1].record()
+            for r0, r1 in self.chunks:
+                bcs.bcs_prepare_rows(p, r0, r1, self.recv, ws)
+            ev[2].record()
+            for r0, r1 in self.chunks:
+                bcs.bcs_build_prepared(p, r0, r1, None, self.send, ws)
+            ev[3].record()
+            torch.cuda.synchronize()
+            for i in range(3):
+                acc[i] += ev[i].elapsed_time(ev[i + 1]) / reps
+        return acc
+
+    def checked_step(self):
+        """The step with a checksum of every chunk and the property check of its rows."""
+        torch, bcs, p, q, ws = self.torch, self.bcs, self.p, self.q, self.ws
+        sums = torch.zeros(2, dtype=torch.int64, device="cuda")
+        viol = torch.zeros(3, dtype=torch.int64, device="cuda")
+        total = torch.zeros(3, dtype=torch.int64, device="cuda")
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        bcs.bcs_prepare_codes(p, ws)
+        for r0, r1 in self.chunks:
+            bcs.bcs_prepare_rows(p, r0, r1, self.recv, ws)
+            bcs.bcs_checksum(self.recv, r0 * q, sums[0:1], n_entries=(r1 - r0) * q)
+            bcs.bcs_validate(p, r0, r1, self.recv, None, viol)
+            total += viol
+        for r0, r1 in self.chunks:
+            bcs.bcs_build_prepared(p, r0, r1, None, self.send, ws)
+            bcs.bcs_checksum(self.send, (1 << 36) + r0 * q, sums[1:2], n_entries=(r1 - r0) * q)
+            bcs.bcs_validate(p, r0, r1, None, self.send, viol)
+            total += viol
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b), total.cpu().tolist()
+
+    def e2e(self, steps):
+        """The step with every chunk copied to pinned HOST buffers inside the timed region."""
+        torch, bcs, p, ws = self.torch, self.bcs, self.p, self.ws
+        h_recv = torch.empty(self.recv.numel(), dtype=torch.int8).pin_memory()
+        h_send = torch.empty(self.send.numel(), dtype=torch.int8).pin_memory()
+
+        def one():
+            bcs.bcs_prepare_codes(p, ws)
+            for r0, r1 in self.chunks:
+                n = (r1 - r0) * self.q
+                bcs.bcs_prepare_rows(p, r0, r1, self.recv, ws)
+                h_recv[:n].copy_(self.recv[:n], non_blocking=True)
+            for r0, r1 in self.chunks:
+                n = (r1 - r0) * self.q
+                bcs.bcs_build_prepared(p, r0, r1, None, self.send, ws)
+                h_send[:n].copy_(self.send[:n], non_blocking=True)
+            torch.cuda.synchronize()
+
+        one()
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            one()
+        dt = (time.perf_counter() - t0) / steps
+        return {"value": p / dt, "unit": UNIT, "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": 2 * p * self.q, "ms_per_step": dt * 1e3, "steps": steps,
+                "how": "bcs_prepare_codes / bcs_prepare_rows / bcs_build_prepared through the C ABI, every "
+                       "chunk copied to pinned host memory on the same stream (inputs are scalars: no H2D)"}
+
+
+def _bench_single(torch, bcs, workloads, flush, steps, hbm_gbs, sm_max_mhz, counts, model, measured):
+    """Single p = 2^20+1: one bcs_build per step, L2 flushed before every step."""
+    p = workloads.P_SINGLE
+    q = bcs.bcs_q(p)
+    nb = p * q
+    recv = torch.empty(nb, dtype=torch.int8, device="cuda")
+    send = torch.empty(nb, dtype=torch.int8, device="cuda")
+    ws = torch.empty(bcs.bcs_build_workspace_bytes(p, 0, p), dtype=torch.int8, device="cuda")
+    ms = _event_ms(torch, lambda: bcs.bcs_build(p, 0, p, recv, send, ws), flush, steps, 5)
+    step_ms = statistics.mean(ms)
+    # codes + receive kernel as the step runs them (rows and round-major copy), by bcs_prepare_rows
+    pws = torch.empty(bcs.bcs_prepare_workspace_bytes(p), dtype=torch.int8, device="cuda")
+
+    def recv_part():
+        bcs.bcs_prepare_codes(p, pws)
+        bcs.bcs_prepare_rows(p, 0, p, recv, pws)
+    recv_ms = statistics.mean(_event_ms(torch, recv_part, flush, max(20, steps // 4), 3))
+    slow_ms = statistics.mean(_event_ms(torch, lambda: bcs.bcs_build(p, 0, p, recv, send, None), flush, 10, 2))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(2000):
+        bcs.bcs_build(p, 0, p, recv, send, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    res = {"workload": "single p=2^20+1 (q=21), all ranks, recv+send int8 (44 MB), one bcs_build per step",
+           "ranks": p, "ms": step_ms, "median_ms": statistics.median(ms), "min_ms": min(ms),
+           "ranks_per_s": p / step_ms * 1e3, "out_gbs": 2 * nb / step_ms / 1e6,
+           "l2": "flushed before every timed step (256 MiB write)",
+           "back_to_back_ms": e0.elapsed_time(e1) / 2000,
+           "kernel_ms": {"codes+recv (bcs_prepare_codes + bcs_prepare_rows)": recv_ms,
+                         "send transposition (difference)": max(step_ms - recv_ms, 0.0),
+                         "self_contained_construction_step": slow_ms},
+           "roofline": _alu_roofline(["codes_single_kernel@q21", "recv_codes_quad_kernel<true,true>@q21"], p,
+                                     recv_ms, nb + nb, hbm_gbs, sm_max_mhz, counts,
+                                     model["q21_p1048577"]["recv_int_ops_per_rank"], measured),
+           "step_roofline": _alu_roofline(["codes_single_kernel@q21", "recv_codes_quad_kernel<true,true>@q21",
+                                           "send_transpose_kernel@q21"], p, step_ms, 2 * nb, hbm_gbs,
+                                          sm_max_mhz, counts,
+                                          model["q21_p1048577"]["recv_int_ops_per_rank"]
+                                          + model["q21_p1048577"]["send_int_ops_per_rank"], measured)}
+    res["roofline"]["traffic"] = counts["recv_codes_quad_kernel<true,true>@q21"]["dram_bytes"]
+    # property check and brute-force broadcast of the tables just built
+    viol = torch.zeros(3, dtype=torch.int64, device="cuda")
+    v_ms = statistics.mean(_event_ms(torch, lambda: bcs.bcs_validate(p, 0, p, recv, send, viol), flush, 10, 2))
+    res["validate"] = {"ms": v_ms, "violations": viol.cpu().tolist()}
+    state = torch.empty(2 * p, dtype=torch.int64, device="cuda")
+    cnt = torch.zeros(5, dtype=torch.int64, device="cuda")
+    s_ms = statistics.mean(_event_ms(torch, lambda: bcs.bcs_simulate(p, 5, recv, send, state, cnt), flush, 5, 1))
+    res["simulate_5_blocks_25_rounds"] = {"ms": s_ms, "counts": cnt.cpu().tolist()}
+    return res
+
+
+def _bench_expand(torch, bcs, workloads, flush, hbm_gbs, peak_src, steps, counts):
     pe, ne = workloads.P_EXPAND, workloads.N_EXPAND
     qe = bcs.bcs_q(pe)
     er = torch.empty(pe * qe, dtype=torch.int8, device="cuda")
@@ -159,10 +403,11 @@ def _bench_expand(torch, bcs, workloads, flush, hbm_gbs, peak_src, steps):
         torch, lambda: bcs.bcs_expand(pe, ne, 0, pe, er, es, table), flush, steps, 3))
     nbytes = pe * rounds * 16
     gbs = nbytes / ms / 1e6
-    res = {"workload": "p=100003, n=1000, all ranks, 1016 rounds, 16 B records", "ms": ms,
-           "bytes": nbytes, "gbs": gbs,
+    res = {"workload": "round-table expansion p=100003, n=1000, all ranks, 1016 rounds, 16 B records", "ms": ms,
+           "bytes": nbytes, "gbs": gbs, "ranks_per_s": pe / ms * 1e3,
            "roofline": {"bound": "hbm", "kernel": "expand_kernel", "achieved": gbs, "peak": hbm_gbs,
-                        "unit": "GB/s", "frac": gbs / hbm_gbs, "traffic": EXPAND_TRAFFIC_BYTES,
+                        "unit": "GB/s", "frac": gbs / hbm_gbs,
+                        "traffic": counts["expand_kernel@p100003_n1000"]["dram_bytes"],
                         "peak_source": peak_src}}
     # context: a plain store-only stream over the same buffer (cudaMemset through torch) and the
     # nominal HBM3e figure -- the measured copy peak mixes reads and writes
@@ -174,7 +419,7 @@ def _bench_expand(torch, bcs, workloads, flush, hbm_gbs, peak_src, steps):
     return res, table
 
 
-def _bench_allgather(torch, bcs, workloads, flush, hbm_gbs, peak_src, steps):
+def _bench_allgather(torch, bcs, workloads, flush, hbm_gbs, peak_src, steps, counts):
     p, n = workloads.P_EXPAND, workloads.N_EXPAND
     q = bcs.bcs_q(p)
     er = torch.empty(p * q, dtype=torch.int8, device="cuda")
@@ -192,10 +437,11 @@ def _bench_allgather(torch, bcs, workloads, flush, hbm_gbs, peak_src, steps):
             "ms": ms, "bytes": nbytes, "gbs": gbs,
             "roofline": {"bound": "hbm", "kernel": "allgather_kernel", "achieved": gbs,
                          "peak": hbm_gbs, "unit": "GB/s", "frac": gbs / hbm_gbs,
-                         "traffic": ALLGATHER_TRAFFIC_BYTES, "peak_source": peak_src}}
+                         "traffic": counts["allgather_kernel@p100003_n1000"]["dram_bytes"],
+                         "peak_source": peak_src}}
 
 
-def _bench_checksum(torch, bcs, flush, hbm_gbs, peak_src, table, steps):
+def _bench_checksum(torch, bcs, flush, hbm_gbs, peak_src, table, steps, counts):
     sums = torch.zeros(1, dtype=torch.int64, device="cuda")
     tb = table.view(torch.int8).view(-1)
     ms = statistics.mean(_event_ms(torch, lambda: bcs.bcs_checksum(tb, 0, sums), flush, steps, 3))
@@ -203,51 +449,12 @@ def _bench_checksum(torch, bcs, flush, hbm_gbs, peak_src, table, steps):
     return {"workload": "%.2f GB buffer" % (tb.numel() / 1e9), "ms": ms, "gbs": gbs,
             "roofline": {"bound": "hbm", "kernel": "checksum_kernel", "achieved": gbs,
                          "peak": hbm_gbs, "unit": "GB/s", "frac": gbs / hbm_gbs,
-                         "traffic": CHECKSUM_TRAFFIC_BYTES if tb.numel() == 1625648768 else None,
+                         "traffic": counts["checksum_kernel@1625648768B"]["dram_bytes"]
+                         if tb.numel() == 1625648768 else None,
                          "peak_source": peak_src}}
 
 
-def _bench_large(torch, bcs, workloads, hbm_gbs):
-    """p = 2^30 - 1 in 8 rank chunks through one buffer: build, checksum and property check of
-    every chunk on one stream (64 GB of tables in total, never resident together)."""
-    p = workloads.P_LARGE
-    q = bcs.bcs_q(p)
-    chunks = workloads.large_chunks()
-    cap = max(r1 - r0 for r0, r1 in chunks)
-    recv = torch.empty(cap * q, dtype=torch.int8, device="cuda")
-    send = torch.empty(cap * q, dtype=torch.int8, device="cuda")
-    ws = torch.empty(bcs.bcs_prepare_workspace_bytes(p), dtype=torch.int8, device="cuda")
-    sums = torch.zeros(2, dtype=torch.int64, device="cuda")
-    viol = torch.zeros(3, dtype=torch.int64, device="cuda")
-    total_viol = torch.zeros(3, dtype=torch.int64, device="cuda")
-    res = {}
-    for what in ("build", "build+checksum+validate"):
-        bcs.bcs_build(p, 0, 1 << 20, recv, send, None)                    # warm-up
-        torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        bcs.bcs_prepare(p, ws)
-        for r0, r1 in chunks:
-            bcs.bcs_build_prepared(p, r0, r1, recv, send, ws)
-            if what != "build":
-                nb = (r1 - r0) * q
-                bcs.bcs_checksum(recv, r0 * q, sums[0:1], n_entries=nb)
-                bcs.bcs_checksum(send, (1 << 36) + r0 * q, sums[1:2], n_entries=nb)
-                bcs.bcs_validate(p, r0, r1, recv, send, viol)
-                total_viol += viol
-        b.record()
-        torch.cuda.synchronize()
-        res[what] = a.elapsed_time(b)
-    ms = res["build"]
-    return {"workload": "p=2^30-1 (q=30), bcs_prepare + 8 chunks of 2^27 ranks by "
-                        "bcs_build_prepared, recv+send, one reused chunk buffer",
-            "workspace_bytes": ws.numel(),
-            "ranks": p, "ms": ms, "ranks_per_s": p / ms * 1e3, "out_gbs": 2 * p * q / ms / 1e6,
-            "ms_with_checksum_and_validate": res["build+checksum+validate"],
-            "violations": total_viol.cpu().tolist()}
-
-
-def _bench_batch(torch, bcs, workloads, flush, full):
+def _bench_batch(torch, bcs, workloads, flush, full, hbm_gbs, sm_max_mhz, counts, model, measured):
     out = {}
     plan = bcs.bcs_batch_plan(workloads.small_sweep())
     dplan = plan.to("cuda")
@@ -258,9 +465,16 @@ def _bench_batch(torch, bcs, workloads, flush, full):
     ms = statistics.mean(_event_ms(
         torch, lambda: bcs.bcs_build_batch(dplan, plan.total_ranks, plan.total_entries, br, bs, bw),
         flush, 20, 3))
-    out["batch_small_sweep"] = {"workload": "every p in 2..1024, one launch pair",
-                                "ranks": plan.total_ranks, "ms": ms,
-                                "ranks_per_s": plan.total_ranks / ms * 1e3}
+    batch_kernels = ["codes_batch_kernel", "recv_quad_batch_kernel<true>", "send_batch_kernel"]
+    out["batch_small_sweep"] = {
+        "workload": "every p in 2..1024, all ranks, one bcs_build_batch (three launches)",
+        "ranks": plan.total_ranks, "ms": ms, "ranks_per_s": plan.total_ranks / ms * 1e3,
+        "out_gbs": 2 * plan.total_entries / ms / 1e6,
+        "l2": "flushed before every timed step",
+        "roofline": _alu_roofline([k + "@small_sweep" for k in batch_kernels], plan.total_ranks, ms,
+                                  2 * plan.total_entries, hbm_gbs, sm_max_mhz, counts,
+                                  model["small_sweep_2_1024"]["recv_int_ops_per_rank"]
+                                  + model["small_sweep_2_1024"]["send_int_ops_per_rank"], measured)}
     plist = workloads.batch_p_list() if full else workloads.batch_p_list(count=256)
     plan = bcs.bcs_batch_plan(plist)
     dplan = plan.to("cuda")
@@ -271,14 +485,77 @@ def _bench_batch(torch, bcs, workloads, flush, full):
                      dtype=torch.int8, device="cuda")
     ms = statistics.mean(_event_ms(
         torch, lambda: bcs.bcs_build_batch(dplan, plan.total_ranks, plan.total_entries, br, bs, bw),
-        lambda: None, 3, 1))                       # the outputs exceed L2 by themselves
+        _no_flush, 3, 1))                          # the outputs exceed L2 by themselves
     out["batch_irregular_sweep"] = {
-        "workload": "%d octave-uniform p in [2^10,2^20), seed %d" % (len(plist), workloads.SEED_BATCH),
+        "workload": "%d octave-uniform p in [2^10,2^20), seed %d, one bcs_build_batch"
+                    % (len(plist), workloads.SEED_BATCH),
         "ranks": plan.total_ranks, "ms": ms, "ranks_per_s": plan.total_ranks / ms * 1e3,
-        "out_gbs": 2 * plan.total_entries / ms / 1e6}
+        "out_gbs": 2 * plan.total_entries / ms / 1e6,
+        "l2": "outputs (%.1f GB) exceed L2" % (2 * plan.total_entries / 1e9),
+        "roofline": _alu_roofline([k + "@256p_sample" for k in batch_kernels], plan.total_ranks, ms,
+                                  2 * plan.total_entries, hbm_gbs, sm_max_mhz, counts,
+                                  model["batch_4096p"]["recv_int_ops_per_rank"]
+                                  + model["batch_4096p"]["send_int_ops_per_rank"], measured)}
     return out
 
 
+def _cpu_baselines(oracle, workloads):
+    """The oracle as it stands on the host cores: a bounded sample of every workload."""
+    res = {}
+    cores = oracle.num_threads()
+    # headline: seeded ranks of p = 2^30-1, per-rank form, about 10 s
+    p = workloads.P_LARGE
+    ranks = workloads.spot_ranks(p, 1 << 16)
+    n, dt = 0, 0.0
+    while dt < 10.0:
+        t0 = time.perf_counter()
+        oracle.build_ranks(p, ranks)
+        dt += time.perf_counter() - t0
+        n += len(ranks)
+    head = {"value": n / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d x 65536 seeded ranks (next() %% p, splitmix64 seed %d) of p=2^30-1, per-rank form "
+                      "(Algorithms 4+5), %.1f s; the whole workload at this rate would take %.0f s "
+                      "(extrapolated)" % (n // 65536, workloads.SEED_SPOT, dt, p / (n / dt))}
+    t0 = time.perf_counter()
+    oracle.build_ranks(p, ranks, want_send=False)
+    head["recv_only_value"] = len(ranks) / (time.perf_counter() - t0)
+    # every p <= 1024 (array form, all of it)
+    t0 = time.perf_counter()
+    total = 0
+    for pj in workloads.small_sweep():
+        oracle.full_table(pj)
+        total += pj
+    res["batch_small_sweep"] = {"value": total / (time.perf_counter() - t0), "unit": UNIT, "cores": cores,
+                                "sample": "all of it, array form"}
+    # single p = 2^20+1: array form (all of it) and per-rank form (2^18 ranks)
+    p2 = workloads.P_SINGLE
+    t0 = time.perf_counter()
+    want_r, want_s = oracle.full_table(p2)
+    res["single_p"] = {"array_form_value": p2 / (time.perf_counter() - t0), "unit": UNIT, "cores": cores}
+    t0 = time.perf_counter()
+    oracle.build_range(p2, 0, 1 << 18)
+    res["single_p"]["value"] = (1 << 18) / (time.perf_counter() - t0)
+    res["single_p"]["sample"] = "ranks 0..262143, per-rank form; array form: all ranks"
+    # batched irregular sweep: the first 64 p of the list, array form
+    t0 = time.perf_counter()
+    total = 0
+    for pj in workloads.batch_p_list(count=64):
+        oracle.full_table(pj)
+        total += pj
+    res["batch_irregular_sweep"] = {"value": total / (time.perf_counter() - t0), "unit": UNIT, "cores": cores,
+                                    "sample": "the first 64 p of the list (%d ranks), array form" % total}
+    # expansion: Algorithm 6's literal loop for 4096 ranks of p = 100003, n = 1000
+    pe, ne = workloads.P_EXPAND, workloads.N_EXPAND
+    er, es = oracle.full_table(pe)
+    t0 = time.perf_counter()
+    oracle.expand(pe, ne, er, es, 0, 4096)
+    dt = time.perf_counter() - t0
+    res["expand"] = {"value": 4096 / dt, "unit": UNIT, "gbs": 4096 * (ne - 1 + oracle.q_of(pe)) * 16 / dt / 1e9,
+                     "cores": cores, "sample": "ranks 0..4095 of p=100003, n=1000 (schedules given)"}
+    return head, res
+
+
+# ------------------------------------------------------------------------------------ our arm
 def run_ours(args) -> None:
     import torch
     import torch.distributed as dist
@@ -297,44 +574,22 @@ def run_ours(args) -> None:
     bcs.lib()
 
     hbm_gbs, sm_max_mhz, peak_src = _peaks()
+    counts = _executed_counts()
+    model = _model_ops()
     flush_buf = torch.empty(256 << 20, dtype=torch.int8, device="cuda")   # > 126 MB L2
 
     def flush():
         flush_buf.fill_(1)
 
-    if args.only in ("expand", "checksum", "batch", "allgather", "probe"):   # small single-part runs (profiling)
+    if args.only != "all":                         # small single-part runs (what profiles/ cites)
         if rank == 0:
-            res = {}
-            if args.only == "probe":
-                names = ("logic_only", "logic_imad_mix", "logic_add_mix")
-                res["int_rate_probe"] = {nm: [bcs.bcs_probe_int_rate(mix, 1024) / 1e12 for _ in range(2)]
-                                         for mix, nm in enumerate(names)}
-                res["int_rate_probe"]["unit"] = "Tint-op/s"
-            elif args.only == "allgather":
-                res["allgather_tables"] = _bench_allgather(torch, bcs, workloads, flush, hbm_gbs,
-                                                           peak_src, args.steps)
-            elif args.only in ("expand", "checksum"):
-                ex, table = _bench_expand(torch, bcs, workloads, flush, hbm_gbs, peak_src,
-                                          args.steps)
-                res["expand"] = ex
-                if args.only == "checksum":
-                    res["checksum"] = _bench_checksum(torch, bcs, flush, hbm_gbs, peak_src, table,
-                                                      args.steps)
-            else:
-                res = _bench_batch(torch, bcs, workloads, flush, full=False)
-            print(json.dumps({"only": args.only, "steps": args.steps, "aux": res}))
+            print(json.dumps({"only": args.only, "steps": args.steps,
+                              "aux": _run_part(args, torch, bcs, workloads, flush, hbm_gbs, sm_max_mhz,
+                                               peak_src, counts, model)}))
         return
 
-    p = workloads.P_SINGLE
-    q = bcs.bcs_q(p)
-    nb = p * q
-    recv = torch.empty(nb, dtype=torch.int8, device="cuda")
-    send = torch.empty(nb, dtype=torch.int8, device="cuda")
-    ws_bytes = bcs.bcs_build_workspace_bytes(p, 0, p)
-    ws = torch.empty(ws_bytes, dtype=torch.int8, device="cuda")
-
-    def step():
-        bcs.bcs_build(p, 0, p, recv, send, ws)
+    large = LargeP(torch, bcs, workloads)
+    p, q = large.p, large.q
 
     def barrier():
         torch.cuda.synchronize()
@@ -342,14 +597,14 @@ def run_ours(args) -> None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- the timed region: K steps, device time per step by CUDA events, L2 flushed between
+    # ---- the timed region: K steps, device time per step by CUDA events (a step writes 64 GB
+    # through 8 GB chunk buffers: far more than the L2 holds, so no flush between steps)
     for _ in range(args.warmup):
-        flush()
-        step()
+        large.step()
     barrier()
     with ClockSampler(local) as clk:
         t_wall0 = time.perf_counter()
-        ms = _event_ms(torch, step, flush, args.steps, 0)
+        ms = _event_ms(torch, large.step, _no_flush, args.steps, 0)
         barrier()
         t_wall = time.perf_counter() - t_wall0
     total_ms = sum(ms)
@@ -362,146 +617,66 @@ def run_ours(args) -> None:
 
     out = None
     if rank == 0:
-        # ---- per-kernel times (same protocol).  A receive-only call runs the codes kernel and the
-        # receive kernel (without the round-major copy); the send kernel is the difference.
-        recv_ms = statistics.mean(_event_ms(torch, lambda: bcs.bcs_build(p, 0, p, recv, None, ws),
-                                            flush, max(5, args.steps // 4), 3))
-        send_ms = max(ms_per_step - recv_ms, 0.0)
-        slow_ms = statistics.mean(_event_ms(torch, lambda: bcs.bcs_build(p, 0, p, recv, send, None),
-                                            flush, 10, 2))
-        model = ALU_MODEL[q]
-        alu_peak = SM_COUNT * ALU_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12     # T int-op/s
-        achieved = model * p / (recv_ms * 1e-3) / 1e12
-        roof = {"bound": "alu", "kernel": "codes_single_kernel+recv_codes_quad_kernel", "achieved": achieved,
-                "peak": alu_peak, "unit": "Tint-op/s", "frac": achieved / alu_peak,
-                "traffic": RECV_TRAFFIC_BYTES, "ms": recv_ms, "model_int_ops_per_rank": model,
-                "peak_source": "148 SMs x 64 INT32 lanes x %.0f MHz (max SM clock)" % sm_max_mhz,
-                "hbm_bound_ms": 2 * nb / (hbm_gbs * 1e6),
-                "hbm_time_frac": (2 * nb / (hbm_gbs * 1e9)) / (ms_per_step * 1e-3),
-                "hbm_peak_source": peak_src}
-        # measured integer instruction rates of this GPU in this session (probe kernel)
-        meas = [max(bcs.bcs_probe_int_rate(mix) for _ in range(3)) / 1e12 for mix in (0, 1, 2)]
-        roof["peak_measured"] = {"logic_only": meas[0], "logic_imad_mix": meas[1],
-                                 "logic_add_mix": meas[2], "unit": "Tint-op/s"}
-        roof["frac_of_measured_logic_only"] = achieved / meas[0]
-        # the same time against the issue limit (one warp instruction per cycle and SM
-        # sub-partition), with the instructions the kernels really execute
-        issue_peak = SM_COUNT * 4 * 32 * sm_max_mhz * 1e6 / 1e12
-        executed = EXECUTED_INST_PER_RANK[q] * p / (recv_ms * 1e-3) / 1e12
-        roof["issue"] = {"executed_thread_inst_per_rank": EXECUTED_INST_PER_RANK[q],
-                         "achieved": executed, "peak": issue_peak, "unit": "Tthread-inst/s",
-                         "frac": executed / issue_peak,
-                         "frac_of_measured_two_pipe_mix": executed / max(meas[1], meas[2])}
-        # ---- the same step timed in other ways (reported beside the headline, not instead of it)
-        def back_to_back(count):
-            e0 = torch.cuda.Event(enable_timing=True)
-            e1 = torch.cuda.Event(enable_timing=True)
-            e0.record()
-            for _ in range(count):
-                step()
-            e1.record()
-            torch.cuda.synchronize()
-            return e0.elapsed_time(e1) / count
-        b2b_ms = back_to_back(2000)                      # no L2 flush: the workspace stays in L2
-        sustained_steps, sustained_ms, t_s0 = 0, 0.0, time.perf_counter()
-        with ClockSampler(local) as clk_sustained:
-            while time.perf_counter() - t_s0 < 2.0:      # at least 2 s of back-to-back steps
-                sustained_ms += back_to_back(4000) * 4000
-                sustained_steps += 4000
-        timing = {"best_of_10_ms": min(ms[:10]) if len(ms) >= 10 else min(ms), "min_ms": min(ms),
-                  "median_ms": statistics.median(ms),
-                  "back_to_back_ms_per_step": b2b_ms,
-                  "sustained_ms_per_step": sustained_ms / sustained_steps,
-                  "sustained_steps": sustained_steps,
-                  "sustained_clocks": clk_sustained.summary()}
+        measured = Probe(torch).all()
+        codes_ms, rows_ms, send_ms = large.parts_ms()
+        m30 = model["q30_p1073741823"]
+        roof = _alu_roofline(["recv_codes_quad_kernel<true,true>@q30"], p, rows_ms, 2 * p * q, hbm_gbs,
+                             sm_max_mhz, counts, m30["recv_int_ops_per_rank"] - m30["code_ops_per_rank"],
+                             measured)
+        roof["kernel"] = "recv_codes_quad_kernel<true,true> (8 launches of bcs_prepare_rows: %.1f%% of the step)" \
+                         % (100 * rows_ms / (codes_ms + rows_ms + send_ms))
+        roof["traffic"] = None
+        roof["traffic_note"] = ("not captured at this size (8 GB per launch); the DRAM bytes of a 2^22-rank "
+                                "range of the same p are in profiles/, they do not scale in proportion "
+                                "(re-reads of the skip codes depend on what the L2 still holds)")
+        step_roof = _alu_roofline(["codes_single_kernel@q30", "recv_codes_quad_kernel<true,true>@q30",
+                                   "send_transpose_kernel@q30"], p, ms_per_step, 2 * p * q, hbm_gbs,
+                                  sm_max_mhz, counts,
+                                  m30["recv_int_ops_per_rank"] + m30["send_int_ops_per_rank"], measured)
+        checked_ms, violations = large.checked_step()
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
-            "config": {"workload": "single p=2^20+1 (q=21), all ranks, recv+send int8 (44 MB)",
-                       "p": p, "q": q,
-                       "send_variant": "lookup (transposition of the round-major receive copy)",
-                       "l2": "flushed between timed steps (256 MiB write)",
+            "config": {"workload": WORKLOAD_LARGE, "p": p, "q": q, "chunks": len(large.chunks),
+                       "send_variant": "lookup (rotated transposition of the round-major receive copy)",
+                       "l2": "no flush: every step streams 64 GB of outputs through 8 GB chunk buffers, "
+                             "far beyond the 126 MB L2",
+                       "workspace_bytes": large.ws.numel(),
                        "parallelism": "replicas" if world > 1 else "1 GPU",
                        "timed_wall_s": t_wall},
-            "out_gbs": 2 * nb / ms_per_step / 1e6,
-            "kernel_ms": {"codes+recv_codes": recv_ms, "send_rm": send_ms,
-                          "self_contained_path_step": slow_ms},
-            "workspace_bytes": ws_bytes, "timing": timing,
-            "roofline": roof, "gpu_launches": 3 * args.steps, "clocks": clk.summary(),
+            "out_gbs": 2 * p * q / ms_per_step / 1e6,
+            "timing": {"median_ms": statistics.median(ms), "min_ms": min(ms), "max_ms": max(ms)},
+            "kernel_ms": {"codes (bcs_prepare_codes)": codes_ms, "receive rows (8 x bcs_prepare_rows)": rows_ms,
+                          "send rows (8 x bcs_build_prepared)": send_ms},
+            "roofline": roof, "step_roofline": step_roof,
+            "gpu_launches": large.launches_per_step * args.steps, "clocks": clk.summary(),
+            "checked_step": {"what": "the step plus a checksum and the property check of every chunk",
+                             "ms": checked_ms, "violations": violations},
+            "wait_expired": bcs.bcs_wait_expired(),
         }
-        if args.only == "all":
-            # ---- end to end: host buffers, D2H copies inside the timed region
-            stage = torch.empty(2 * ((nb + 255) // 256 * 256) + ws_bytes, dtype=torch.int8,
-                                device="cuda")
-            h_recv = torch.empty(nb, dtype=torch.int8).pin_memory()
-            h_send = torch.empty(nb, dtype=torch.int8).pin_memory()
-            e2e_steps = max(5, min(args.steps, 50))
-            for _ in range(3):
-                bcs.bcs_build_to_host(p, 0, p, h_recv, h_send, stage)
-            torch.cuda.synchronize()
-            t0 = time.perf_counter()
-            for _ in range(e2e_steps):
-                bcs.bcs_build_to_host(p, 0, p, h_recv, h_send, stage)
-                torch.cuda.synchronize()
-            e2e_dt = (time.perf_counter() - t0) / e2e_steps
-            del stage
-            out["e2e"] = {"value": p / e2e_dt, "unit": UNIT, "h2d_bytes_per_step": 0,
-                          "d2h_bytes_per_step": 2 * nb, "ms_per_step": e2e_dt * 1e3}
-
-            # ---- other entry points of the path (reported, not part of the metric)
-            aux = {}
-            aux["expand"], table = _bench_expand(torch, bcs, workloads, flush, hbm_gbs, peak_src, 20)
-            aux["checksum"] = _bench_checksum(torch, bcs, flush, hbm_gbs, peak_src, table, 20)
-            viol = torch.zeros(3, dtype=torch.int64, device="cuda")
-            v_ms = statistics.mean(_event_ms(
-                torch, lambda: bcs.bcs_validate(p, 0, p, recv, send, viol), flush, 20, 3))
-            aux["validate"] = {"workload": "p=2^20+1, both tables, all ranks", "ms": v_ms,
-                               "ranks_per_s": p / v_ms * 1e3, "violations": viol.cpu().tolist()}
-            state = torch.empty(2 * p, dtype=torch.int64, device="cuda")
-            counts = torch.zeros(5, dtype=torch.int64, device="cuda")
-            s_ms = statistics.mean(_event_ms(
-                torch, lambda: bcs.bcs_simulate(p, 5, recv, send, state, counts), flush, 5, 1))
-            aux["simulate"] = {"workload": "p=2^20+1, n=5 blocks, 25 rounds, all ranks", "ms": s_ms,
-                               "counts": counts.cpu().tolist()}
-            del table
-            aux["allgather_tables"] = _bench_allgather(torch, bcs, workloads, flush, hbm_gbs,
-                                                       peak_src, 20)
-            aux.update(_bench_batch(torch, bcs, workloads, flush, full=True))
-            aux["large_p_chunked"] = _bench_large(torch, bcs, workloads, hbm_gbs)
-            out["aux"] = aux
-
-            # ---- CPU baseline: the oracle as it stands, per-rank form, bounded sample
-            import oracle
-            cpu_sample = 1 << 20
-            lo = 0
-            reps, cpu_dt = 0, 0.0
-            while cpu_dt < 10.0:                     # about 10 s of oracle work
-                t0 = time.perf_counter()
-                oracle.build_range(p, lo, lo + cpu_sample)
-                cpu_dt += time.perf_counter() - t0
-                reps += 1
-            t0 = time.perf_counter()
-            oracle.full_table(p)
-            cpu_arr_dt = time.perf_counter() - t0
-            out["cpu_baseline"] = {
-                "value": reps * cpu_sample / cpu_dt, "unit": UNIT, "cores": oracle.num_threads(),
-                "kind": "oracle",
-                "sample": "ranks %d..%d of p=2^20+1, per-rank form (Algorithms 4+5), %d passes, %.1f s"
-                          % (lo, lo + cpu_sample - 1, reps, cpu_dt),
-                "array_form_value": p / cpu_arr_dt}
-            try:                                     # the same oracle on one core (OpenMP runtime call)
-                import ctypes
-                gomp = ctypes.CDLL("libgomp.so.1")
-                threads = oracle.num_threads()
-                gomp.omp_set_num_threads(1)
-                one = 1 << 16
-                t0 = time.perf_counter()
-                oracle.build_range(p, lo, lo + one)
-                out["cpu_baseline"]["single_core_value"] = one / (time.perf_counter() - t0)
-                gomp.omp_set_num_threads(threads)
-            except OSError:
-                pass
+        out["e2e"] = large.e2e(2)
+        del large
+        torch.cuda.empty_cache()
+        # ---- the other workloads (each with its own roofline block)
+        cfg = {}
+        cfg["single_p"] = _bench_single(torch, bcs, workloads, flush, 300, hbm_gbs, sm_max_mhz, counts,
+                                        model, measured)
+        cfg.update(_bench_batch(torch, bcs, workloads, flush, True, hbm_gbs, sm_max_mhz, counts, model,
+                                measured))
+        cfg["expand"], table = _bench_expand(torch, bcs, workloads, flush, hbm_gbs, peak_src, 20, counts)
+        cfg["checksum"] = _bench_checksum(torch, bcs, flush, hbm_gbs, peak_src, table, 20, counts)
+        del table
+        cfg["allgather_tables"] = _bench_allgather(torch, bcs, workloads, flush, hbm_gbs, peak_src, 20,
+                                                   counts)
+        out["configs"] = cfg
+        # ---- CPU baseline: the oracle as it stands, bounded samples
+        import oracle
+        out["cpu_baseline"], per_cfg = _cpu_baselines(oracle, workloads)
+        for name, base in per_cfg.items():
+            cfg[name]["cpu_baseline"] = base
+    else:
+        del large
     barrier()
     if world > 1:
         dist.destroy_process_group()
@@ -509,36 +684,61 @@ def run_ours(args) -> None:
         print(json.dumps(out))
 
 
-# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of the
-# current kernels); None until counters have been taken for the kernel as it stands.
-RECV_TRAFFIC_BYTES = 4257536 + 238080        # recv_codes_quad_kernel<true,true>, p = 2^20+1
-# thread instructions per rank that the codes kernel and the receive-only variant of the receive
-# kernel (the one timed for the roofline line) execute on that workload
-# (smsp__thread_inst_executed.sum of the same capture / p): 91 + 477
-EXECUTED_INST_PER_RANK = {21: 91 + 477}
-EXPAND_TRAFFIC_BYTES = 1566649856 + 3409408   # expand_kernel, p = 100003, n = 1000
-ALLGATHER_TRAFFIC_BYTES = 753529344 + 3564800  # allgather_kernel, p = 100003, n = 1000
-CHECKSUM_TRAFFIC_BYTES = 1625745664 + 3475200  # checksum_kernel over the 1 625 648 768 B round tables
-
-# Integer operations per rank of the receive-schedule construction as the kernels run it (four
-# ranks per thread share a round's address arithmetic), by q: skip code (3 per level + 5); the six
-# rounds read from the tile's run table 18 each (four words and their addresses 8, the two window
-# sets and the choice between them 4, leading block, its bit and the entry 3, set update, row
-# store, share of the column store); the other rounds 10 each (code load and share of its address
-# 1.5, xor, leading bit, taken-test 4, bit and set update 2, entry, row store, share of the packed
-# column store 1.5); plus 2 for the 0.23 % of the rounds whose first head is taken (CPU count over
-# sampled ranks of p = 2^20+1).
-ALU_MODEL = {21: (3 * 21 + 5) + 6 * 18 + (21 - 6) * 10 + 2}
+def _run_part(args, torch, bcs, workloads, flush, hbm_gbs, sm_max_mhz, peak_src, counts, model):
+    """One part alone, small enough for a profiler (see profiles/ for the commands)."""
+    res = {}
+    if args.only == "probe":
+        probe = Probe(torch)
+        res["int_rate_probe"] = {nm: [probe.rate(mix, 1024) / 1e12 for _ in range(2)]
+                                 for mix, nm in enumerate(("logic_only", "logic_imad_mix", "logic_add_mix"))}
+        res["int_rate_probe"]["unit"] = "Tint-op/s"
+    elif args.only == "build":
+        res["single_p"] = _bench_single(torch, bcs, workloads, flush, args.steps, hbm_gbs, sm_max_mhz, counts,
+                                        model, None)
+    elif args.only == "large-sample":
+        # 2^22 ranks in the middle of p = 2^30-1 through bcs_build with its workspace: the same codes and
+        # receive kernels as the headline's step on 4.4 GB of device memory (the send rows of a
+        # sub-range come from the gather kernel, which the headline does not use)
+        p = workloads.P_LARGE
+        q = bcs.bcs_q(p)
+        r0, r1 = 1 << 29, (1 << 29) + (1 << 22)
+        recv = torch.empty((r1 - r0) * q, dtype=torch.int8, device="cuda")
+        send = torch.empty((r1 - r0) * q, dtype=torch.int8, device="cuda")
+        ws = torch.empty(bcs.bcs_build_workspace_bytes(p, r0, r1), dtype=torch.int8, device="cuda")
+        ms = _event_ms(torch, lambda: bcs.bcs_build(p, r0, r1, recv, send, ws), _no_flush, args.steps, 1)
+        res["large_sample"] = {"p": p, "ranks": r1 - r0, "ms": statistics.mean(ms)}
+    elif args.only == "large-transpose":
+        # the send transposition of the headline on a p with the same q = 30 that fits in 20 GB
+        p = (1 << 29) + 1
+        q = bcs.bcs_q(p)
+        ws = torch.empty(bcs.bcs_prepare_workspace_bytes(p), dtype=torch.int8, device="cuda")
+        bcs.bcs_prepare(p, ws)
+        r0, r1 = 1 << 28, (1 << 28) + (1 << 24)
+        send = torch.empty((r1 - r0) * q, dtype=torch.int8, device="cuda")
+        ms = _event_ms(torch, lambda: bcs.bcs_build_prepared(p, r0, r1, None, send, ws), _no_flush, args.steps, 1)
+        res["large_transpose"] = {"p": p, "ranks": r1 - r0, "ms": statistics.mean(ms)}
+    elif args.only == "allgather":
+        res["allgather_tables"] = _bench_allgather(torch, bcs, workloads, flush, hbm_gbs, peak_src, args.steps,
+                                                   counts)
+    elif args.only in ("expand", "checksum"):
+        ex, table = _bench_expand(torch, bcs, workloads, flush, hbm_gbs, peak_src, args.steps, counts)
+        res["expand"] = ex
+        if args.only == "checksum":
+            res["checksum"] = _bench_checksum(torch, bcs, flush, hbm_gbs, peak_src, table, args.steps, counts)
+    elif args.only == "batch":
+        res = _bench_batch(torch, bcs, workloads, flush, False, hbm_gbs, sm_max_mhz, counts, model, None)
+    return res
 
 
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--only", default="all",
-                    choices=["all", "build", "expand", "checksum", "batch", "allgather", "probe"],
+                    choices=["all", "build", "large-sample", "large-transpose", "expand", "checksum", "batch",
+                             "allgather", "probe"],
                     help="run one part only (small, profiler-friendly runs); 'all' is the benchmark")
     args = ap.parse_args()
     if args.impl == "reference":
