@@ -396,6 +396,20 @@ __device__ __forceinline__ uint32_t bit_or_none(int k)
     return bit;
 }
 
+// Position of the highest set bit, -1 for 0 (one instruction).
+__device__ __forceinline__ int top_bit(uint32_t v)
+{
+    int d;
+    asm("bfind.u32 %0, %1;" : "=r"(d) : "r"(v));
+    return d;
+}
+
+// byte 0 of a, b, c, d as the four bytes of one word
+__device__ __forceinline__ uint32_t pack_bytes(uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    return __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
+}
+
 struct QuadConsts {
     // Table round i, word w (0, 1: the two runs that cover the first window; 2, 3: the second
     // window, or the first again), rank j of the quad: byte offset of that word from the thread's
@@ -642,25 +656,24 @@ __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh
         for (int unrolled = 0; unrolled < kQuadTableRounds; ++unrolled) {
             if (unrolled >= first_lane_round) break;           // uniform over the grid
             i = unrolled;
-            uint32_t packed = 0;
+            uint32_t entry[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const uint32_t free_blocks = ~B[j];
                 uint32_t U = (word(env.word(unrolled, 0, j)) | word(env.word(unrolled, 1, j))) & free_blocks;
                 const uint32_t U2 = (word(env.word(unrolled, 2, j)) | word(env.word(unrolled, 3, j))) & free_blocks;
                 if (U == 0) U = U2;
-                const int lead = __clz(U);                     // 32 when U == 0
-                B[j] |= U ? 0x80000000u >> lead : 0u;
-                const int entry = U ? 31 - q - lead : BCS_BAD_ENTRY;
-                if (kRowOut) row0[j * q + unrolled] = (uint8_t)entry;
-                packed |= ((uint32_t)entry & 0xffu) << (8 * j);
+                const int lead = top_bit(U);                   // -1 when there is no new block at all
+                B[j] |= bit_or_none(lead);
+                entry[j] = U ? (uint32_t)(lead - q) : (uint32_t)BCS_BAD_ENTRY;
+                if (kRowOut) row0[j * q + unrolled] = (uint8_t)entry[j];
             }
             if (kColOut) {
                 if (kPackedCol) {
-                    *reinterpret_cast<uint32_t *>(col) = packed;
+                    *reinterpret_cast<uint32_t *>(col) = pack_bytes(entry[0], entry[1], entry[2], entry[3]);
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) col[j] = (int8_t)(packed >> (8 * j));
+                    for (int j = 0; j < 4; ++j) col[j] = (int8_t)entry[j];
                 }
                 col += t_stride;
             }
@@ -682,9 +695,8 @@ __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh
             }
             if (kColOut) {
                 if (kPackedCol) {
-                    *reinterpret_cast<uint32_t *>(col) =
-                        ((uint32_t)entry[0] & 0xffu) | (((uint32_t)entry[1] & 0xffu) << 8) |
-                        (((uint32_t)entry[2] & 0xffu) << 16) | ((uint32_t)entry[3] << 24);
+                    *reinterpret_cast<uint32_t *>(col) = pack_bytes((uint32_t)entry[0], (uint32_t)entry[1],
+                                                                    (uint32_t)entry[2], (uint32_t)entry[3]);
                 } else {
 #pragma unroll
                     for (int j = 0; j < 4; ++j) col[j] = (int8_t)entry[j];
@@ -703,24 +715,26 @@ __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh
 #pragma unroll
                 for (int j = 0; j < 4; ++j) lower[j] = ahead[j];
                 if (i + 1 < end) load4(ahead, from - env.skip(i + 2));
-                // The first head of each of the four windows, then ONE test whether any of them is
-                // already taken (or its window empty): the four chains stay free of branches.
+                // The first head of each of the four windows and B with its bit; B unchanged means
+                // that the head is already taken or the window empty.  ONE test whether that holds
+                // for any of the four: the four chains stay free of branches.
                 int blk[4];
+                uint32_t with[4];
                 bool taken = false;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    const uint32_t diff = lower[j] ^ upper[j];
-                    blk[j] = 31 - __clz(diff);                 // -1 for an empty window
-                    taken |= diff == 0 || ((B[j] >> blk[j]) & 1u);
+                    blk[j] = top_bit(lower[j] ^ upper[j]);     // -1 for an empty window
+                    with[j] = B[j] | bit_or_none(blk[j]);
+                    taken |= with[j] == B[j];
                 }
                 if (taken) {
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const uint32_t diff = lower[j] ^ upper[j];
-                        if (diff == 0 || ((B[j] >> blk[j]) & 1u)) {
+                        if (with[j] == B[j]) {
                             // The usual case, decided here: the first head is taken and the search
                             // of pick_block ends at its second step, with a new block in the run
                             // of low blocks behind the head.  Everything else: the full search.
+                            const uint32_t diff = lower[j] ^ upper[j];
                             const uint32_t below_head = (1u << (blk[j] & 31)) - 1u;
                             const uint32_t rest = upper[j] & below_head;
                             const uint32_t low = rest ? (2u << (31 - __clz(rest))) - 1u : 0u;
@@ -733,13 +747,14 @@ __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh
                                 b = pick_rest(codes, full_sh, p, q, below + j, lower[j], upper[j],
                                               env.len2(i), B[j]);
                             blk[j] = b >= 0 ? b : BCS_BAD_ENTRY + q;   // entry BCS_BAD_ENTRY, no bit
+                            with[j] = B[j] | bit_or_none(blk[j]);
                         }
                     }
                 }
                 int entry[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    B[j] |= bit_or_none(blk[j]);
+                    B[j] = with[j];
                     entry[j] = blk[j] - q;
                     upper[j] = lower[j];
                 }
