@@ -460,10 +460,10 @@ def _bench_batch(torch, bcs, workloads, flush, full, hbm_gbs, sm_max_mhz, counts
     dplan = plan.to("cuda")
     br = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
     bs = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
-    bw = torch.empty(bcs.bcs_build_batch_workspace_bytes(plan.total_ranks, plan.total_entries),
+    bw = torch.empty(plan.workspace_bytes(),
                      dtype=torch.int8, device="cuda")
     ms = statistics.mean(_event_ms(
-        torch, lambda: bcs.bcs_build_batch(dplan, plan.total_ranks, plan.total_entries, br, bs, bw),
+        torch, lambda: bcs.bcs_build_batch(dplan, br, bs, bw),
         flush, 20, 3))
     batch_kernels = ["codes_batch_kernel", "recv_quad_batch_kernel<true>", "send_batch_kernel"]
     out["batch_small_sweep"] = {
@@ -481,10 +481,10 @@ def _bench_batch(torch, bcs, workloads, flush, full, hbm_gbs, sm_max_mhz, counts
     del br, bs, bw
     br = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
     bs = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
-    bw = torch.empty(bcs.bcs_build_batch_workspace_bytes(plan.total_ranks, plan.total_entries),
+    bw = torch.empty(plan.workspace_bytes(),
                      dtype=torch.int8, device="cuda")
     ms = statistics.mean(_event_ms(
-        torch, lambda: bcs.bcs_build_batch(dplan, plan.total_ranks, plan.total_entries, br, bs, bw),
+        torch, lambda: bcs.bcs_build_batch(dplan, br, bs, bw),
         _no_flush, 3, 1))                          # the outputs exceed L2 by themselves
     out["batch_irregular_sweep"] = {
         "workload": "%d octave-uniform p in [2^10,2^20), seed %d, one bcs_build_batch"

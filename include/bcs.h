@@ -177,29 +177,37 @@ bcs_status bcs_build_to_host(uint32_t p, uint64_t r_begin, uint64_t r_end,
 /* Host helper for bcs_build_batch: for a list of num_p values of p fills
  *   rank_off_host[num_p+1]  prefix sums of p_j            (flattened rank index),
  *   entry_off_host[num_p+1] prefix sums of p_j * q_j      (byte offset of p_j's table),
+ *   tile_off_host[num_p+1]  prefix sums of ceil(p_j / 512) (the fast construction works in tiles
+ *                           of 512 ranks that start anew with every p),
+ *   copy_off_host[num_p+1]  prefix sums of q_j * align16(p_j) (where p_j's round-major scratch
+ *                           copy starts in the workspace; align16 = round up to 16),
  *   skips_tab_host[num_p * BCS_SKIPS_STRIDE] row j = skips[0..q_j] of p_j (Algorithm 1),
  *                           the rest of the row 0,
  *   full_tab_host[num_p * BCS_SKIPS_STRIDE]  row j, word d = skip code of rank
  *                           skips[d]-1 of p_j, d = 0..q_j.
- * The caller copies the four arrays and p_list to the device. */
+ * The caller copies the six arrays and p_list to the device. */
 bcs_status bcs_batch_plan(const uint32_t *p_list_host, uint32_t num_p,
                           uint64_t *rank_off_host, uint64_t *entry_off_host,
+                          uint64_t *tile_off_host, uint64_t *copy_off_host,
                           uint32_t *skips_tab_host, uint32_t *full_tab_host);
 
 /* All ranks of many p at once (the "full schedule" of Algorithm 9 for each p_j),
- * one launch sequence over the flattened list of (p_j, r) pairs.  Device inputs as
- * laid out by bcs_batch_plan; total_ranks = rank_off[num_p], total_entries =
- * entry_off[num_p] (the host knows both).  Outputs: device int8, total_entries
- * bytes each, 16-byte aligned; the table of p_j starts at byte entry_off[j] and
- * is rank-major with q_j bytes per rank.  send_out may be NULL; recv_out is
- * required.  workspace as for bcs_build, of
- * bcs_build_batch_workspace_bytes(total_ranks, total_entries) bytes for the fast
- * construction, or NULL. */
-size_t bcs_build_batch_workspace_bytes(uint64_t total_ranks, uint64_t total_entries);
+ * one launch sequence over the list of (p_j, r) pairs.  Device inputs as laid out by
+ * bcs_batch_plan; total_ranks = rank_off[num_p], total_entries = entry_off[num_p],
+ * total_tiles = tile_off[num_p], total_copy = copy_off[num_p] (the host knows all four).
+ * Outputs: device int8, total_entries bytes each, 16-byte aligned; the table of p_j starts at
+ * byte entry_off[j] and is rank-major with q_j bytes per rank, unpadded.  send_out may be NULL;
+ * recv_out is required.  workspace as for bcs_build, of
+ * bcs_build_batch_workspace_bytes(total_ranks, total_copy) bytes for the fast construction
+ * (which also needs tile_off_dev and copy_off_dev), or NULL: then tile_off_dev and copy_off_dev
+ * may be NULL too and the self-contained construction runs. */
+size_t bcs_build_batch_workspace_bytes(uint64_t total_ranks, uint64_t total_copy);
 bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_dev,
-                           const uint64_t *entry_off_dev, const uint32_t *skips_tab_dev,
+                           const uint64_t *entry_off_dev, const uint64_t *tile_off_dev,
+                           const uint64_t *copy_off_dev, const uint32_t *skips_tab_dev,
                            const uint32_t *full_tab_dev,
                            uint32_t num_p, uint64_t total_ranks, uint64_t total_entries,
+                           uint64_t total_tiles, uint64_t total_copy,
                            int8_t *recv_out, int8_t *send_out,
                            void *workspace, size_t workspace_bytes, void *cuda_stream);
 

@@ -62,11 +62,12 @@ def lib():
         L.bcs_build_static.restype = i32
         L.bcs_build_to_host.argtypes = [u32, u64, u64, vp, vp, vp, _c.c_size_t, vp]
         L.bcs_build_to_host.restype = i32
-        L.bcs_batch_plan.argtypes = [vp, u32, vp, vp, vp, vp]
+        L.bcs_batch_plan.argtypes = [vp, u32, vp, vp, vp, vp, vp, vp]
         L.bcs_batch_plan.restype = i32
         L.bcs_build_batch_workspace_bytes.argtypes = [u64, u64]
         L.bcs_build_batch_workspace_bytes.restype = _c.c_size_t
-        L.bcs_build_batch.argtypes = [vp, vp, vp, vp, vp, u32, u64, u64, vp, vp, vp, _c.c_size_t, vp]
+        L.bcs_build_batch.argtypes = [vp, vp, vp, vp, vp, vp, vp, u32, u64, u64, u64, u64, vp, vp, vp,
+                                      _c.c_size_t, vp]
         L.bcs_build_batch.restype = i32
         L.bcs_expand.argtypes = [u32, u32, u64, u64, vp, vp, vp, vp]
         L.bcs_expand.restype = i32
@@ -201,8 +202,11 @@ class BatchPlan:
     p_list: torch.Tensor      # int32 [num_p]
     rank_off: torch.Tensor    # int64 [num_p+1]
     entry_off: torch.Tensor   # int64 [num_p+1]
+    tile_off: torch.Tensor    # int64 [num_p+1]
+    copy_off: torch.Tensor    # int64 [num_p+1]
     skips_tab: torch.Tensor   # int32 [num_p, 32]
     full_tab: torch.Tensor    # int32 [num_p, 32]
+    totals: tuple = ()        # (ranks, entries, tiles, copy bytes), kept on the host
 
     @property
     def num_p(self) -> int:
@@ -210,16 +214,28 @@ class BatchPlan:
 
     @property
     def total_ranks(self) -> int:
-        return int(self.rank_off[-1])
+        return self.totals[0]
 
     @property
     def total_entries(self) -> int:
-        return int(self.entry_off[-1])
+        return self.totals[1]
+
+    @property
+    def total_tiles(self) -> int:
+        return self.totals[2]
+
+    @property
+    def total_copy(self) -> int:
+        return self.totals[3]
+
+    def workspace_bytes(self) -> int:
+        """bcs_build_batch_workspace_bytes for this plan."""
+        return bcs_build_batch_workspace_bytes(self.total_ranks, self.total_copy)
 
     def to(self, device, non_blocking: bool = False) -> "BatchPlan":
         return BatchPlan(*(t.to(device, non_blocking=non_blocking)
-                           for t in (self.p_list, self.rank_off, self.entry_off, self.skips_tab,
-                                     self.full_tab)))
+                           for t in (self.p_list, self.rank_off, self.entry_off, self.tile_off,
+                                     self.copy_off, self.skips_tab, self.full_tab)), totals=self.totals)
 
 
 def bcs_batch_plan(p_list, pin: bool = False) -> BatchPlan:
@@ -230,30 +246,32 @@ def bcs_batch_plan(p_list, pin: bool = False) -> BatchPlan:
     n = pl.numel()
     # uint32 bit patterns in an int32 tensor
     p32 = torch.where(pl >= 2**31, pl - 2**32, pl).to(torch.int32).contiguous()
-    rank_off = torch.zeros(n + 1, dtype=torch.int64)
-    entry_off = torch.zeros(n + 1, dtype=torch.int64)
+    offs = [torch.zeros(n + 1, dtype=torch.int64) for _ in range(4)]
     skips_tab = torch.zeros((n, BCS_SKIPS_STRIDE), dtype=torch.int32)
     full_tab = torch.zeros((n, BCS_SKIPS_STRIDE), dtype=torch.int32)
     if pin:
-        p32, rank_off, entry_off, skips_tab, full_tab = (
-            t.pin_memory() for t in (p32, rank_off, entry_off, skips_tab, full_tab))
-    _check(lib().bcs_batch_plan(p32.data_ptr(), n, rank_off.data_ptr(), entry_off.data_ptr(),
-                                skips_tab.data_ptr(), full_tab.data_ptr()), "bcs_batch_plan")
-    return BatchPlan(p32, rank_off, entry_off, skips_tab, full_tab)
+        p32, skips_tab, full_tab = (t.pin_memory() for t in (p32, skips_tab, full_tab))
+        offs = [t.pin_memory() for t in offs]
+    _check(lib().bcs_batch_plan(p32.data_ptr(), n, offs[0].data_ptr(), offs[1].data_ptr(),
+                                offs[2].data_ptr(), offs[3].data_ptr(), skips_tab.data_ptr(),
+                                full_tab.data_ptr()), "bcs_batch_plan")
+    return BatchPlan(p32, offs[0], offs[1], offs[2], offs[3], skips_tab, full_tab,
+                     totals=tuple(int(t[-1]) for t in offs))
 
 
-def bcs_build_batch_workspace_bytes(total_ranks: int, total_entries: int) -> int:
-    return lib().bcs_build_batch_workspace_bytes(total_ranks, total_entries)
+def bcs_build_batch_workspace_bytes(total_ranks: int, total_copy: int) -> int:
+    return lib().bcs_build_batch_workspace_bytes(total_ranks, total_copy)
 
 
-def bcs_build_batch(plan_dev: BatchPlan, total_ranks: int, total_entries: int, recv_out, send_out,
-                    workspace=None, stream=None) -> None:
+def bcs_build_batch(plan_dev: BatchPlan, recv_out, send_out, workspace=None, stream=None) -> None:
     """plan_dev: a BatchPlan whose tensors live on the CUDA device; workspace: CUDA tensor of
-    bcs_build_batch_workspace_bytes(...) bytes (fast path) or None."""
+    plan.workspace_bytes() bytes (fast construction) or None."""
     _check(lib().bcs_build_batch(plan_dev.p_list.data_ptr(), plan_dev.rank_off.data_ptr(),
-                                 plan_dev.entry_off.data_ptr(), plan_dev.skips_tab.data_ptr(),
-                                 plan_dev.full_tab.data_ptr(), plan_dev.num_p, total_ranks,
-                                 total_entries, _ptr(recv_out), _ptr(send_out), _ptr(workspace),
+                                 plan_dev.entry_off.data_ptr(), plan_dev.tile_off.data_ptr(),
+                                 plan_dev.copy_off.data_ptr(), plan_dev.skips_tab.data_ptr(),
+                                 plan_dev.full_tab.data_ptr(), plan_dev.num_p, plan_dev.total_ranks,
+                                 plan_dev.total_entries, plan_dev.total_tiles, plan_dev.total_copy,
+                                 _ptr(recv_out), _ptr(send_out), _ptr(workspace),
                                  _nbytes(workspace), _stream(stream)), "bcs_build_batch")
 
 

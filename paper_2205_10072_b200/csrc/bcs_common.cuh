@@ -32,6 +32,10 @@ struct BatchArgs {
     const uint32_t *full_tab;    // [num_p][kRow]
     uint32_t num_p;
     uint64_t total_ranks;
+    // workspace construction only: tiles of 512 ranks that start anew with every p, and where
+    // the round-major copy of each p starts (every round padded to a multiple of 16 bytes)
+    const uint64_t *tile_off;    // [num_p + 1] prefix sums of ceil(p_j / 512)
+    const uint64_t *copy_off;    // [num_p + 1] prefix sums of q_j * align16(p_j)
 };
 
 __host__ __device__ inline int ceil_log2_u32(uint32_t p)
@@ -321,6 +325,6 @@ inline bcs_status check_range(uint32_t p, uint64_t r_begin, uint64_t r_end)
     return BCS_OK;
 }
 
-inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
+__host__ __device__ inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 
 }  // namespace bcs

@@ -816,17 +816,17 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
     }
 }
 
-// Batch: 512 flattened ranks per CTA.  A CTA whose ranks all belong to one p >= 64 (nearly all
-// CTAs when the p are large) runs the quad tile with that p's constants computed into shared
-// memory; a CTA that straddles several p, or a small p, runs the per-lane search rank by rank.
-// The tile's rows start at any byte of the output (staged shifted by that byte's offset in its
-// 16-byte group), and a round of the round-major copy is p bytes long: no packed column stores.
+// Batch: the tiles of 512 ranks start anew with every p (the host's plan gives the prefix sums of
+// the tiles per p), so a CTA works inside ONE p: the quad tile with that p's constants computed
+// into shared memory when p >= 64, the per-lane search for the ranks of a smaller p.  The round-
+// major copy of a p has every round padded to a multiple of 16 bytes, so that the four entries of
+// a quad and round are one aligned word there as in the single-p kernel; the tile's rows start at
+// any byte of the output (staged shifted by that byte's offset in its 16-byte group).
 struct QuadBatchShared {
     uint32_t skips[kRow], full[kRow];
     QuadConsts qc;
-    uint64_t span_begin, span_end;          // bytes of the output that the CTA writes
-    uint64_t rank0, entry0;                 // flattened rank and byte offset of rank 0 of the first p
-    uint32_t j_first, j_last, p_first;
+    uint32_t j, p;                          // index of the tile's p in the list; the p itself
+    uint64_t tile0, rank0, entry0, copy0;   // of that p: first tile, flattened rank 0, first byte, copy
     __align__(16) uint8_t stage[kQuadTile * BCS_MAX_Q + 16];
     uint32_t runs[kRunLevels][kQuadLevelWords];
 };
@@ -837,62 +837,52 @@ recv_quad_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t 
                        int8_t *recv_t)
 {
     __shared__ QuadBatchShared sh;
+    grid_launch_dependents();
     const uint32_t t = threadIdx.x;
-    const uint64_t g0 = (uint64_t)blockIdx.x * kQuadTile;
-    const uint64_t g1 = g0 + kQuadTile < ba.total_ranks ? g0 + kQuadTile : ba.total_ranks;
     if (t < 32) {
-        const uint32_t jf = find_segment_warp(ba.rank_off, ba.num_p, g0);
-        const uint32_t jl = ba.rank_off[jf + 1] >= g1 ? jf : find_segment_warp(ba.rank_off, ba.num_p, g1 - 1);
+        const uint32_t j = find_segment_warp(ba.tile_off, ba.num_p, blockIdx.x);
         if (t == 0) {
-            sh.j_first = jf;
-            sh.j_last = jl;
-            sh.p_first = ba.p_list[jf];
-            sh.rank0 = ba.rank_off[jf];
-            sh.entry0 = ba.entry_off[jf];
-            const int qf = ceil_log2_fast(sh.p_first);
-            const int ql = ceil_log2_fast(ba.p_list[jl]);
-            sh.span_begin = sh.entry0 + (g0 - sh.rank0) * (uint64_t)qf;
-            sh.span_end = ba.entry_off[jl] + (g1 - ba.rank_off[jl]) * (uint64_t)ql;
+            sh.j = j;
+            sh.p = ba.p_list[j];
+            sh.tile0 = ba.tile_off[j];
+            sh.rank0 = ba.rank_off[j];
+            sh.entry0 = ba.entry_off[j];
+            sh.copy0 = ba.copy_off[j];
         }
     }
     __syncthreads();
-    const uint32_t jf = sh.j_first, jl = sh.j_last;
-    const uint32_t shift = (uint32_t)(sh.span_begin & 15u);
-    if (jf == jl && sh.p_first >= 64u) {                           // uniform over the CTA
-        const uint32_t p = sh.p_first;
-        const int q = ceil_log2_fast(p);
-        const uint32_t *skips = ba.skips_tab + (size_t)jf * kRow;  // the constants of this p
+    const uint32_t j = sh.j, p = sh.p;
+    const int q = ceil_log2_fast(p);
+    if (q == 0) return;                                            // p == 1: a tile without entries
+    const uint32_t first = (uint32_t)(blockIdx.x - sh.tile0) * kQuadTile;
+    const uint32_t n = p - first < (uint32_t)kQuadTile ? p - first : (uint32_t)kQuadTile;
+    const uint64_t span_begin = sh.entry0 + (uint64_t)first * (uint64_t)q;
+    const uint32_t shift = (uint32_t)(span_begin & 15u);
+    const uint64_t pitch = align_up(p, 16);
+    const uint32_t *skips = ba.skips_tab + (size_t)j * kRow;       // the constants of this p
+    int8_t *col_tile = kColOut ? recv_t + sh.copy0 + first : nullptr;
+    if (p >= 64u) {                                                // uniform over the CTA
         if (t < kRow) {
             sh.skips[t] = skips[t];
-            sh.full[t] = ba.full_tab[(size_t)jf * kRow + t];
+            sh.full[t] = ba.full_tab[(size_t)j * kRow + t];
             if (t < (uint32_t)q) sh.qc.len2[t] = quad_len2(skips, (int)t);
             if (t == 0) sh.qc.table_rounds = quad_table_rounds(skips, q);
         } else if (t < kRow + kQuadTableRounds * 16 && (int)((t - kRow) >> 4) < q) {
             const uint32_t e = t - kRow;                           // round e / 16, word (e / 4) % 4, rank e % 4
             sh.qc.word[e >> 4][(e >> 2) & 3u][e & 3u] = quad_word_offset(skips, (int)(e >> 4), (int)((e >> 2) & 3u), (int)(e & 3u));
         }
-        // (the tile's first barrier comes before anything here is read)
-        const uint64_t first = g0 - sh.rank0;
-        quad_tile<true, kColOut, false>(SharedEnv{sh.skips, &sh.qc}, sh.full, p, q, first, (uint32_t)(g1 - g0),
-                                        codes + sh.rank0, sh.stage + shift,
-                                        kColOut ? recv_t + sh.entry0 + first : nullptr, (uint64_t)p, sh.runs);
+        grid_dependency_wait();                                    // the codes are complete from here on
+        // (the tile's first barrier comes before anything above is read)
+        quad_tile<true, kColOut, true>(SharedEnv{sh.skips, &sh.qc}, sh.full, p, q, first, n, codes + sh.rank0,
+                                       sh.stage + shift, col_tile, pitch, sh.runs);
     } else {
-        for (uint64_t g = g0 + t; g < g1; g += kQuadThreads) {
-            const uint32_t j = find_segment(ba.rank_off, jf, jl, g);
-            const uint32_t p = ba.p_list[j];
-            const int q = ceil_log2_fast(p);
-            if (q == 0) continue;
-            const uint64_t rank0 = ba.rank_off[j], entry0 = ba.entry_off[j];
-            const uint32_t r = (uint32_t)(g - rank0);
-            uint8_t *row = sh.stage + shift + (entry0 + (uint64_t)r * (uint64_t)q - sh.span_begin);
-            int8_t *col = kColOut ? recv_t + entry0 + r : nullptr;
-            recv_rounds_codes<true, kColOut>(codes + rank0, ba.skips_tab + (size_t)j * kRow,
-                                             ba.full_tab + (size_t)j * kRow, p, q, r, q - 1, row, col,
-                                             (uint64_t)p);
-        }
+        grid_dependency_wait();
+        if (t < n)
+            recv_rounds_codes<true, kColOut>(codes + sh.rank0, skips, ba.full_tab + (size_t)j * kRow, p, q, t, q - 1,
+                                             sh.stage + shift + t * (uint32_t)q, kColOut ? col_tile + t : nullptr, pitch);
     }
     __syncthreads();
-    flush_span(sh.stage, shift, (uint32_t)(sh.span_end - sh.span_begin), recv_out, sh.span_begin);
+    flush_span(sh.stage, shift, n * (uint32_t)q, recv_out, span_begin);
 }
 
 // Send rows of a sub-range of one p from the round-major receive copy of that range;
@@ -1089,6 +1079,7 @@ __device__ __forceinline__ void gather_rows_unaligned(const BatchRoundBuffer &rb
 {
     uint32_t W[kQ];
     load_four_ranks(rb, threadIdx.x, W);
+    __syncthreads();                                          // everyone has read: `out` may lie in the round buffer
     uint8_t *mine = out + 4u * threadIdx.x * kQ;
     const uint32_t sh = (uint32_t)(__cvta_generic_to_shared(mine) & 3u);
     uint32_t *words = reinterpret_cast<uint32_t *>(mine - sh);
@@ -1151,15 +1142,14 @@ inline void launch_transpose(const PTable &tab, const int8_t *recv_t, uint64_t t
                                          dependent, stream);
 }
 
-// Batch: 256 flattened ranks and 64 threads per CTA, as in the single-p kernel.  A CTA inside one
-// p transposes; a CTA that straddles several p gathers byte by byte.
+// Batch: 256 ranks and 64 threads per CTA, as in the single-p kernel; two CTAs per tile of the
+// plan (512 ranks of one p), the second with nothing to do where a p ends in the first half.
 struct SendBatchShared {
     uint32_t skips[kRow];
-    uint64_t span_begin, span_end;          // bytes of the output that the CTA writes
-    uint64_t rank0, entry0;                 // flattened rank and byte offset of rank 0 of the first p
-    uint32_t j_first, j_last, p_first;
-    __align__(16) uint8_t stage[kStageBytes];
+    uint32_t j, p;
+    uint64_t tile0, entry0, copy0;
 };
+static_assert(BCS_MAX_Q * kTrPitch >= kTile * BCS_MAX_Q + 16, "the rows of a tile fit in its round buffer");
 
 __global__ void __launch_bounds__(kTrThreads, 16)
 send_batch_kernel(BatchArgs ba, const int8_t *__restrict__ recv_t, int8_t *send_out)
@@ -1167,55 +1157,33 @@ send_batch_kernel(BatchArgs ba, const int8_t *__restrict__ recv_t, int8_t *send_
     __shared__ SendBatchShared sh;
     __shared__ BatchRoundBuffer rb;
     const uint32_t t = threadIdx.x;
-    const uint64_t g0 = (uint64_t)blockIdx.x * kTile;
-    const uint64_t g1 = g0 + kTile < ba.total_ranks ? g0 + kTile : ba.total_ranks;
+    const uint64_t tile = blockIdx.x >> 1;
     if (t < 32) {
-        const uint32_t jf = find_segment_warp(ba.rank_off, ba.num_p, g0);
-        const uint32_t jl = ba.rank_off[jf + 1] >= g1 ? jf : find_segment_warp(ba.rank_off, ba.num_p, g1 - 1);
-        sh.skips[t] = ba.skips_tab[(size_t)jf * kRow + t];
+        const uint32_t j = find_segment_warp(ba.tile_off, ba.num_p, tile);
+        sh.skips[t] = ba.skips_tab[(size_t)j * kRow + t];
         if (t == 0) {
-            sh.j_first = jf;
-            sh.j_last = jl;
-            sh.p_first = ba.p_list[jf];
-            sh.rank0 = ba.rank_off[jf];
-            sh.entry0 = ba.entry_off[jf];
-            const int qf = ceil_log2_fast(sh.p_first);
-            const int ql = ceil_log2_fast(ba.p_list[jl]);
-            sh.span_begin = sh.entry0 + (g0 - sh.rank0) * (uint64_t)qf;
-            sh.span_end = ba.entry_off[jl] + (g1 - ba.rank_off[jl]) * (uint64_t)ql;
+            sh.j = j;
+            sh.p = ba.p_list[j];
+            sh.tile0 = ba.tile_off[j];
+            sh.entry0 = ba.entry_off[j];
+            sh.copy0 = ba.copy_off[j];
         }
     }
     __syncthreads();
-    const uint32_t jf = sh.j_first, jl = sh.j_last;
-    const uint32_t shift = (uint32_t)(sh.span_begin & 15u);
-    if (jf == jl) {                                            // uniform over the CTA
-        const uint32_t p = sh.p_first;
-        const int q = ceil_log2_fast(p);
-        if (q > 0) {
-            if (!load_rounds(SharedSkips{sh.skips}, p, q, recv_t + sh.entry0, (uint64_t)p,
-                             (uint32_t)(g0 - sh.rank0), (uint32_t)(g1 - g0), true, rb))
-                return;
-            GatherDispatch<BCS_MAX_Q>::run(q, rb, sh.stage + shift);
-        }
-    } else {
-        for (uint64_t g = g0 + t; g < g1; g += kTrThreads) {
-            const uint32_t j = find_segment(ba.rank_off, jf, jl, g);
-            const uint32_t p = ba.p_list[j];
-            const int q = ceil_log2_fast(p);
-            const uint64_t entry0 = ba.entry_off[j];
-            const uint32_t r = (uint32_t)(g - ba.rank_off[j]);
-            const uint32_t *skips = ba.skips_tab + (size_t)j * kRow;
-            uint8_t *row = sh.stage + shift + (entry0 + (uint64_t)r * (uint64_t)q - sh.span_begin);
-            const int8_t *tbl = recv_t + entry0;
-            for (int k = 0; k < q; ++k) {
-                uint32_t to = r + skips[k];
-                if (to >= p) to -= p;
-                row[k] = (uint8_t)tbl[(uint64_t)k * p + to];
-            }
-        }
-    }
+    const uint32_t p = sh.p;
+    const int q = ceil_log2_fast(p);
+    const uint64_t first64 = (tile - sh.tile0) * kQuadTile + (blockIdx.x & 1u) * kTile;
+    if (q == 0 || first64 >= p) return;                            // uniform over the CTA
+    const uint32_t first = (uint32_t)first64;
+    const uint32_t n = p - first < (uint32_t)kTile ? p - first : (uint32_t)kTile;
+    const uint64_t span_begin = sh.entry0 + (uint64_t)first * (uint64_t)q;
+    const uint32_t shift = (uint32_t)(span_begin & 15u);
+    if (!load_rounds(SharedSkips{sh.skips}, p, q, recv_t + sh.copy0, align_up(p, 16), first, n, true, rb))
+        return;
+    // the rows take the round buffer over (after a barrier inside the gather): 9 KB per CTA
+    GatherDispatch<BCS_MAX_Q>::run(q, rb, rb.rounds + shift);
     __syncthreads();
-    flush_span(sh.stage, shift, (uint32_t)(sh.span_end - sh.span_begin), send_out, sh.span_begin);
+    flush_span(rb.rounds, shift, n * (uint32_t)q, send_out, span_begin);
 }
 
 struct Workspace {
@@ -1533,17 +1501,19 @@ bcs_status bcs_build_to_host(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_
     return BCS_OK;
 }
 
-size_t bcs_build_batch_workspace_bytes(uint64_t total_ranks, uint64_t total_entries)
+size_t bcs_build_batch_workspace_bytes(uint64_t total_ranks, uint64_t total_copy)
 {
-    if (total_ranks == 0 || total_entries == 0) return 0;
-    return (size_t)(align_up(4ull * total_ranks, 256) + align_up(total_entries, 16) + 16);
+    if (total_ranks == 0 || total_copy == 0) return 0;
+    return (size_t)(align_up(4ull * total_ranks, 256) + total_copy);
 }
 
 bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_dev,
-                           const uint64_t *entry_off_dev, const uint32_t *skips_tab_dev,
+                           const uint64_t *entry_off_dev, const uint64_t *tile_off_dev,
+                           const uint64_t *copy_off_dev, const uint32_t *skips_tab_dev,
                            const uint32_t *full_tab_dev, uint32_t num_p, uint64_t total_ranks,
-                           uint64_t total_entries, int8_t *recv_out, int8_t *send_out,
-                           void *workspace, size_t workspace_bytes, void *cuda_stream)
+                           uint64_t total_entries, uint64_t total_tiles, uint64_t total_copy,
+                           int8_t *recv_out, int8_t *send_out, void *workspace, size_t workspace_bytes,
+                           void *cuda_stream)
 {
     if (num_p == 0 || total_ranks == 0) return BCS_OK;
     if (p_list_dev == nullptr || rank_off_dev == nullptr || entry_off_dev == nullptr ||
@@ -1553,27 +1523,30 @@ bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_
     if (recv_out == nullptr) return BCS_ERR_ARG;
     if (!aligned16(recv_out) || !aligned16(send_out) || !aligned16(workspace)) return BCS_ERR_ALIGN;
     const uint64_t blocks64 = (total_ranks + kTile - 1) / kTile;
-    if (blocks64 > 0x7fffffffull) return BCS_ERR_UNSUPPORTED;
+    if (blocks64 > 0x7fffffffull || total_tiles > 0x3fffffffull) return BCS_ERR_UNSUPPORTED;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     BatchArgs ba = {p_list_dev, rank_off_dev, entry_off_dev, skips_tab_dev, full_tab_dev, num_p,
-                    total_ranks};
+                    total_ranks, tile_off_dev, copy_off_dev};
     PTable none = {};
     const unsigned blocks = (unsigned)blocks64;
     bcs_status st;
-    if (workspace != nullptr &&
-        workspace_bytes >= bcs_build_batch_workspace_bytes(total_ranks, total_entries)) {
+    if (workspace != nullptr && tile_off_dev != nullptr && copy_off_dev != nullptr && total_tiles != 0 &&
+        workspace_bytes >= bcs_build_batch_workspace_bytes(total_ranks, total_copy)) {
         uint32_t *codes = static_cast<uint32_t *>(workspace);
         int8_t *recv_t = static_cast<int8_t *>(workspace) + align_up(4ull * total_ranks, 256);
         codes_batch_kernel<<<(unsigned)((total_ranks + kCodesTile - 1) / kCodesTile), kTile, 0, stream>>>(ba, codes);
         if ((st = launch_status()) != BCS_OK) return st;
-        const unsigned qblocks = (unsigned)((total_ranks + kQuadTile - 1) / kQuadTile);
+        // the receive and the send kernel are launched as dependents of the kernel before them
         if (send_out != nullptr)
-            recv_quad_batch_kernel<true><<<qblocks, kQuadThreads, 0, stream>>>(ba, codes, recv_out, recv_t);
+            launch_dependent(true, recv_quad_batch_kernel<true>, (unsigned)total_tiles, kQuadThreads, stream, ba,
+                             (const uint32_t *)codes, recv_out, recv_t);
         else
-            recv_quad_batch_kernel<false><<<qblocks, kQuadThreads, 0, stream>>>(ba, codes, recv_out, nullptr);
+            launch_dependent(true, recv_quad_batch_kernel<false>, (unsigned)total_tiles, kQuadThreads, stream, ba,
+                             (const uint32_t *)codes, recv_out, (int8_t *)nullptr);
         if ((st = launch_status()) != BCS_OK) return st;
         if (send_out != nullptr) {
-            send_batch_kernel<<<blocks, kTrThreads, 0, stream>>>(ba, recv_t, send_out);
+            launch_dependent(true, send_batch_kernel, (unsigned)(2 * total_tiles), kTrThreads, stream, ba,
+                             (const int8_t *)recv_t, send_out);
             if ((st = launch_status()) != BCS_OK) return st;
         }
         return BCS_OK;

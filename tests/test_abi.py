@@ -66,6 +66,9 @@ def test_batch_plan_host_side(lib):
     plan = lib.bcs_batch_plan([2, 3, 20, 1, 1025])
     assert plan.rank_off.tolist() == [0, 2, 5, 25, 26, 1051]
     assert plan.entry_off.tolist() == [0, 2, 8, 108, 108, 108 + 1025 * 11]
+    assert plan.tile_off.tolist() == [0, 1, 2, 3, 4, 7]                    # ceil(p / 512) tiles per p
+    assert plan.copy_off.tolist() == [0, 16, 48, 208, 208, 208 + 11 * 1040]  # q rounds of align16(p) bytes
+    assert plan.total_tiles == 7 and plan.workspace_bytes() == 4352 + 208 + 11 * 1040
     assert plan.skips_tab[2].tolist()[:6] == [1, 2, 3, 5, 10, 20]
     assert plan.skips_tab[3].tolist()[:2] == [1, 0]
     # full_tab[d] = skip code of rank skips[d]-1: p = 20, skips 1 2 3 5 10 20:
@@ -89,12 +92,13 @@ def test_argument_errors_need_no_gpu(lib):
     assert L.bcs_build(10, 3, 3, None, None, None, 0, None) == 0 # empty range
     assert L.bcs_build_workspace_bytes(2**20 + 1, 0, 2**20 + 1) == 4194560 + 21 * 1048592
     assert L.bcs_build_workspace_bytes(0, 0, 0) == 0
-    assert L.bcs_build_batch_workspace_bytes(1000, 9000) == 4096 + 9008 + 16
+    assert L.bcs_build_batch_workspace_bytes(1000, 9008) == 4096 + 9008
     assert L.bcs_expand(10, 0, 0, 10, 16, 16, 16, None) == 1     # n == 0
     assert L.bcs_expand(10, 4, 0, 10, None, 16, 16, None) == 1
     assert L.bcs_expand(10, 4, 0, 10, 16, 16, 8, None) == 3
     assert L.bcs_checksum(16, 8, 2, 16, None) == 3               # first index not a multiple of 4
     assert L.bcs_checksum(16, 8, 0, None, None) == 1
-    assert L.bcs_build_batch(None, None, None, None, None, 3, 10, 40, 16, None, None, 0, None) == 1
+    assert L.bcs_build_batch(None, None, None, None, None, None, None, 3, 10, 40, 1, 48, 16, None, None, 0,
+                             None) == 1
     assert L.bcs_build_to_host(10, 0, 10, None, None, 16, 1024, None) == 1
     assert L.bcs_build_to_host(10, 0, 10, 16, None, 16, 16, None) == 1   # staging too small

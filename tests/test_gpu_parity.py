@@ -80,7 +80,7 @@ def test_every_p_up_to_1024_single_calls(bcs, fast):
 def _batch_ws(bcs, plan, fast):
     if not fast:
         return None, None
-    return _guarded(bcs.bcs_build_batch_workspace_bytes(plan.total_ranks, plan.total_entries))
+    return _guarded(plan.workspace_bytes())
 
 
 @pytest.mark.parametrize("fast", [True, False])
@@ -92,7 +92,7 @@ def test_every_p_up_to_1024_batched_and_simulated(bcs, fast):
     raw_r, recv = _guarded(plan.total_entries)
     raw_s, send = _guarded(plan.total_entries)
     raw_w, ws = _batch_ws(bcs, plan, fast)
-    bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, send, ws)
+    bcs.bcs_build_batch(dev, recv, send, ws)
     torch.cuda.synchronize()
     assert raw_w is None or _guards_intact(raw_w, ws.numel())
     assert _guards_intact(raw_r, plan.total_entries) and _guards_intact(raw_s, plan.total_entries)
@@ -121,7 +121,7 @@ def test_batch_with_trivial_and_duplicate_p(bcs, fast):
     raw_r, recv = _guarded(plan.total_entries)
     raw_s, send = _guarded(plan.total_entries)
     raw_w, ws = _batch_ws(bcs, plan, fast)
-    bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, send, ws)
+    bcs.bcs_build_batch(dev, recv, send, ws)
     torch.cuda.synchronize()
     assert raw_w is None or _guards_intact(raw_w, ws.numel())
     assert _guards_intact(raw_r, plan.total_entries) and _guards_intact(raw_s, plan.total_entries)
@@ -135,7 +135,7 @@ def test_batch_with_trivial_and_duplicate_p(bcs, fast):
         assert np.array_equal(send[eo[j]:eo[j + 1]].cpu().numpy().reshape(p, -1), want_s)
     # receive table alone
     raw_r, recv = _guarded(plan.total_entries)
-    bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, None, ws)
+    bcs.bcs_build_batch(dev, recv, None, ws)
     torch.cuda.synchronize()
     assert np.array_equal(recv[eo[3]:eo[4]].cpu().numpy().reshape(300, -1), oracle.full_table(300)[0])
 
@@ -182,8 +182,8 @@ def test_seeded_p_sweep_full_tables_sub_ranges_and_one_batch(bcs):
     dplan = plan.to("cuda")
     raw_r, recv = _guarded(plan.total_entries)
     raw_s, send = _guarded(plan.total_entries)
-    raw_w, ws = _guarded(bcs.bcs_build_batch_workspace_bytes(plan.total_ranks, plan.total_entries))
-    bcs.bcs_build_batch(dplan, plan.total_ranks, plan.total_entries, recv, send, ws)
+    raw_w, ws = _guarded(plan.workspace_bytes())
+    bcs.bcs_build_batch(dplan, recv, send, ws)
     torch.cuda.synchronize()
     assert bcs.bcs_wait_expired() == 0
     assert _guards_intact(raw_r, plan.total_entries) and _guards_intact(raw_s, plan.total_entries)
@@ -419,9 +419,9 @@ def test_batched_irregular_sweep_full_size(bcs):
     dev = plan.to("cuda")
     recv = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
     send = torch.empty(plan.total_entries, dtype=torch.int8, device="cuda")
-    ws = torch.empty(bcs.bcs_build_batch_workspace_bytes(plan.total_ranks, plan.total_entries),
+    ws = torch.empty(plan.workspace_bytes(),
                      dtype=torch.int8, device="cuda")
-    bcs.bcs_build_batch(dev, plan.total_ranks, plan.total_entries, recv, send, ws)
+    bcs.bcs_build_batch(dev, recv, send, ws)
     torch.cuda.synchronize()
     assert bcs.bcs_wait_expired() == 0
     del ws
