@@ -832,7 +832,7 @@ struct QuadBatchShared {
 };
 
 template <bool kColOut>
-__global__ void __launch_bounds__(kQuadThreads, 7)
+__global__ void __launch_bounds__(kQuadThreads, 6)
 recv_quad_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t *recv_out,
                        int8_t *recv_t)
 {
