@@ -100,5 +100,15 @@ def test_argument_errors_need_no_gpu(lib):
     assert L.bcs_checksum(16, 8, 0, None, None) == 1
     assert L.bcs_build_batch(None, None, None, None, None, None, None, 3, 10, 40, 1, 48, 16, None, None, 0,
                              None) == 1
+    assert L.bcs_prepare_codes(0, 16, 1 << 20, None) == 2
+    assert L.bcs_prepare_codes(1000, None, 0, None) == 1
+    assert L.bcs_prepare_codes(1000, 16, 64, None) == 1                       # workspace too small
+    assert L.bcs_prepare_codes(1000, 8, 1 << 20, None) == 3                    # misaligned workspace
+    assert L.bcs_prepare_rows(1000, 8, 100, 16, 16, 1 << 20, None) == 3        # r_begin not a multiple of 16
+    assert L.bcs_prepare_rows(1000, 16, 1001, 16, 16, 1 << 20, None) == 2
+    assert L.bcs_prepare_rows(1000, 16, 100, 24, 16, 1 << 20, None) == 3       # misaligned rows
+    assert L.bcs_prepare_rows(1000, 16, 16, None, 16, 1 << 20, None) == 0      # empty range
+    assert L.bcs_prepare_workspace_bytes(1000) == 4096 + 10 * 1008
+    assert L.bcs_expand(10, 4, 0, 10, None, None, None, None) == 1             # no table to write to
     assert L.bcs_build_to_host(10, 0, 10, None, None, 16, 1024, None) == 1
     assert L.bcs_build_to_host(10, 0, 10, 16, None, 16, 16, None) == 1   # staging too small
