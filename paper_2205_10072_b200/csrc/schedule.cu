@@ -417,6 +417,10 @@ struct QuadConsts {
     int32_t word[kQuadTableRounds][4][4];
     uint32_t len2[kRow];     // length of the second window of round i, or 0
     int table_rounds;        // rounds 0 .. table_rounds-1 are decided from the run table
+    // bit k of aligned[w]: the four window bounds that a quad loads at its first rank minus
+    // skips[k] (w = 0) or plus p minus skips[k] (w = 1: past the home round) start on a 16-byte
+    // boundary of the codes, so that they can be loaded as one 16-byte word
+    uint32_t aligned[2];
     // tiles that (may) hold a quad for the general code: those of the ranks skips[k], the first
     // and the last of the range; distinct, n_special <= 32 (missing one costs time, not correctness)
     uint32_t special[kRow];
@@ -480,6 +484,11 @@ inline QuadConsts make_quad_consts(const PTable &tab, uint64_t r_begin, uint64_t
     }
     for (int i = 0; i < tab.q; ++i) qc.len2[i] = quad_len2(tab.s, i);
     qc.table_rounds = quad_table_rounds(tab.s, tab.q);
+    // quads start at ranks r_begin + multiples of 4, the codes at a 16-byte boundary
+    for (int k = 0; k <= tab.q; ++k) {
+        if ((((uint32_t)r_begin - tab.s[k]) & 3u) == 0) qc.aligned[0] |= 1u << k;
+        if ((((uint32_t)r_begin + tab.p - tab.s[k]) & 3u) == 0) qc.aligned[1] |= 1u << k;
+    }
     for (int i = 0; i < qc.table_rounds; ++i)
         for (int w = 0; w < 4; ++w)
             for (int j = 0; j < 4; ++j) qc.word[i][w][j] = quad_word_offset(tab.s, i, w, j);
@@ -495,6 +504,7 @@ struct ParamEnv {
     __device__ __forceinline__ int word(int i, int w, int j) const { return qc.word[i][w][j]; }
     __device__ __forceinline__ uint32_t len2(int i) const { return qc.len2[i]; }
     __device__ __forceinline__ int table_rounds() const { return qc.table_rounds; }
+    __device__ __forceinline__ uint32_t aligned(int w) const { return qc.aligned[w]; }
 };
 // ... or shared memory (batch: the CTA computes them for the p of its tile).
 struct SharedEnv {
@@ -504,6 +514,7 @@ struct SharedEnv {
     __device__ __forceinline__ int word(int i, int w, int j) const { return qc->word[i][w][j]; }
     __device__ __forceinline__ uint32_t len2(int i) const { return qc->len2[i]; }
     __device__ __forceinline__ int table_rounds() const { return qc->table_rounds; }
+    __device__ __forceinline__ uint32_t aligned(int w) const { return qc->aligned[w]; }
 };
 
 // One tile: the n <= 512 ranks first .. first+n-1 of a p >= 64 (first may exceed p for the
@@ -512,7 +523,7 @@ struct SharedEnv {
 // col_tile: byte of the tile's first rank in round 0 of the round-major copy, rounds t_stride
 // bytes apart (kPackedCol: both multiples of 4, so that the four entries of a quad and round are
 // stored as one word).
-template <bool kRowOut, bool kColOut, bool kPackedCol, class Env>
+template <bool kRowOut, bool kColOut, bool kPackedCol, bool kWideLoads, class Env>
 __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh, uint32_t p, int q,
                                           uint64_t first, uint32_t n,
                                           const uint32_t *__restrict__ codes, uint8_t *stage,
@@ -681,10 +692,23 @@ __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh
         }
         // Per-lane rounds.  upper[j]: code of r[j] - skips[i]; lower[j]: code of r[j] - skips[i+1].
         uint32_t upper[4], lower[4];
-        auto load4 = [&](uint32_t (&dst)[4], uint32_t index) {
-            const uint32_t *src = codes + index;
+        // The four bounds of a quad are four consecutive words.  Where they start in their 16-byte
+        // group is the same for all quads of a launch (the ranks of quads are multiples of 4
+        // apart); where they fill the group -- skips that are multiples of 4, e.g. the powers of
+        // two of a p just below one -- they come as ONE 16-byte load, which touches a quarter of
+        // the L1 sectors of four one-word loads with the lanes 16 bytes apart.  The host says for
+        // which skips that holds (a test on the address would not be uniform for the compiler) and
+        // picks the instantiation with this test only for a p with many such skips: the test
+        // costs the other rounds a few percent.
+        auto load4 = [&](uint32_t (&dst)[4], uint32_t from, int k, uint32_t aligned_skips) {
+            const uint32_t *src = codes + (from - env.skip(k));
+            if (kWideLoads && ((aligned_skips >> k) & 1u)) {
+                const uint4 v = *reinterpret_cast<const uint4 *>(src);
+                dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+            } else {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) dst[j] = src[j];
+                for (int j = 0; j < 4; ++j) dst[j] = src[j];
+            }
         };
         uint8_t *out = row0 + i;
         auto store_round = [&](const int (&entry)[4]) {
@@ -705,16 +729,16 @@ __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh
             }
         };
         // rounds i .. end-1 with the window bounds at from - skip (from = r[0] or r[0] + p)
-        auto rounds_until = [&](int end, uint32_t from) {
+        auto rounds_until = [&](int end, uint32_t from, const uint32_t aligned_skips) {
             if (i >= end) return;
             uint32_t ahead[4];
-            load4(ahead, from - env.skip(i + 1));
+            load4(ahead, from, i + 1, aligned_skips);
 #pragma unroll 2
             for (; i < end; ++i) {
                 const uint32_t below = from - env.skip(i + 1);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) lower[j] = ahead[j];
-                if (i + 1 < end) load4(ahead, from - env.skip(i + 2));
+                if (i + 1 < end) load4(ahead, from, i + 2, aligned_skips);
                 // The first head of each of the four windows and B with its bit; B unchanged means
                 // that the head is already taken or the window empty.  ONE test whether that holds
                 // for any of the four: the four chains stay free of branches.
@@ -761,21 +785,21 @@ __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh
                 store_round(entry);
             }
         };
-        load4(upper, r[0] - env.skip(i));                         // i <= h0: skips[i] <= r[0]
-        rounds_until(h0, r[0]);
+        load4(upper, r[0], i, env.aligned(0));                   // i <= h0: skips[i] <= r[0]
+        rounds_until(h0, r[0], env.aligned(0));
         {                                                      // home round: the baseblocks themselves
             int entry[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) entry[j] = __ffs(c[j]) - 1;
             store_round(entry);
-            load4(upper, r[0] + p - env.skip(h0 + 1));            // r[3] < skips[h0+1]
+            load4(upper, r[0] + p, h0 + 1, env.aligned(1));       // r[3] < skips[h0+1]
             i = h0 + 1;
         }
-        rounds_until(q, r[0] + p);
+        rounds_until(q, r[0] + p, env.aligned(1));
     }
 }
 
-template <bool kRowOut, bool kColOut>
+template <bool kRowOut, bool kColOut, bool kWideLoads>
 __global__ void __launch_bounds__(kQuadThreads, 8)
 recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant__ QuadConsts qc,
                        uint64_t r_begin, uint64_t r_end, const uint32_t *__restrict__ codes,
@@ -803,7 +827,7 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
     const uint64_t g0 = tile * kQuadTile;
     const uint32_t n = (uint32_t)(count - g0 < (uint64_t)kQuadTile ? count - g0 : (uint64_t)kQuadTile);
     // g0 and t_stride are multiples of 4 and recv_t is 16-byte aligned: packed column stores
-    quad_tile<kRowOut, kColOut, true>(ParamEnv{tab, qc}, full_sh, p, q, r_begin + g0, n, codes, stage,
+    quad_tile<kRowOut, kColOut, true, kWideLoads>(ParamEnv{tab, qc}, full_sh, p, q, r_begin + g0, n, codes, stage,
                                       kColOut ? recv_t + g0 : nullptr, t_stride, runs);
     if (kRowOut) {
         const uint32_t len = n * (uint32_t)q;                  // the tile's rows start at byte g0 * q: 16-byte aligned
@@ -873,7 +897,7 @@ recv_quad_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t 
         }
         grid_dependency_wait();                                    // the codes are complete from here on
         // (the tile's first barrier comes before anything above is read)
-        quad_tile<true, kColOut, true>(SharedEnv{sh.skips, &sh.qc}, sh.full, p, q, first, n, codes + sh.rank0,
+        quad_tile<true, kColOut, true, false>(SharedEnv{sh.skips, &sh.qc}, sh.full, p, q, first, n, codes + sh.rank0,
                                        sh.stage + shift, col_tile, pitch, sh.runs);
     } else {
         grid_dependency_wait();
@@ -1186,6 +1210,31 @@ send_batch_kernel(BatchArgs ba, const int8_t *__restrict__ recv_t, int8_t *send_
     flush_span(rb.rounds, shift, n * (uint32_t)q, send_out, span_begin);
 }
 
+// Launches the quad receive kernel of one p >= 64 for a range, as a dependent of the kernel
+// before it on the stream.  The instantiation that loads aligned window bounds as 16-byte words
+// is taken when the bounds of at least four fifths of the rounds before the home round are
+// aligned (a p just below a power of two: its skips are powers of two); measured, it gains
+// 2-5 % there and loses as much where only few rounds, or only those past the home round, are.
+template <bool kRowOut, bool kColOut>
+inline void launch_recv_quad(const PTable &tab, const QuadConsts &qc, uint64_t r_begin, uint64_t r_end,
+                             const uint32_t *codes, int8_t *recv_out, int8_t *recv_t, uint64_t t_stride,
+                             cudaStream_t stream)
+{
+    const uint64_t count = r_end - r_begin;
+    const unsigned grid = (unsigned)((count + kQuadTile - 1) / kQuadTile) + (unsigned)qc.n_special;
+    int wide = 0, rounds = 0;
+    for (int k = qc.table_rounds + 1; k <= tab.q; ++k) {
+        wide += (int)((qc.aligned[0] >> k) & 1u);
+        rounds += 1;
+    }
+    if (5 * wide >= 4 * rounds)
+        launch_dependent(true, recv_codes_quad_kernel<kRowOut, kColOut, true>, grid, kQuadThreads, stream, tab, qc,
+                         r_begin, r_end, codes, recv_out, recv_t, t_stride);
+    else
+        launch_dependent(true, recv_codes_quad_kernel<kRowOut, kColOut, false>, grid, kQuadThreads, stream, tab, qc,
+                         r_begin, r_end, codes, recv_out, recv_t, t_stride);
+}
+
 struct Workspace {
     uint32_t *codes;
     int8_t *recv_t;
@@ -1250,25 +1299,21 @@ bcs_status bcs_build(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t *recv_
         if ((st = launch_status()) != BCS_OK) return st;
         const bool warp_rounds = p >= 64;      // the table kernel needs 64 distinct ranks back
         const QuadConsts rc = make_quad_consts(tab, r_begin, r_end);
-        const unsigned qblocks = (unsigned)((count + kQuadTile - 1) / kQuadTile) + (unsigned)rc.n_special;
         if (recv_out != nullptr && send_out != nullptr) {
             if (warp_rounds)
-                launch_dependent(true, recv_codes_quad_kernel<true, true>, qblocks, kQuadThreads, stream, tab, rc,
-                                 r_begin, r_end, ws.codes, recv_out, ws.recv_t, ws.t_stride);
+                launch_recv_quad<true, true>(tab, rc, r_begin, r_end, ws.codes, recv_out, ws.recv_t, ws.t_stride, stream);
             else
                 recv_codes_kernel<true, true><<<blocks, kTile, 0, stream>>>(
                     tab, r_begin, r_end, ws.codes, recv_out, ws.recv_t, ws.t_stride);
         } else if (recv_out != nullptr) {
             if (warp_rounds)
-                launch_dependent(true, recv_codes_quad_kernel<true, false>, qblocks, kQuadThreads, stream, tab, rc,
-                                 r_begin, r_end, ws.codes, recv_out, nullptr, 0);
+                launch_recv_quad<true, false>(tab, rc, r_begin, r_end, ws.codes, recv_out, nullptr, 0, stream);
             else
                 recv_codes_kernel<true, false><<<blocks, kTile, 0, stream>>>(
                     tab, r_begin, r_end, ws.codes, recv_out, nullptr, 0);
         } else {
             if (warp_rounds)
-                launch_dependent(true, recv_codes_quad_kernel<false, true>, qblocks, kQuadThreads, stream, tab, rc,
-                                 r_begin, r_end, ws.codes, nullptr, ws.recv_t, ws.t_stride);
+                launch_recv_quad<false, true>(tab, rc, r_begin, r_end, ws.codes, nullptr, ws.recv_t, ws.t_stride, stream);
             else
                 recv_codes_kernel<false, true><<<blocks, kTile, 0, stream>>>(
                     tab, r_begin, r_end, ws.codes, nullptr, ws.recv_t, ws.t_stride);
@@ -1343,14 +1388,11 @@ bcs_status bcs_prepare_rows(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_t
     const uint64_t count = r_end - r_begin;
     if (p >= 64) {
         const QuadConsts qc = make_quad_consts(tab, r_begin, r_end);
-        const unsigned grid = (unsigned)((count + kQuadTile - 1) / kQuadTile) + (unsigned)qc.n_special;
         // (dependent launch: harmless when the kernel before it on the stream is not the codes kernel)
         if (recv_out != nullptr)
-            launch_dependent(true, recv_codes_quad_kernel<true, true>, grid, kQuadThreads, stream, tab, qc, r_begin,
-                             r_end, codes, recv_out, recv_t, t_stride);
+            launch_recv_quad<true, true>(tab, qc, r_begin, r_end, codes, recv_out, recv_t, t_stride, stream);
         else
-            launch_dependent(true, recv_codes_quad_kernel<false, true>, grid, kQuadThreads, stream, tab, qc, r_begin,
-                             r_end, codes, nullptr, recv_t, t_stride);
+            launch_recv_quad<false, true>(tab, qc, r_begin, r_end, codes, nullptr, recv_t, t_stride, stream);
     } else {
         const unsigned blocks = (unsigned)((count + kTile - 1) / kTile);
         if (recv_out != nullptr)
