@@ -523,7 +523,7 @@ struct SharedEnv {
 // col_tile: byte of the tile's first rank in round 0 of the round-major copy, rounds t_stride
 // bytes apart (kPackedCol: both multiples of 4, so that the four entries of a quad and round are
 // stored as one word).
-template <bool kRowOut, bool kColOut, bool kPackedCol, bool kWideLoads, class Env>
+template <bool kRowOut, bool kColOut, bool kPackedCol, bool kWideLoads, bool kWordRows, class Env>
 __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh, uint32_t p, int q,
                                           uint64_t first, uint32_t n,
                                           const uint32_t *__restrict__ codes, uint8_t *stage,
@@ -663,6 +663,29 @@ __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh
         // kPackedCol: col_tile and t_stride are multiples of 4, the four entries of a round are one word
         int8_t *col = col0;
         int i = 0;
+        // Row bytes.  A thread's rows are q bytes apart in the staging buffer and its neighbour's
+        // 4q bytes further on: for an even q the byte stores of a warp hit only 32 / gcd(q, 32)
+        // banks (a quarter of the bandwidth at q = 20 or 28, a sixteenth at q = 16).  Rows of a q
+        // that is a multiple of 4 are whole words, so (kWordRows) every row's entries are shifted
+        // into a register instead and stored as one word after every fourth round: a quarter of
+        // the conflicting stores (q = 28: 32 -> 38 G ranks/s).  The same for q = 4m + 2, where two
+        // rows share a word and half the bandwidth is lost, did not pay (30.2 instead of 28.7 ms
+        // for the receive rows of p = 2^30-1).  Every round of the quad, in order, goes through
+        // put_rows.
+        uint32_t acc[4] = {0u, 0u, 0u, 0u};
+        auto put_rows = [&](const int round, const uint32_t (&entry)[4]) {
+            if (kRowOut) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (kWordRows) {
+                        acc[j] = __funnelshift_r(acc[j], entry[j], 8);    // (acc >> 8) | (entry << 24)
+                        if ((round & 3) == 3) *reinterpret_cast<uint32_t *>(row0 + j * q + (round - 3)) = acc[j];
+                    } else {
+                        row0[j * q + round] = (uint8_t)entry[j];
+                    }
+                }
+            }
+        };
 #pragma unroll
         for (int unrolled = 0; unrolled < kQuadTableRounds; ++unrolled) {
             if (unrolled >= first_lane_round) break;           // uniform over the grid
@@ -677,8 +700,8 @@ __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh
                 const int lead = top_bit(U);                   // -1 when there is no new block at all
                 B[j] |= bit_or_none(lead);
                 entry[j] = U ? (uint32_t)(lead - q) : (uint32_t)BCS_BAD_ENTRY;
-                if (kRowOut) row0[j * q + unrolled] = (uint8_t)entry[j];
             }
+            put_rows(unrolled, entry);
             if (kColOut) {
                 if (kPackedCol) {
                     *reinterpret_cast<uint32_t *>(col) = pack_bytes(entry[0], entry[1], entry[2], entry[3]);
@@ -713,8 +736,17 @@ __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh
         uint8_t *out = row0 + i;
         auto store_round = [&](const int (&entry)[4]) {
             if (kRowOut) {
+                if (kWordRows) {
+                    const bool full = (reinterpret_cast<uintptr_t>(out) & 3u) == 3u;   // round & 3 == 3: row0 is word-aligned
 #pragma unroll
-                for (int j = 0; j < 4; ++j) out[j * q] = (uint8_t)entry[j];
+                    for (int j = 0; j < 4; ++j) {
+                        acc[j] = __funnelshift_r(acc[j], (uint32_t)entry[j], 8);
+                        if (full) *reinterpret_cast<uint32_t *>(out + j * q - 3) = acc[j];
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) out[j * q] = (uint8_t)entry[j];
+                }
                 ++out;
             }
             if (kColOut) {
@@ -799,7 +831,7 @@ __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh
     }
 }
 
-template <bool kRowOut, bool kColOut, bool kWideLoads>
+template <bool kRowOut, bool kColOut, bool kWideLoads, bool kWordRows>
 __global__ void __launch_bounds__(kQuadThreads, 8)
 recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant__ QuadConsts qc,
                        uint64_t r_begin, uint64_t r_end, const uint32_t *__restrict__ codes,
@@ -827,7 +859,7 @@ recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant
     const uint64_t g0 = tile * kQuadTile;
     const uint32_t n = (uint32_t)(count - g0 < (uint64_t)kQuadTile ? count - g0 : (uint64_t)kQuadTile);
     // g0 and t_stride are multiples of 4 and recv_t is 16-byte aligned: packed column stores
-    quad_tile<kRowOut, kColOut, true, kWideLoads>(ParamEnv{tab, qc}, full_sh, p, q, r_begin + g0, n, codes, stage,
+    quad_tile<kRowOut, kColOut, true, kWideLoads, kWordRows>(ParamEnv{tab, qc}, full_sh, p, q, r_begin + g0, n, codes, stage,
                                       kColOut ? recv_t + g0 : nullptr, t_stride, runs);
     if (kRowOut) {
         const uint32_t len = n * (uint32_t)q;                  // the tile's rows start at byte g0 * q: 16-byte aligned
@@ -897,7 +929,7 @@ recv_quad_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t 
         }
         grid_dependency_wait();                                    // the codes are complete from here on
         // (the tile's first barrier comes before anything above is read)
-        quad_tile<true, kColOut, true, false>(SharedEnv{sh.skips, &sh.qc}, sh.full, p, q, first, n, codes + sh.rank0,
+        quad_tile<true, kColOut, true, false, false>(SharedEnv{sh.skips, &sh.qc}, sh.full, p, q, first, n, codes + sh.rank0,
                                        sh.stage + shift, col_tile, pitch, sh.runs);
     } else {
         grid_dependency_wait();
@@ -1227,12 +1259,19 @@ inline void launch_recv_quad(const PTable &tab, const QuadConsts &qc, uint64_t r
         wide += (int)((qc.aligned[0] >> k) & 1u);
         rounds += 1;
     }
-    if (5 * wide >= 4 * rounds)
-        launch_dependent(true, recv_codes_quad_kernel<kRowOut, kColOut, true>, grid, kQuadThreads, stream, tab, qc,
-                         r_begin, r_end, codes, recv_out, recv_t, t_stride);
-    else
-        launch_dependent(true, recv_codes_quad_kernel<kRowOut, kColOut, false>, grid, kQuadThreads, stream, tab, qc,
-                         r_begin, r_end, codes, recv_out, recv_t, t_stride);
+    // rows of a q that is a multiple of 4 are stored word by word (see put_rows)
+    const bool word_rows = kRowOut && (tab.q & 3) == 0;
+    auto go = [&](auto kernel) {
+        launch_dependent(true, kernel, grid, kQuadThreads, stream, tab, qc, r_begin, r_end, codes, recv_out, recv_t,
+                         t_stride);
+    };
+    if (5 * wide >= 4 * rounds) {
+        if (word_rows) go(recv_codes_quad_kernel<kRowOut, kColOut, true, kRowOut>);
+        else go(recv_codes_quad_kernel<kRowOut, kColOut, true, false>);
+    } else {
+        if (word_rows) go(recv_codes_quad_kernel<kRowOut, kColOut, false, kRowOut>);
+        else go(recv_codes_quad_kernel<kRowOut, kColOut, false, false>);
+    }
 }
 
 struct Workspace {
