@@ -115,6 +115,35 @@ __device__ __forceinline__ void flush_span(const uint8_t *stage, uint32_t shift,
     }
 }
 
+// The same for a staging buffer whose span starts `lag` = 1..3 bytes EARLIER in its 16-byte group
+// than the span does in global memory: stage[shift - lag, shift - lag + len) goes to
+// out[byte0, byte0 + len) with (byte0 & 15) == shift, shift >= lag.  (Rows that must start on a word
+// in shared memory while the table starts at any byte of the output.)  Every 16-byte vector of the
+// output is put together from five aligned words of the staging buffer, funnel-shifted by `lag`
+// bytes; the ragged ends go out as bytes.  The four bytes before `stage` must be readable.
+__device__ __forceinline__ void flush_span_lagging(const uint8_t *stage, uint32_t shift, uint32_t lag, uint32_t len,
+                                                   int8_t *out, uint64_t byte0)
+{
+    uint8_t *dst = reinterpret_cast<uint8_t *>(out) + (byte0 - shift);
+    const uint32_t end = shift + len;
+    const uint32_t nvec = (end + 15u) >> 4;
+    const uint32_t bits = 8u * (4u - lag);
+    for (uint32_t v = threadIdx.x; v < nvec; v += blockDim.x) {
+        const uint32_t lo = v << 4, hi = lo + 16u;
+        if (lo >= shift && hi <= end) {
+            // output bytes lo .. lo+15 are staging bytes lo-lag .. lo+15-lag: words at lo-4, lo, ..., lo+12
+            const uint32_t *w = reinterpret_cast<const uint32_t *>(stage + lo) - 1;
+            const uint32_t w0 = w[0], w1 = w[1], w2 = w[2], w3 = w[3], w4 = w[4];
+            *reinterpret_cast<uint4 *>(dst + lo) =
+                make_uint4(__funnelshift_r(w0, w1, bits), __funnelshift_r(w1, w2, bits),
+                           __funnelshift_r(w2, w3, bits), __funnelshift_r(w3, w4, bits));
+        } else {
+            const uint32_t from = lo < shift ? shift : lo, to = hi > end ? end : hi;
+            for (uint32_t e = from; e < to; ++e) dst[e] = stage[e - lag];
+        }
+    }
+}
+
 // The same for a span that starts 16-byte aligned in shared and global memory and is a multiple
 // of 16 bytes long, as one bulk copy of the TMA unit (cp.async.bulk, shared -> global) issued by
 // one thread.  Call with all threads of the CTA, after the rows have been written and INSTEAD of

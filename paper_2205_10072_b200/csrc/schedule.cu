@@ -883,6 +883,7 @@ struct QuadBatchShared {
     QuadConsts qc;
     uint32_t j, p;                          // index of the tile's p in the list; the p itself
     uint64_t tile0, rank0, entry0, copy0;   // of that p: first tile, flattened rank 0, first byte, copy
+    __align__(16) uint8_t stage_pad[16];    // (readable bytes before the staging buffer)
     __align__(16) uint8_t stage[kQuadTile * BCS_MAX_Q + 16];
     uint32_t runs[kRunLevels][kQuadLevelWords];
 };
@@ -917,6 +918,7 @@ recv_quad_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t 
     const uint64_t pitch = align_up(p, 16);
     const uint32_t *skips = ba.skips_tab + (size_t)j * kRow;       // the constants of this p
     int8_t *col_tile = kColOut ? recv_t + sh.copy0 + first : nullptr;
+    uint32_t lag = 0;                                              // see below
     if (p >= 64u) {                                                // uniform over the CTA
         if (t < kRow) {
             sh.skips[t] = skips[t];
@@ -929,8 +931,17 @@ recv_quad_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t 
         }
         grid_dependency_wait();                                    // the codes are complete from here on
         // (the tile's first barrier comes before anything above is read)
-        quad_tile<true, kColOut, true, false, false>(SharedEnv{sh.skips, &sh.qc}, sh.full, p, q, first, n, codes + sh.rank0,
-                                       sh.stage + shift, col_tile, pitch, sh.runs);
+        if ((q & 3) == 0) {
+            // rows of whole words are stored word by word (see put_rows): they must start on a
+            // word in shared memory, `lag` bytes before their place in the output's 16-byte group
+            lag = shift & 3u;
+            quad_tile<true, kColOut, true, false, true>(SharedEnv{sh.skips, &sh.qc}, sh.full, p, q, first, n,
+                                                        codes + sh.rank0, sh.stage + (shift - lag), col_tile, pitch,
+                                                        sh.runs);
+        } else {
+            quad_tile<true, kColOut, true, false, false>(SharedEnv{sh.skips, &sh.qc}, sh.full, p, q, first, n,
+                                                         codes + sh.rank0, sh.stage + shift, col_tile, pitch, sh.runs);
+        }
     } else {
         grid_dependency_wait();
         if (t < n)
@@ -938,7 +949,10 @@ recv_quad_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t 
                                              sh.stage + shift + t * (uint32_t)q, kColOut ? col_tile + t : nullptr, pitch);
     }
     __syncthreads();
-    flush_span(sh.stage, shift, n * (uint32_t)q, recv_out, span_begin);
+    if (lag != 0)
+        flush_span_lagging(sh.stage, shift, lag, n * (uint32_t)q, recv_out, span_begin);
+    else
+        flush_span(sh.stage, shift, n * (uint32_t)q, recv_out, span_begin);
 }
 
 // Send rows of a sub-range of one p from the round-major receive copy of that range;
