@@ -1,6 +1,6 @@
 // Receive and send schedules (arXiv 2205.10072, Algorithms 2-5 and the lookup of Algorithm 9):
 // kernels and the entry points bcs_build, bcs_build_static, bcs_build_to_host, bcs_prepare,
-// bcs_build_prepared, bcs_build_batch.
+// bcs_prepare_codes, bcs_prepare_rows, bcs_build_prepared, bcs_build_rooted, bcs_build_batch.
 //
 // Two constructions, bit-identical in their results:
 //
@@ -16,8 +16,8 @@
 //    send_transpose_kernel / send_batch_kernel produce
 //    sendsched[r][k] = recvsched[(r+skips[k]) mod p][k] as a transposition with row k rotated by
 //    skips[k] (send_rm_kernel: sub-ranges, byte gathers and recomputation for to-processors
-//    outside the range).  The three kernels of a single-p build are launched as dependents of one
-//    another (bcs_common.cuh), so each is brought onto the SMs while the one before it drains.
+//    outside the range).  The kernels of a build are launched as dependents of one another
+//    (bcs_common.cuh), so each is brought onto the SMs while the one before it drains.
 //
 //  * self-contained path (no workspace).  One thread per rank runs Algorithm 4 with the range
 //    search done by descending the homeranges; the send schedule is looked up in the rank-major
@@ -831,6 +831,8 @@ __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh
     }
 }
 
+// The quad tile for a range of one p >= 64.  kRowOut: rank-major rows; kColOut: round-major copy;
+// kWideLoads, kWordRows: see load4 and put_rows in quad_tile (picked per launch by launch_recv_quad).
 template <bool kRowOut, bool kColOut, bool kWideLoads, bool kWordRows>
 __global__ void __launch_bounds__(kQuadThreads, 8)
 recv_codes_quad_kernel(const __grid_constant__ PTable tab, const __grid_constant__ QuadConsts qc,
