@@ -196,6 +196,30 @@ def test_seeded_p_sweep_full_tables_sub_ranges_and_one_batch(bcs):
         assert np.array_equal(got_s[eo[j]:eo[j + 1]].reshape(p, -1), want_s), p
 
 
+def test_receive_kernel_instantiations(bcs):
+    """The quad receive kernel has four instantiations picked per launch: window bounds loaded as
+    16-byte words where a p's skips are multiples of 4 (p just below a power of two), rows stored
+    word by word where q is a multiple of 4.  Values of p that take each combination, all ranks
+    and a sub-range that starts off a multiple of 4, with and without rows / round-major copy."""
+    for p in (4095, 4097, 65535, 65537, 1048575, 1000003, 262143, 300007, 16383, 16385):
+        q = oracle.q_of(p)
+        want_r, want_s = oracle.full_table(p)
+        recv, send = _build(bcs, p, 0, p)
+        assert np.array_equal(recv, want_r) and np.array_equal(send, want_s), p
+        (recv,) = _build(bcs, p, 0, p, want_send=False)[:1]
+        assert np.array_equal(recv, want_r), p
+        r0, r1 = 1001, p - 77                                   # rows of the range only, start not on a quad
+        recv, send = _build(bcs, p, r0, r1)
+        assert np.array_equal(recv, want_r[r0:r1]) and np.array_equal(send, want_s[r0:r1]), p
+        raw_w, ws = _guarded(bcs.bcs_prepare_workspace_bytes(p))
+        bcs.bcs_prepare(p, ws)                                  # round-major copy only
+        raw_s, out = _guarded(p * q)
+        bcs.bcs_build_prepared(p, 0, p, None, out, ws)
+        torch.cuda.synchronize()
+        assert _guards_intact(raw_w, ws.numel()) and _guards_intact(raw_s, p * q)
+        assert np.array_equal(out.cpu().numpy().reshape(p, q), want_s), p
+
+
 def test_prepare_then_build_ranges(bcs):
     """bcs_prepare once, then receive and send rows of arbitrary ranges by bcs_build_prepared."""
     for p in (2, 3, 33, 63, 64, 1000, 4097, 100003):
