@@ -83,36 +83,116 @@ send_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, BatchArgs ba,
 }
 
 // ================================================================ workspace path
-// Skip code of every rank of one p: codes[x].  The scan over the levels is unrolled for the q at
-// hand (one instantiation per q), so every skip is an immediate operand from the kernel
-// parameters and no level is tested in vain.
-template <int kQ>
-__global__ void __launch_bounds__(kTile)
-codes_single_kernel(const __grid_constant__ PTable tab, uint32_t *__restrict__ codes)
+// Skip codes of many consecutive ranks at the price of one scan.  The greedy scan of rank g+e
+// (0 < e < 32) decides like that of g at every level until the one where the remainder R of g
+// has R < skips[k] <= R + e: there g+e takes skips[k] and keeps R + e - skips[k] < 31, while g
+// does not.  From such a level on g takes every level of the scanned range (its remainder stays
+// within a few dozen below the next skip), so one such level per 32 ranks is the rule; a second
+// one is only recorded as a flag and sends the 32 ranks to the plain scan.  The levels below
+// kCodesLow come from a table in shared memory, low[v] = code of v < skips[kCodesLow] over those
+// levels, which also holds the codes of the remainders below 31.
+constexpr int kCodesThreads = 256;
+constexpr int kCodesSub = 32;                                   // consecutive ranks scanned as one
+constexpr int kCodesCta = kCodesThreads * kCodesSub;            // ranks per CTA
+constexpr int kCodesLow = 8;
+
+struct BlockScan {
+    uint32_t biased;   // remainder of the block's first rank, plus 31
+    uint32_t code;     // its code so far
+    uint32_t stay;     // ranks g .. g+stay-1 decide like g; 32 while no level has split the block
+    uint32_t left;     // code, down to the splitting level, of the ranks that left there
+    uint32_t plain;    // a second splitting level was met
+};
+
+__device__ __forceinline__ void scan_level(BlockScan &b, uint32_t skip, int k)
 {
-    grid_launch_dependents();
-    // four consecutive ranks per thread: four independent scans, one 16-byte store
-    const uint32_t g = (blockIdx.x * kTile + threadIdx.x) * 4u;
-    if (g >= tab.p) return;
-    uint32_t x[4], code[4] = {0, 0, 0, 0};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) x[e] = g + e;            // ranks >= p give unused codes
-#pragma unroll
-    for (int k = kQ - 1; k >= 0; --k) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            if (x[e] >= tab.s[k]) {
-                x[e] -= tab.s[k];
-                code[e] |= 1u << k;
-            }
+    const uint32_t u = b.biased - skip;
+    if (u < (uint32_t)(kCodesSub - 1)) {              // skip - 31 <= remainder < skip: rare
+        if (b.stay == kCodesSub) {
+            b.stay = (kCodesSub - 1) - u;             // = skip - remainder
+            b.left = b.code | (1u << k);
+        } else {
+            b.plain = 1;
         }
     }
-    if (g + 4u <= tab.p) {
-        *reinterpret_cast<uint4 *>(codes + g) = make_uint4(code[0], code[1], code[2], code[3]);
+    if ((int32_t)u >= kCodesSub - 1) {
+        b.biased = u;
+        b.code |= 1u << k;
+    }
+}
+
+__device__ __forceinline__ uint4 pack_scan(const BlockScan &b)
+{
+    return make_uint4(b.biased - (kCodesSub - 1), b.code, b.stay | (b.plain << 8), b.left);
+}
+
+// Codes of the four ranks at offset e0 .. e0+3 of a block whose scan is sb (no second split).
+__device__ __forceinline__ uint4 quad_codes(const uint4 sb, const uint16_t *low, uint32_t e0)
+{
+    const uint32_t stay = sb.z;
+    uint32_t out[4];
+    if (stay >= e0 + 4u || stay <= e0) {              // the four on one side of the split
+        const bool with_g = stay > e0;
+        const uint16_t *at = low + (with_g ? sb.x + e0 : e0 - stay);
+        const uint32_t high = with_g ? sb.y : sb.w;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) out[e] = high | at[e];
     } else {
 #pragma unroll
-        for (int e = 0; e < 4; ++e)
-            if (g + e < tab.p) codes[g + e] = code[e];
+        for (uint32_t e = 0; e < 4; ++e) {
+            const bool with_g = e0 + e < stay;
+            out[e] = (with_g ? sb.y : sb.w) | low[(with_g ? sb.x + e0 : e0 - stay) + e];
+        }
+    }
+    return make_uint4(out[0], out[1], out[2], out[3]);
+}
+
+// Skip code of every rank of one p: codes[x].  A warp takes 1024 consecutive ranks: lane l
+// scans the levels above the table for the 32 ranks from first + 32 l (unrolled for the q at
+// hand, every skip an immediate operand from the kernel parameters), then the warp writes its
+// 256 quads, lane l the quads l, l+32, ..., one 16-byte store each.
+template <int kQ>
+__global__ void __launch_bounds__(kCodesThreads)
+codes_single_kernel(const __grid_constant__ PTable tab, uint32_t *__restrict__ codes)
+{
+    constexpr int kLow = kQ < kCodesLow ? kQ : kCodesLow;
+    __shared__ uint16_t low[1 << kLow];
+    __shared__ uint4 sub[kCodesThreads];
+    grid_launch_dependents();
+    if (threadIdx.x < (1u << kLow)) {
+        uint32_t v = threadIdx.x, c = 0;
+#pragma unroll
+        for (int k = kLow - 1; k >= 0; --k) {
+            if (v >= tab.s[k]) {
+                v -= tab.s[k];
+                c |= 1u << k;
+            }
+        }
+        low[threadIdx.x] = (uint16_t)c;
+    }
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t first = (blockIdx.x * kCodesThreads + (threadIdx.x & ~31u)) * (uint32_t)kCodesSub;
+    {
+        const uint32_t g = first + kCodesSub * lane;
+        BlockScan b = {g + (kCodesSub - 1), 0, kCodesSub, 0, 0};
+        if (g < tab.p) {
+#pragma unroll
+            for (int k = kQ - 1; k >= kLow; --k) scan_level(b, tab.s[k], k);
+        }
+        sub[threadIdx.x] = pack_scan(b);
+    }
+    __syncthreads();
+    const uint32_t e0 = 4u * (lane & 7u);
+#pragma unroll 2
+    for (uint32_t i = 0; i < 8; ++i) {
+        const uint32_t g = first + 4u * (i * 32u + lane);
+        if (g >= tab.p) break;
+        const uint4 sb = sub[(threadIdx.x & ~31u) + i * 4u + (lane >> 3)];
+        if (sb.z < 256u && g + 4u <= tab.p) {
+            *reinterpret_cast<uint4 *>(codes + g) = quad_codes(sb, low, e0);
+        } else {
+            for (uint32_t e = 0; e < 4 && g + e < tab.p; ++e) codes[g + e] = skip_code(tab.s, kQ, g + e);
+        }
     }
 }
 
@@ -121,7 +201,7 @@ struct CodesLauncher {
     static void launch(int q, const PTable &tab, uint32_t *codes, unsigned blocks, cudaStream_t stream)
     {
         if (q == kQ)
-            codes_single_kernel<kQ><<<blocks, kTile, 0, stream>>>(tab, codes);
+            codes_single_kernel<kQ><<<blocks, kCodesThreads, 0, stream>>>(tab, codes);
         else
             CodesLauncher<kQ - 1>::launch(q, tab, codes, blocks, stream);
     }
@@ -133,21 +213,100 @@ struct CodesLauncher<0> {
 
 inline void launch_codes(const PTable &tab, uint32_t *codes, cudaStream_t stream)
 {
-    CodesLauncher<BCS_MAX_Q>::launch(tab.q, tab, codes, (unsigned)((tab.p + 4 * kTile - 1) / (4 * kTile)),
-                                     stream);
+    CodesLauncher<BCS_MAX_Q>::launch(tab.q, tab, codes, (unsigned)((tab.p + kCodesCta - 1) / kCodesCta), stream);
 }
 
-// Batch: codes[g] for the flattened rank g, 1024 flattened ranks per CTA.  A CTA inside one p
-// (nearly all when the p are large) scans four consecutive ranks per thread, one shared-memory
-// load of the skip per level for the four, and stores their codes as one 16-byte vector; a CTA
-// that straddles several p finds the p of every rank.
+// Batch: codes[g] for the flattened rank g, 8192 flattened ranks per CTA, scanned in blocks of
+// 32 as above.  The CTA keeps the skips and the table of the first and of the last p it touches;
+// a block of 32 that lies inside one of the two is scanned once, every other block (one that
+// crosses from one p to the next, or lies in a p between the two) rank by rank.
+__global__ void __launch_bounds__(kCodesThreads)
+codes_batch_kernel(BatchArgs ba, uint32_t *__restrict__ codes)
+{
+    __shared__ uint32_t skips_sh[2][kRow];
+    __shared__ uint16_t low[2][1 << kCodesLow];
+    __shared__ uint4 sub[kCodesThreads];
+    __shared__ uint32_t seg[2];
+    __shared__ int q_sh[2];
+    __shared__ uint64_t edge[3];                 // rank 0 of the first p, its end, rank 0 of the last p
+    grid_launch_dependents();
+    const uint64_t g0 = (uint64_t)blockIdx.x * kCodesCta;
+    const uint64_t g1 = g0 + kCodesCta < ba.total_ranks ? g0 + kCodesCta : ba.total_ranks;
+    if (threadIdx.x < 32) {
+        const uint32_t jf = find_segment_warp(ba.rank_off, ba.num_p, g0);
+        const uint32_t jl = ba.rank_off[jf + 1] >= g1 ? jf : find_segment_warp(ba.rank_off, ba.num_p, g1 - 1);
+        skips_sh[0][threadIdx.x] = ba.skips_tab[(size_t)jf * kRow + threadIdx.x];
+        skips_sh[1][threadIdx.x] = ba.skips_tab[(size_t)jl * kRow + threadIdx.x];
+        if (threadIdx.x == 0) {
+            seg[0] = jf;
+            seg[1] = jl;
+            q_sh[0] = ceil_log2_fast(ba.p_list[jf]);
+            q_sh[1] = ceil_log2_fast(ba.p_list[jl]);
+            edge[0] = ba.rank_off[jf];
+            edge[1] = ba.rank_off[jf + 1];
+            edge[2] = ba.rank_off[jl];
+        }
+    }
+    __syncthreads();
+    const uint32_t jf = seg[0], jl = seg[1];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        const int levels = q_sh[t] < kCodesLow ? q_sh[t] : kCodesLow;
+        if (threadIdx.x < (1u << levels)) {
+            low[t][threadIdx.x] = (uint16_t)skip_code(skips_sh[t], levels, threadIdx.x);
+        }
+    }
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint64_t first = g0 + (uint64_t)(threadIdx.x & ~31u) * kCodesSub;
+    {
+        const uint64_t g = first + kCodesSub * lane;
+        // which of the two p the block lies in: the last one from its rank 0 on (all ranks up to
+        // g1 are its), the first one if the block ends inside it; 2 = neither
+        const uint32_t which = g >= edge[2] ? 1u : (g + kCodesSub <= edge[1] ? 0u : 2u);
+        BlockScan b = {0, 0, kCodesSub, 0, which >> 1};
+        if (g < g1 && which < 2u) {
+            b.biased = (uint32_t)(g - edge[2 * which]) + (kCodesSub - 1);
+            const int q = q_sh[which];
+            for (int k = q - 1; k >= kCodesLow; --k) scan_level(b, skips_sh[which][k], k);
+        }
+        uint4 packed = pack_scan(b);
+        packed.z |= which << 9;
+        sub[threadIdx.x] = packed;
+    }
+    __syncthreads();
+    const uint32_t e0 = 4u * (lane & 7u);
+#pragma unroll 2
+    for (uint32_t i = 0; i < 8; ++i) {
+        const uint64_t g = first + 4u * (i * 32u + lane);
+        if (g >= g1) break;
+        uint4 sb = sub[(threadIdx.x & ~31u) + i * 4u + (lane >> 3)];
+        if ((sb.z & 256u) == 0 && g + 4 <= g1) {
+            const uint16_t *table = low[sb.z >> 9];
+            sb.z &= 255u;
+            *reinterpret_cast<uint4 *>(codes + g) = quad_codes(sb, table, e0);
+        } else {
+            for (uint32_t e = 0; e < 4 && g + e < g1; ++e) {
+                const uint32_t j = find_segment(ba.rank_off, jf, jl, g + e);
+                codes[g + e] = skip_code(ba.skips_tab + (size_t)j * kRow, ceil_log2_fast(ba.p_list[j]),
+                                         (uint32_t)(g + e - ba.rank_off[j]));
+            }
+        }
+    }
+}
+
+// Batch of small p (a few thousand ranks each or fewer, where most blocks of 32 would cross from
+// one p to the next): codes[g] for the flattened rank g, 1024 flattened ranks per CTA.  A CTA
+// inside one p scans four consecutive ranks per thread, one shared-memory load of the skip per
+// level for the four, and stores their codes as one 16-byte vector; a CTA that straddles several
+// p finds the p of every rank.
 constexpr int kCodesTile = 4 * kTile;
 __global__ void __launch_bounds__(kTile)
-codes_batch_kernel(BatchArgs ba, uint32_t *__restrict__ codes)
+codes_batch_flat_kernel(BatchArgs ba, uint32_t *__restrict__ codes)
 {
     __shared__ uint32_t skips_sh[kRow];
     __shared__ uint32_t seg[3];                  // first and last p of the CTA, the first p itself
     __shared__ uint64_t rank0_sh;
+    grid_launch_dependents();
     const uint64_t g0 = (uint64_t)blockIdx.x * kCodesTile;
     const uint64_t g1 = g0 + kCodesTile < ba.total_ranks ? g0 + kCodesTile : ba.total_ranks;
     if (threadIdx.x < 32) {
@@ -1631,7 +1790,12 @@ bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_
         workspace_bytes >= bcs_build_batch_workspace_bytes(total_ranks, total_copy)) {
         uint32_t *codes = static_cast<uint32_t *>(workspace);
         int8_t *recv_t = static_cast<int8_t *>(workspace) + align_up(4ull * total_ranks, 256);
-        codes_batch_kernel<<<(unsigned)((total_ranks + kCodesTile - 1) / kCodesTile), kTile, 0, stream>>>(ba, codes);
+        // blocks of 32 ranks scanned as one where the p are large enough for most blocks to lie
+        // inside one of them
+        if (total_ranks / num_p >= (uint64_t)kCodesCta)
+            codes_batch_kernel<<<(unsigned)((total_ranks + kCodesCta - 1) / kCodesCta), kCodesThreads, 0, stream>>>(ba, codes);
+        else
+            codes_batch_flat_kernel<<<(unsigned)((total_ranks + kCodesTile - 1) / kCodesTile), kTile, 0, stream>>>(ba, codes);
         if ((st = launch_status()) != BCS_OK) return st;
         // the receive and the send kernel are launched as dependents of the kernel before them
         if (send_out != nullptr)
