@@ -26,7 +26,7 @@
 
 enum {
     SKM_RANKS = 0,          /* ranks whose receive row was built                                */
-    SKM_CODE_OPS,           /* skip code of the rank itself: compare, subtract, set bit per level */
+    SKM_CODE_OPS,           /* skip codes (one scan per block of 32 ranks); homerange, baseblock, B */
     SKM_TABLE_OPS,          /* rounds decided from the window's exact block set (short windows)  */
     SKM_HEAD_OPS,           /* rounds decided by the first head                                  */
     SKM_STEP2_OPS,          /* extra work when the first head was taken and the second step decides */
@@ -156,7 +156,8 @@ static void recv_row(const skm_ctx *c, uint32_t r, int last, int8_t *row, uint64
     uint32_t B = own ? 1u << bb : 0;
     if (cnt) {
         cnt[SKM_RANKS] += 1;
-        cnt[SKM_CODE_OPS] += Q4(3 * q + 3);   /* per level compare, subtract, or; then h, bb, B */
+        cnt[SKM_CODE_OPS] += Q4(3);           /* h, bb, B from the rank's code; the code itself is
+                                                 charged by the caller, per block of 32 ranks */
     }
     uint64_t dummy[SKM_NCOUNT];
     if (!cnt) { memset(dummy, 0, sizeof dummy); cnt = dummy; }
@@ -234,6 +235,104 @@ static void recv_row(const skm_ctx *c, uint32_t r, int last, int8_t *row, uint64
     }
 }
 
+/* ------------------------------------------------------------------ codes, 32 ranks per scan
+ * The codes of the 32 consecutive ranks g .. g+31 from one greedy scan.  Rank g+e decides like g
+ * at every level until the one where the remainder R of g has R < skips[k] <= R + e: there g+e
+ * takes skips[k] and keeps R + e - skips[k] < 31, and g does not take it.  The levels below LOW
+ * come from a table, low[v] = code of v over those levels (v < skips[LOW]), which also serves
+ * the small remainders of the ranks that left.  One such level per block is recorded; a second
+ * one sends the block to the plain scan (none has been seen for any p tried).
+ * Operations charged (whole operations, to ops[0]): per level of the scan 5 (subtract, the two
+ * tests, select, or), 3 more at a splitting level; per four ranks 3 for the side of the split and
+ * the table address, 4 table loads, 4 or, 1 vector store, and 8 more where the split falls
+ * inside the four; the table's 3 per level and entry once per 8192 ranks; a plain scan 3 per
+ * level and rank.  ops[1] = blocks, ops[2] = blocks with a splitting level, ops[3] = plain. */
+#define SKM_LOW 8
+#define SKM_BLOCK 32
+#define SKM_BLOCKS_FROM 8192   /* smaller p are charged the plain scan, 3 per level and rank (the
+                                  GPU scans them rank by rank: most blocks would cross p) */
+
+static void codes_block(const skm_ctx *c, const uint16_t *low, int low_levels, uint32_t g,
+                        uint32_t *out /* 32, or NULL */, uint64_t *ops)
+{
+    const uint32_t p = c->p;
+    uint32_t rem = g, code = 0, stay = SKM_BLOCK, left = 0;
+    int plain = 0;
+    for (int k = c->q - 1; k >= low_levels; --k) {
+        const uint32_t skip = c->s[k];
+        ops[0] += 5;
+        if (rem < skip && skip <= rem + (SKM_BLOCK - 1)) {
+            ops[0] += 3;
+            if (stay == SKM_BLOCK) { stay = skip - rem; left = code | (1u << k); }
+            else plain = 1;
+        }
+        if (rem >= skip) { rem -= skip; code |= 1u << k; }
+    }
+    ops[1] += 1;
+    if (stay != SKM_BLOCK) ops[2] += 1;
+    if (plain) ops[3] += 1;
+    for (uint32_t e0 = 0; e0 < SKM_BLOCK && g + e0 < p; e0 += 4) {
+        if (plain) ops[0] += 4ull * 3 * (uint64_t)c->q;
+        else ops[0] += 12 + ((stay > e0 && stay < e0 + 4) ? 8 : 0);
+        for (uint32_t e = e0; e < e0 + 4 && g + e < p; ++e) {
+            uint32_t v;
+            if (plain) {
+                uint32_t x = g + e;
+                v = 0;
+                for (int k = c->q - 1; k >= 0; --k)
+                    if (x >= c->s[k]) { x -= c->s[k]; v |= 1u << k; }
+            } else if (e < stay) {
+                v = code | low[rem + e];
+            } else {
+                v = left | low[e - stay];
+            }
+            if (out) out[e] = v;
+        }
+    }
+}
+
+static int build_low(const skm_ctx *c, uint16_t *low /* 1 << SKM_LOW */)
+{
+    const int levels = c->q < SKM_LOW ? c->q : SKM_LOW;
+    for (uint32_t v = 0; v < (1u << levels); ++v) {
+        uint32_t x = v, code = 0;
+        for (int k = levels - 1; k >= 0; --k)
+            if (x >= c->s[k]) { x -= c->s[k]; code |= 1u << k; }
+        low[v] = (uint16_t)code;
+    }
+    return levels;
+}
+
+/* Codes of the ranks g_begin .. g_end-1 (g_begin a multiple of 32); codes may be NULL (count
+ * only); ops[4] accumulated as described above. */
+int skm_codes_blocks(uint32_t p, uint64_t g_begin, uint64_t g_end, uint32_t *codes, uint64_t *ops)
+{
+    if (p == 0 || p > 0x7fffffffu || g_begin % SKM_BLOCK || g_begin > g_end || g_end > p || ops == NULL)
+        return -1;
+    skm_ctx c;
+    ctx_init(&c, p);
+    uint16_t low[1 << SKM_LOW];
+    const int levels = build_low(&c, low);
+    uint32_t tmp[SKM_BLOCK];
+    for (uint64_t g = g_begin; g < g_end; g += SKM_BLOCK) {
+        if ((g - g_begin) % 8192 == 0) ops[0] += (3ull * levels) << levels;
+        codes_block(&c, low, levels, (uint32_t)g, tmp, ops);
+        if (codes)
+            for (uint32_t e = 0; e < SKM_BLOCK && g + e < g_end; ++e) codes[g - g_begin + e] = tmp[e];
+    }
+    return 0;
+}
+
+/* The same codes by the plain scan, rank by rank (what skm_codes_blocks must reproduce). */
+int skm_codes_plain(uint32_t p, uint64_t g_begin, uint64_t g_end, uint32_t *codes)
+{
+    if (p == 0 || p > 0x7fffffffu || g_begin > g_end || g_end > p || codes == NULL) return -1;
+    skm_ctx c;
+    ctx_init(&c, p);
+    for (uint64_t g = g_begin; g < g_end; ++g) codes[g - g_begin] = code_of(&c, (uint32_t)g);
+    return 0;
+}
+
 /* ------------------------------------------------------------------------------------ API */
 int skm_q(uint32_t p)
 {
@@ -254,9 +353,13 @@ int skm_rows(uint32_t p, const uint64_t *ranks, uint64_t n, int8_t *recv, int8_t
     ctx_init(&c, p);
     const int q = c.q;
     int8_t tmp[SKM_MAX_Q + 1];
+    uint16_t low[1 << SKM_LOW];
+    const int levels = build_low(&c, low);
+    uint64_t block_ops[4] = {0, 0, 0, 0};
     for (uint64_t m = 0; m < n; ++m) {
         const uint32_t r = (uint32_t)ranks[m];
         if (r >= p) return -2;
+        if (p >= SKM_BLOCKS_FROM) codes_block(&c, low, levels, r & ~(uint32_t)(SKM_BLOCK - 1), NULL, block_ops);
         if (recv) recv_row(&c, r, q - 1, recv + m * (uint64_t)q, counters);
         else recv_row(&c, r, q - 1, tmp, counters);
         if (send) {
@@ -268,6 +371,11 @@ int skm_rows(uint32_t p, const uint64_t *ranks, uint64_t n, int8_t *recv, int8_t
             }
         }
     }
+    /* every listed rank pays 1/32 of its block's scan and of the table's share of 32 ranks */
+    if (counters && p >= SKM_BLOCKS_FROM)
+        counters[SKM_CODE_OPS] += Q4(block_ops[0]) / SKM_BLOCK + Q4(n * ((3ull * levels) << levels)) / 8192;
+    else if (counters)
+        counters[SKM_CODE_OPS] += Q4(n * 3ull * (uint64_t)q);
     return 0;
 }
 
@@ -280,7 +388,9 @@ int skm_full(uint32_t p, int8_t *recv, int8_t *send, uint64_t *counters)
     const int q = c.q;
     uint32_t *codes = (uint32_t *)malloc((size_t)p * sizeof(uint32_t));
     if (codes == NULL) return -3;
-    for (uint32_t x = 0; x < p; ++x) codes[x] = code_of(&c, x);
+    uint64_t block_ops[4] = {0, 0, 0, 0};
+    if (skm_codes_blocks(p, 0, p, codes, block_ops) != 0) { free(codes); return -4; }
+    if (counters) counters[SKM_CODE_OPS] += p >= SKM_BLOCKS_FROM ? Q4(block_ops[0]) : Q4(3ull * p * (uint64_t)q);
     c.codes = codes;
     for (uint32_t r = 0; r < p; ++r) recv_row(&c, r, q - 1, recv + (uint64_t)r * q, counters);
     free(codes);

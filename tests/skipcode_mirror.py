@@ -42,6 +42,8 @@ def _load():
         L.skm_q.argtypes = [c.c_uint32]
         L.skm_rows.argtypes = [c.c_uint32, c.c_void_p, c.c_uint64, c.c_void_p, c.c_void_p, c.c_void_p]
         L.skm_full.argtypes = [c.c_uint32, c.c_void_p, c.c_void_p, c.c_void_p]
+        L.skm_codes_blocks.argtypes = [c.c_uint32, c.c_uint64, c.c_uint64, c.c_void_p, c.c_void_p]
+        L.skm_codes_plain.argtypes = [c.c_uint32, c.c_uint64, c.c_uint64, c.c_void_p]
         L.skm_set_table_mode.argtypes = [c.c_int]
         L.skm_set_table_mode.restype = None
         assert L.skm_ncount() == len(COUNTERS)
@@ -87,6 +89,28 @@ def rows(p: int, ranks, want_send: bool = True):
     if rc:
         raise RuntimeError("skm_rows: %d" % rc)
     return recv, send, _counts(cnt)
+
+
+def codes_blocks(p: int, g_begin: int, g_end: int, want_codes: bool = True):
+    """(codes of the ranks g_begin..g_end-1 or None, {"ops", "blocks", "split", "plain"}) by one
+    scan per block of 32 ranks; g_begin a multiple of 32."""
+    L = _load()
+    codes = np.zeros(g_end - g_begin, dtype=np.uint32) if want_codes else None
+    ops = np.zeros(4, dtype=np.uint64)
+    rc = L.skm_codes_blocks(p, g_begin, g_end, codes.ctypes.data if want_codes else None, ops.ctypes.data)
+    if rc:
+        raise RuntimeError("skm_codes_blocks: %d" % rc)
+    return codes, dict(zip(("ops", "blocks", "split", "plain"), (int(v) for v in ops)))
+
+
+def codes_plain(p: int, g_begin: int, g_end: int):
+    """The same codes by the greedy scan of every rank."""
+    L = _load()
+    codes = np.zeros(g_end - g_begin, dtype=np.uint32)
+    rc = L.skm_codes_plain(p, g_begin, g_end, codes.ctypes.data)
+    if rc:
+        raise RuntimeError("skm_codes_plain: %d" % rc)
+    return codes
 
 
 def per_rank(counts: dict) -> dict:

@@ -77,3 +77,31 @@ def test_committed_model_table_is_what_the_mirror_counts():
     for entry in table.values():
         assert 50 < entry["recv_int_ops_per_rank"] < 1000
         json.dumps(entry)
+
+
+def test_block_codes_equal_the_plain_scan():
+    """One greedy scan per block of 32 consecutive ranks (plus the table of the low levels) gives
+    the code of every rank that its own scan gives; the second splitting level that would send
+    a block to the plain scan does not occur."""
+    import numpy as np
+    from tests import skipcode_mirror as skm
+    split = 0
+    for p in list(range(1, 400)) + [1000, 4097, 65535, 65537, 100003, 300007, 2**20 + 1]:
+        got, st = skm.codes_blocks(p, 0, p)
+        assert np.array_equal(got, skm.codes_plain(p, 0, p)), p
+        assert st["plain"] == 0, (p, st)
+        split += st["split"]
+    assert split > 1000                      # the splitting levels are exercised
+    rng = np.random.default_rng(11)
+    for p in (2**24 - 3, 2**29 + 12345, 2**30 - 1, 2**30 - 12345, 2**31 - 1):
+        starts = [0, (p - 5000) // 32 * 32] + [int(v) // 32 * 32 for v in rng.integers(0, p - 70000, 12)]
+        q = skm.skm_q(p)
+        v = p
+        for _ in range(q - 8):               # just below the larger skips, where blocks split
+            v = (v + 1) // 2
+            starts.append(max(0, v - 3000) // 32 * 32)
+        for g in starts:
+            end = min(p, g + 65536)
+            got, st = skm.codes_blocks(p, g, end)
+            assert np.array_equal(got, skm.codes_plain(p, g, end)), (p, g)
+            assert st["plain"] == 0, (p, g, st)
