@@ -86,9 +86,11 @@ send_kernel(PTable tab, uint64_t r_begin, uint64_t r_end, BatchArgs ba,
 // Skip codes of many consecutive ranks at the price of one scan.  The greedy scan of rank g+e
 // (0 < e < 32) decides like that of g at every level until the one where the remainder R of g
 // has R < skips[k] <= R + e: there g+e takes skips[k] and keeps R + e - skips[k] < 31, while g
-// does not.  From such a level on g takes every level of the scanned range (its remainder stays
-// within a few dozen below the next skip), so one such level per 32 ranks is the rule; a second
-// one is only recorded as a flag and sends the 32 ranks to the plain scan.  The levels below
+// does not.  From such a level on g takes every level of the scanned range: with R = skips[k] - d,
+// 1 <= d <= 31, and skips[k] = 2 skips[k-1] or 2 skips[k-1] - 1, the remainder before level j < k
+// is skips[j+1] - d' with d' <= d + (k - 1 - j) < 55 <= skips[j] (the scanned levels are 8 and up,
+// skips[8] > 128), which is at least skips[j].  So a block has at most one such level; a second
+// one is still recorded as a flag that sends the 32 ranks to the plain scan.  The levels below
 // kCodesLow come from a table in shared memory, low[v] = code of v < skips[kCodesLow] over those
 // levels, which also holds the codes of the remainders below 31.
 constexpr int kCodesThreads = 256;

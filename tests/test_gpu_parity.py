@@ -140,6 +140,34 @@ def test_batch_with_trivial_and_duplicate_p(bcs, fast):
     assert np.array_equal(recv[eo[3]:eo[4]].cpu().numpy().reshape(300, -1), oracle.full_table(300)[0])
 
 
+def test_batch_of_large_and_tiny_p_mixed(bcs):
+    """A list whose p average more than 8192 ranks (the batch takes the codes kernel that scans
+    blocks of 32 flattened ranks at once) with p = 1, tiny p and p next to multiples of 8192 in
+    between: blocks that cross from one p to the next, whole p inside one block, CTAs that touch
+    three and more p, a last block cut off by the end of the list."""
+    plist = [70001, 1, 2, 3, 65536, 1, 8191, 8193, 31, 32, 33, 16384, 5, 100003, 1, 7, 8192, 40961,
+             64, 63, 65, 262147, 1000, 24576, 9, 131071]
+    assert sum(plist) // len(plist) >= 8192
+    plan = bcs.bcs_batch_plan(plist)
+    dev = plan.to("cuda")
+    raw_r, recv = _guarded(plan.total_entries)
+    raw_s, send = _guarded(plan.total_entries)
+    raw_w, ws = _batch_ws(bcs, plan, True)
+    bcs.bcs_build_batch(dev, recv, send, ws)
+    torch.cuda.synchronize()
+    assert _guards_intact(raw_w, ws.numel())
+    assert _guards_intact(raw_r, plan.total_entries) and _guards_intact(raw_s, plan.total_entries)
+    assert bcs.bcs_wait_expired() == 0
+    eo = plan.entry_off.tolist()
+    for j, p in enumerate(plist):
+        if p == 1:
+            assert eo[j] == eo[j + 1]
+            continue
+        want_r, want_s = oracle.full_table(p)
+        assert np.array_equal(recv[eo[j]:eo[j + 1]].cpu().numpy().reshape(p, -1), want_r), (j, p)
+        assert np.array_equal(send[eo[j]:eo[j + 1]].cpu().numpy().reshape(p, -1), want_s), (j, p)
+
+
 # ---------------------------------------------------------------- ranges, tails, degenerate
 @pytest.mark.parametrize("fast", [True, False])
 def test_sub_ranges_ragged_tails_and_single_outputs(bcs, fast):
