@@ -177,10 +177,13 @@ bcs_status bcs_build_to_host(uint32_t p, uint64_t r_begin, uint64_t r_end,
 /* Host helper for bcs_build_batch: for a list of num_p values of p fills
  *   rank_off_host[num_p+1]  prefix sums of p_j            (flattened rank index),
  *   entry_off_host[num_p+1] prefix sums of p_j * q_j      (byte offset of p_j's table),
- *   tile_off_host[num_p+1]  prefix sums of ceil(p_j / 512) (the fast construction works in tiles
- *                           of 512 ranks that start anew with every p),
- *   copy_off_host[num_p+1]  prefix sums of q_j * align16(p_j) (where p_j's round-major scratch
- *                           copy starts in the workspace; align16 = round up to 16),
+ *   tile_off_host[num_p+1]  prefix sums of ceil(p_j / 512) over the p_j above 1024, 0 for the
+ *                           others (the fast construction works on a larger p in tiles of 512
+ *                           ranks that start anew with every p, and builds both tables of a
+ *                           p_j <= 1024 in one thread block that keeps everything on chip),
+ *   copy_off_host[num_p+1]  prefix sums of q_j * align16(p_j) over the p_j above 1024 (where
+ *                           p_j's round-major scratch copy starts in the workspace; align16 =
+ *                           round up to 16),
  *   skips_tab_host[num_p * BCS_SKIPS_STRIDE] row j = skips[0..q_j] of p_j (Algorithm 1),
  *                           the rest of the row 0,
  *   full_tab_host[num_p * BCS_SKIPS_STRIDE]  row j, word d = skip code of rank
@@ -199,8 +202,9 @@ bcs_status bcs_batch_plan(const uint32_t *p_list_host, uint32_t num_p,
  * byte entry_off[j] and is rank-major with q_j bytes per rank, unpadded.  send_out may be NULL;
  * recv_out is required.  workspace as for bcs_build, of
  * bcs_build_batch_workspace_bytes(total_ranks, total_copy) bytes for the fast construction
- * (which also needs tile_off_dev and copy_off_dev), or NULL: then tile_off_dev and copy_off_dev
- * may be NULL too and the self-contained construction runs. */
+ * (which also needs tile_off_dev and copy_off_dev; 256 bytes, never touched, when no p of the
+ * list is above 1024: the pointer then only selects the construction), or NULL: then
+ * tile_off_dev and copy_off_dev may be NULL too and the self-contained construction runs. */
 size_t bcs_build_batch_workspace_bytes(uint64_t total_ranks, uint64_t total_copy);
 bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_dev,
                            const uint64_t *entry_off_dev, const uint64_t *tile_off_dev,

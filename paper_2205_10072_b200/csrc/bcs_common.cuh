@@ -11,6 +11,8 @@ namespace bcs {
 
 constexpr int kTile = 256;                    // ranks (= threads) per CTA of the schedule kernels
 constexpr int kStageBytes = kTile * 32 + 16;  // kTile rows of <= 31 bytes + alignment shift
+constexpr uint32_t kFusedMaxP = 1024;         // batch: a p up to here is built by one CTA of the fused kernel
+constexpr int kFusedMaxQ = 10;                //        (q <= 10)
 constexpr int kCachedRows = 4;                // per-p table rows a batch CTA keeps in shared memory
 constexpr int kRow = BCS_SKIPS_STRIDE;        // words per table row
 

@@ -53,8 +53,10 @@ bcs_status bcs_batch_plan(const uint32_t *p_list_host, uint32_t num_p, uint64_t 
         }
         ranks += tab.p;
         entries += (uint64_t)tab.p * (uint64_t)tab.q;
-        tiles += (tab.p + 511u) / 512u;
-        copy += (uint64_t)tab.q * align_up(tab.p, 16);
+        if (tab.p > kFusedMaxP) {        // smaller p: one CTA of the fused kernel, no tiles, no scratch
+            tiles += (tab.p + 511u) / 512u;
+            copy += (uint64_t)tab.q * align_up(tab.p, 16);
+        }
     }
     rank_off_host[num_p] = ranks;
     entry_off_host[num_p] = entries;

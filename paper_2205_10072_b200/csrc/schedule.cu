@@ -23,6 +23,7 @@
 //    search done by descending the homeranges; the send schedule is looked up in the rank-major
 //    receive table where the to-processor is inside the call's range and recomputed
 //    (Algorithm 5) where it is not.
+#include <cstddef>
 #include <mutex>
 
 #include "bcs_common.cuh"
@@ -1118,6 +1119,141 @@ recv_quad_batch_kernel(BatchArgs ba, const uint32_t *__restrict__ codes, int8_t 
         flush_span(sh.stage, shift, n * (uint32_t)q, recv_out, span_begin);
 }
 
+// Batch, p <= kFusedMaxP: ONE CTA builds both tables of a p, everything in shared memory.
+// With all p ranks on chip the windows of Algorithm 4 are looked up as exact block sets, whatever
+// their length: run[l][x] holds the baseblock bits of the 2^l ranks that end at x (cyclically; the
+// root contributes no bit), built level by level from the ranks' own bits, and a window of L ranks
+// is the union of the two runs of 2^floor(log2 L) ranks at its ends.  So every round of every rank
+// is two (or, when the first window holds nothing new, four) 16-bit loads and a leading-bit
+// search, with no case for the root, the wrap or the homeranges; the send rows are the lookup
+// sendsched[r][k] = recvsched[(r+skips[k]) mod p][k] in the staged receive rows.  No workspace,
+// one launch for any number of such p (the plan gives them no tiles, so the tiled kernels never
+// see them); CTAs of larger p return at once.  The last p of the list come first: lists are
+// often ascending and the largest p take longest.
+constexpr int kFusedThreads = 256;
+struct FusedShared {
+    uint32_t skips[kRow];
+    uint32_t len2[kFusedMaxQ];                    // length of the second window of round i
+    uint8_t level1[kFusedMaxQ], level2[kFusedMaxQ];   // floor(log2) of the two window lengths
+    uint16_t codes[kFusedMaxP];
+    union alignas(16) {                           // (the staging buffers go out as 16-byte vectors)
+        uint16_t run[kFusedMaxQ][kFusedMaxP];     // levels 0 .. floor(log2(p-1)) <= 9
+        uint8_t send_stage[kFusedMaxP * kFusedMaxQ + 16];   // after the last round
+    };
+    __align__(16) uint8_t recv_stage[kFusedMaxP * kFusedMaxQ + 16];
+};
+static_assert(offsetof(FusedShared, send_stage) % 16 == 0 && offsetof(FusedShared, recv_stage) % 16 == 0,
+              "staging buffers start on a 16-byte boundary");
+
+template <bool kSend>
+__global__ void __launch_bounds__(kFusedThreads)
+fused_small_batch_kernel(BatchArgs ba, int8_t *recv_out, int8_t *send_out)
+{
+    __shared__ __align__(16) FusedShared sh;
+    grid_launch_dependents();
+    const uint32_t t = threadIdx.x;
+    const uint32_t j = ba.num_p - 1u - blockIdx.x;
+    const uint32_t p = ba.p_list[j];
+    const int q = ceil_log2_fast(p);
+    if (q == 0 || p > kFusedMaxP) {                                // uniform over the CTA
+        grid_dependency_wait();                                    // see the end of the kernel
+        return;
+    }
+    const uint32_t *skips = ba.skips_tab + (size_t)j * kRow;
+    if (t < kRow) sh.skips[t] = skips[t];
+    if (t < (uint32_t)q) {
+        const uint32_t first_len = skips[t + 1] - skips[t];        // >= 1
+        const uint32_t second_len = quad_len2(skips, (int)t);
+        sh.len2[t] = second_len;
+        sh.level1[t] = (uint8_t)(31 - __clz(first_len));
+        sh.level2[t] = (uint8_t)(second_len != 0 && second_len < p ? 31 - __clz(second_len) : 0);
+    }
+    for (uint32_t x = t; x < p; x += kFusedThreads) {
+        const uint32_t c = skip_code(skips, q, x);
+        sh.codes[x] = (uint16_t)c;
+        sh.run[0][x] = (uint16_t)(c & (0u - c));                   // baseblock as a bit, 0 for the root
+    }
+    __syncthreads();
+    const int top_level = 31 - __clz(p - 1u);                      // the longest window has p - 1 ranks
+    for (int l = 1; l <= top_level; ++l) {
+        const uint32_t half = 1u << (l - 1);
+        for (uint32_t x = t; x < p; x += kFusedThreads)
+            sh.run[l][x] = sh.run[l - 1][x] | sh.run[l - 1][x >= half ? x - half : x + p - half];
+        __syncthreads();
+    }
+    const uint64_t entry0 = ba.entry_off[j];
+    const uint32_t shift = (uint32_t)(entry0 & 15u);
+    const uint32_t all = (1u << q) - 1u;
+    // A thread has the ranks t, t + 256, ... (at most four); the rounds are the outer loop, so
+    // that what a round needs of its skips and window lengths is worked out once for the four.
+    constexpr int kMine = (int)(kFusedMaxP / kFusedThreads);
+    uint32_t B[kMine];
+    int h[kMine], bb[kMine];
+#pragma unroll
+    for (int m = 0; m < kMine; ++m) {
+        const uint32_t r = t + (uint32_t)m * kFusedThreads;
+        const uint32_t c = r < p ? sh.codes[r] : 0u;
+        h[m] = r < p ? 31 - __clz(c) : -2;                         // homerange; -1 for the root
+        bb[m] = __ffs(c) - 1;                                      // baseblock (Algorithm 2)
+        B[m] = c & (0u - c);
+    }
+    uint8_t *const rows = sh.recv_stage + shift + t * (uint32_t)q;
+    for (int i = 0; i < q; ++i) {
+        const uint32_t lo = sh.skips[i], hi = sh.skips[i + 1];
+        const uint32_t len1 = hi - lo, second_len = sh.len2[i];
+        const int l1 = sh.level1[i], l2 = sh.level2[i];
+        const uint32_t back1 = len1 - (1u << l1), back2 = second_len - (1u << l2);
+        const uint16_t *const run1 = sh.run[l1], *const run2 = sh.run[l2];
+        const uint32_t hi_back = hi == p ? 0u : hi;                // r - p is rank r
+#pragma unroll
+        for (int m = 0; m < kMine; ++m) {
+            const uint32_t r = t + (uint32_t)m * kFusedThreads;
+            if (r >= p) break;
+            int entry = bb[m];
+            if (i != h[m]) {
+                // the baseblock bits of the len1 ranks that end at rank e = r - lo
+                const uint32_t e = r >= lo ? r - lo : r + p - lo;
+                uint32_t U = ((uint32_t)run1[e] | (uint32_t)run1[e >= back1 ? e - back1 : e + p - back1]) & ~B[m];
+                if (U == 0) {
+                    if (second_len >= p) {
+                        U = all & ~B[m];
+                    } else if (second_len != 0) {
+                        const uint32_t e2 = r >= hi_back ? r - hi_back : r + p - hi_back;
+                        U = ((uint32_t)run2[e2] | (uint32_t)run2[e2 >= back2 ? e2 - back2 : e2 + p - back2]) & ~B[m];
+                    }
+                }
+                const int blk = top_bit(U);
+                B[m] |= bit_or_none(blk);
+                entry = U ? blk - q : BCS_BAD_ENTRY;
+            }
+            rows[(uint32_t)m * kFusedThreads * (uint32_t)q + (uint32_t)i] = (uint8_t)entry;
+        }
+    }
+    __syncthreads();                                               // the run table is done with
+    flush_span(sh.recv_stage, shift, p * (uint32_t)q, recv_out, entry0);
+    if (kSend) {
+        uint8_t *const out = sh.send_stage + shift + t * (uint32_t)q;
+        for (int k = 0; k < q; ++k) {
+            const uint32_t skip = sh.skips[k];
+#pragma unroll
+            for (int m = 0; m < kMine; ++m) {
+                const uint32_t r = t + (uint32_t)m * kFusedThreads;
+                if (r >= p) break;
+                uint32_t to = r + skip;
+                if (to >= p) to -= p;
+                out[(uint32_t)m * kFusedThreads * (uint32_t)q + (uint32_t)k] =
+                    sh.recv_stage[shift + to * (uint32_t)q + (uint32_t)k];
+            }
+        }
+        __syncthreads();
+        flush_span(sh.send_stage, shift, p * (uint32_t)q, send_out, entry0);
+    }
+    // Launched as a dependent of the tiled kernels (when the list has larger p too), this kernel
+    // needs nothing of theirs and starts beside their tail; but it must not END before them, or
+    // what follows it on the stream could start while they still write.
+    grid_dependency_wait();
+}
+
 // Send rows of a sub-range of one p from the round-major receive copy of that range;
 // to-processors outside the range are recomputed from the codes (Algorithm 5).
 __global__ void __launch_bounds__(kTile)
@@ -1761,7 +1897,9 @@ bcs_status bcs_build_to_host(uint32_t p, uint64_t r_begin, uint64_t r_end, int8_
 
 size_t bcs_build_batch_workspace_bytes(uint64_t total_ranks, uint64_t total_copy)
 {
-    if (total_ranks == 0 || total_copy == 0) return 0;
+    if (total_ranks == 0) return 0;
+    // no p above kFusedMaxP: the fused kernel needs no scratch, and a token workspace selects it
+    if (total_copy == 0) return 256;
     return (size_t)(align_up(4ull * total_ranks, 256) + total_copy);
 }
 
@@ -1788,31 +1926,43 @@ bcs_status bcs_build_batch(const uint32_t *p_list_dev, const uint64_t *rank_off_
     PTable none = {};
     const unsigned blocks = (unsigned)blocks64;
     bcs_status st;
-    if (workspace != nullptr && tile_off_dev != nullptr && copy_off_dev != nullptr && total_tiles != 0 &&
+    if (workspace != nullptr && tile_off_dev != nullptr && copy_off_dev != nullptr &&
         workspace_bytes >= bcs_build_batch_workspace_bytes(total_ranks, total_copy)) {
         uint32_t *codes = static_cast<uint32_t *>(workspace);
         int8_t *recv_t = static_cast<int8_t *>(workspace) + align_up(4ull * total_ranks, 256);
-        // blocks of 32 ranks scanned as one where the p are large enough for most blocks to lie
-        // inside one of them
-        if (total_ranks / num_p >= (uint64_t)kCodesCta)
-            codes_batch_kernel<<<(unsigned)((total_ranks + kCodesCta - 1) / kCodesCta), kCodesThreads, 0, stream>>>(ba, codes);
-        else
-            codes_batch_flat_kernel<<<(unsigned)((total_ranks + kCodesTile - 1) / kCodesTile), kTile, 0, stream>>>(ba, codes);
-        if ((st = launch_status()) != BCS_OK) return st;
-        // the receive and the send kernel are launched as dependents of the kernel before them
-        if (send_out != nullptr)
-            launch_dependent(true, recv_quad_batch_kernel<true>, (unsigned)total_tiles, kQuadThreads, stream, ba,
-                             (const uint32_t *)codes, recv_out, recv_t);
-        else
-            launch_dependent(true, recv_quad_batch_kernel<false>, (unsigned)total_tiles, kQuadThreads, stream, ba,
-                             (const uint32_t *)codes, recv_out, (int8_t *)nullptr);
-        if ((st = launch_status()) != BCS_OK) return st;
-        if (send_out != nullptr) {
-            launch_dependent(true, send_batch_kernel, (unsigned)(2 * total_tiles), kTrThreads, stream, ba,
-                             (const int8_t *)recv_t, send_out);
+        // the p above kFusedMaxP, tile by tile (the plan counts tiles for these only): codes, receive
+        // rows, send rows, each launched as a dependent of the kernel before it
+        if (total_tiles != 0) {
+            // blocks of 32 ranks scanned as one where the p are large enough for most blocks to lie
+            // inside one of them
+            if (total_ranks / num_p >= (uint64_t)kCodesCta)
+                codes_batch_kernel<<<(unsigned)((total_ranks + kCodesCta - 1) / kCodesCta), kCodesThreads, 0, stream>>>(ba, codes);
+            else
+                codes_batch_flat_kernel<<<(unsigned)((total_ranks + kCodesTile - 1) / kCodesTile), kTile, 0, stream>>>(ba, codes);
             if ((st = launch_status()) != BCS_OK) return st;
+            if (send_out != nullptr)
+                launch_dependent(true, recv_quad_batch_kernel<true>, (unsigned)total_tiles, kQuadThreads, stream, ba,
+                                 (const uint32_t *)codes, recv_out, recv_t);
+            else
+                launch_dependent(true, recv_quad_batch_kernel<false>, (unsigned)total_tiles, kQuadThreads, stream, ba,
+                                 (const uint32_t *)codes, recv_out, (int8_t *)nullptr);
+            if ((st = launch_status()) != BCS_OK) return st;
+            if (send_out != nullptr) {
+                launch_dependent(true, send_batch_kernel, (unsigned)(2 * total_tiles), kTrThreads, stream, ba,
+                                 (const int8_t *)recv_t, send_out);
+                if ((st = launch_status()) != BCS_OK) return st;
+            }
         }
-        return BCS_OK;
+        // the p up to kFusedMaxP, one CTA each; needs nothing of the kernels before it and does not
+        // wait for them (the host cannot tell whether the list holds such p: their CTAs return at once
+        // where it does not)
+        if (send_out != nullptr)
+            launch_dependent(total_tiles != 0, fused_small_batch_kernel<true>, num_p, kFusedThreads, stream, ba,
+                             recv_out, send_out);
+        else
+            launch_dependent(total_tiles != 0, fused_small_batch_kernel<false>, num_p, kFusedThreads, stream, ba,
+                             recv_out, (int8_t *)nullptr);
+        return launch_status();
     }
     recv_kernel<true><<<blocks, kTile, 0, stream>>>(none, 0, 0, ba, recv_out);
     if ((st = launch_status()) != BCS_OK) return st;

@@ -66,9 +66,13 @@ def test_batch_plan_host_side(lib):
     plan = lib.bcs_batch_plan([2, 3, 20, 1, 1025])
     assert plan.rank_off.tolist() == [0, 2, 5, 25, 26, 1051]
     assert plan.entry_off.tolist() == [0, 2, 8, 108, 108, 108 + 1025 * 11]
-    assert plan.tile_off.tolist() == [0, 1, 2, 3, 4, 7]                    # ceil(p / 512) tiles per p
-    assert plan.copy_off.tolist() == [0, 16, 48, 208, 208, 208 + 11 * 1040]  # q rounds of align16(p) bytes
-    assert plan.total_tiles == 7 and plan.workspace_bytes() == 4352 + 208 + 11 * 1040
+    # tiles of 512 ranks and q rounds of align16(p) bytes of scratch for a p above 1024 only: a
+    # smaller p is built by one CTA that keeps everything in shared memory
+    assert plan.tile_off.tolist() == [0, 0, 0, 0, 0, 3]
+    assert plan.copy_off.tolist() == [0, 0, 0, 0, 0, 11 * 1040]
+    assert plan.total_tiles == 3 and plan.workspace_bytes() == 4352 + 11 * 1040
+    small = lib.bcs_batch_plan([1024, 7, 1])
+    assert small.total_tiles == 0 and small.total_copy == 0 and small.workspace_bytes() == 256
     assert plan.skips_tab[2].tolist()[:6] == [1, 2, 3, 5, 10, 20]
     assert plan.skips_tab[3].tolist()[:2] == [1, 0]
     # full_tab[d] = skip code of rank skips[d]-1: p = 20, skips 1 2 3 5 10 20:
