@@ -466,9 +466,9 @@ def _bench_batch(torch, bcs, workloads, flush, full, hbm_gbs, sm_max_mhz, counts
         torch, lambda: bcs.bcs_build_batch(dplan, br, bs, bw),
         flush, 20, 3))
     batch_kernels = ["codes_batch_kernel", "recv_quad_batch_kernel<true>", "send_batch_kernel"]
-    small_kernels = ["codes_batch_flat_kernel", "recv_quad_batch_kernel<true>", "send_batch_kernel"]
+    small_kernels = ["fused_small_batch_kernel<true>"]
     out["batch_small_sweep"] = {
-        "workload": "every p in 2..1024, all ranks, one bcs_build_batch (three launches)",
+        "workload": "every p in 2..1024, all ranks, one bcs_build_batch (one launch: a CTA per p)",
         "ranks": plan.total_ranks, "ms": ms, "ranks_per_s": plan.total_ranks / ms * 1e3,
         "out_gbs": 2 * plan.total_entries / ms / 1e6,
         "l2": "flushed before every timed step",

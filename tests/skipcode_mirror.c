@@ -333,6 +333,99 @@ int skm_codes_plain(uint32_t p, uint64_t g_begin, uint64_t g_end, uint32_t *code
     return 0;
 }
 
+/* ------------------------------------------------------------ small p, everything in one block
+ * What the batch kernel for p <= 1024 does: the baseblock bits of all ranks as level 0 of a table
+ * run[l][x] = bits of the 2^l ranks that end at x (cyclically; the root has no bit), one level
+ * from the one below; a window of L ranks that ends at rank e is run[l][e] | run[l][e - (L - 2^l)]
+ * with l = floor(log2 L); every round of every rank looks its first window up, and the second one
+ * when the first holds nothing new.  Operations charged (whole operations): the code of a rank 3
+ * per level; a table entry 4 (index, wrap, two loads counted as one, or); a round 6 for what the
+ * round shares among the ranks of a thread (a quarter each), then 3 for the window's end, 3 for
+ * the other run's index, 2 loads, 2 for or / and-not, 1 test, 3 for leading bit, bit and B, 2 for
+ * the entry, 1 store; a second window 10 more; the home round 2; a send entry 5 (to-processor,
+ * wrap, index, load, store). */
+#define SKM_SMALL_MAX 1024
+
+int skm_small(uint32_t p, int8_t *recv, int8_t *send, uint64_t *counters)
+{
+    if (p == 0 || p > SKM_SMALL_MAX || recv == NULL) return -1;
+    skm_ctx c;
+    ctx_init(&c, p);
+    const int q = c.q;
+    if (q == 0) return 0;
+    static uint16_t run[10][SKM_SMALL_MAX];
+    uint32_t code[SKM_SMALL_MAX];
+    uint64_t ops = 0;
+    for (uint32_t x = 0; x < p; ++x) {
+        uint32_t v = x, cd = 0;
+        for (int k = q - 1; k >= 0; --k)
+            if (v >= c.s[k]) { v -= c.s[k]; cd |= 1u << k; }
+        code[x] = cd;
+        run[0][x] = (uint16_t)(cd & (0u - cd));
+        ops += 3ull * q + 2;
+    }
+    const int top = top_bit(p - 1);
+    for (int l = 1; l <= top; ++l) {
+        const uint32_t half = 1u << (l - 1);
+        for (uint32_t x = 0; x < p; ++x) {
+            run[l][x] = run[l - 1][x] | run[l - 1][(x + p - half) % p];
+            ops += 4;
+        }
+    }
+    uint64_t rounds_first = 0, rounds_second = 0, rounds_home = 0;
+    for (uint32_t r = 0; r < p; ++r) {
+        const uint32_t cd = code[r];
+        const int h = top_bit(cd);
+        uint32_t B = cd & (0u - cd);
+        ops += 3;
+        for (int i = 0; i < q; ++i) {
+            const uint32_t lo = c.s[i], hi = c.s[i + 1];
+            int entry;
+            if (i == h) {
+                entry = cd ? __builtin_ctz(cd) : 0;
+                ops += 2;
+                rounds_home += 1;
+            } else {
+                const uint32_t len1 = hi - lo;
+                const int l1 = top_bit(len1);
+                const uint32_t e = (r + p - lo) % p;
+                uint32_t U = (run[l1][e] | run[l1][(e + p - (len1 - (1u << l1))) % p]) & ~B;
+                ops += 2 + 17;                       /* 6/4 rounded up for the shared part */
+                rounds_first += 1;
+                if (U == 0) {
+                    const uint32_t len = c.len2[i];
+                    if (len >= p) U = ((1u << q) - 1u) & ~B;
+                    else if (len) {
+                        const int l2 = top_bit(len);
+                        const uint32_t e2 = (r + p - hi % p) % p;
+                        U = (run[l2][e2] | run[l2][(e2 + p - (len - (1u << l2))) % p]) & ~B;
+                    }
+                    ops += 10;
+                    rounds_second += 1;
+                }
+                const int blk = top_bit(U);
+                if (blk >= 0) B |= 1u << blk;
+                entry = blk >= 0 ? blk - q : 127;
+            }
+            recv[(uint64_t)r * q + i] = (int8_t)entry;
+        }
+    }
+    if (send) {
+        for (uint32_t r = 0; r < p; ++r)
+            for (int k = 0; k < q; ++k)
+                send[(uint64_t)r * q + k] = recv[(uint64_t)((r + c.s[k]) % p) * q + k];
+    }
+    if (counters) {
+        counters[SKM_RANKS] += p;
+        counters[SKM_TABLE_OPS] += Q4(ops);
+        counters[SKM_SEND_OPS] += Q4(5ull * p * q);
+        counters[SKM_ROUNDS_TABLE] += rounds_first;
+        counters[SKM_ROUNDS_SECOND] += rounds_second;
+        counters[SKM_ROUNDS_HOME] += rounds_home;
+    }
+    return 0;
+}
+
 /* ------------------------------------------------------------------------------------ API */
 int skm_q(uint32_t p)
 {

@@ -44,6 +44,7 @@ def _load():
         L.skm_full.argtypes = [c.c_uint32, c.c_void_p, c.c_void_p, c.c_void_p]
         L.skm_codes_blocks.argtypes = [c.c_uint32, c.c_uint64, c.c_uint64, c.c_void_p, c.c_void_p]
         L.skm_codes_plain.argtypes = [c.c_uint32, c.c_uint64, c.c_uint64, c.c_void_p]
+        L.skm_small.argtypes = [c.c_uint32, c.c_void_p, c.c_void_p, c.c_void_p]
         L.skm_set_table_mode.argtypes = [c.c_int]
         L.skm_set_table_mode.restype = None
         assert L.skm_ncount() == len(COUNTERS)
@@ -88,6 +89,20 @@ def rows(p: int, ranks, want_send: bool = True):
                     send.ctypes.data if want_send else None, cnt.ctypes.data)
     if rc:
         raise RuntimeError("skm_rows: %d" % rc)
+    return recv, send, _counts(cnt)
+
+
+def small(p: int, want_send: bool = True):
+    """(recv [p][q], send [p][q] or None, counters) for all ranks of a p <= 1024 by the run table
+    over all ranks (what the batch kernel for small p does)."""
+    L = _load()
+    q = L.skm_q(p)
+    recv = np.zeros((p, q), dtype=np.int8)
+    send = np.zeros((p, q), dtype=np.int8) if want_send else None
+    cnt = np.zeros(len(COUNTERS), dtype=np.uint64)
+    rc = L.skm_small(p, recv.ctypes.data, send.ctypes.data if want_send else None, cnt.ctypes.data)
+    if rc:
+        raise RuntimeError("skm_small: %d" % rc)
     return recv, send, _counts(cnt)
 
 
@@ -157,11 +172,10 @@ def model_table() -> dict:
         weight += pj
     table["batch_4096p"] = dict(per_rank(tot), sample="512 seeded ranks of each p, weighted by p",
                                 total_ranks=weight)
-    # every p in 2..1024
+    # every p in 2..1024, as one batch: each p by the run table over all its ranks
     tot = {}
     for pj in workloads.small_sweep():
-        _, _, c = full(pj, want_send=False)
-        c["send_ops"] = 7 / 4 * skm_q(pj) * c["ranks"]
+        _, _, c = small(pj, want_send=True)
         for k, v in c.items():
             tot[k] = tot.get(k, 0.0) + v
     table["small_sweep_2_1024"] = dict(per_rank(tot), sample="all ranks of every p")

@@ -105,3 +105,16 @@ def test_block_codes_equal_the_plain_scan():
             got, st = skm.codes_blocks(p, g, end)
             assert np.array_equal(got, skm.codes_plain(p, g, end)), (p, g)
             assert st["plain"] == 0, (p, g, st)
+
+
+def test_small_p_run_table_construction_equals_the_oracle():
+    """The construction of the batch kernel for p <= 1024 (baseblock bits of all ranks, runs of
+    2^l ranks, every window looked up as an exact set) gives the oracle's tables for every such p."""
+    import numpy as np
+    import oracle
+    from tests import skipcode_mirror as skm
+    for p in range(2, 1025):
+        recv, send, _ = skm.small(p)
+        want_r, want_s = oracle.full_table(p)
+        assert np.array_equal(recv, want_r), p
+        assert np.array_equal(send, want_s), p
