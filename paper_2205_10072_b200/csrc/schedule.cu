@@ -17,7 +17,9 @@
 //    sendsched[r][k] = recvsched[(r+skips[k]) mod p][k] as a transposition with row k rotated by
 //    skips[k] (send_rm_kernel: sub-ranges, byte gathers and recomputation for to-processors
 //    outside the range).  The kernels of a build are launched as dependents of one another
-//    (bcs_common.cuh), so each is brought onto the SMs while the one before it drains.
+//    (bcs_common.cuh), so each is brought onto the SMs while the one before it drains.  In a
+//    batch, every p up to 1024 is built by ONE CTA of fused_small_batch_kernel instead: codes,
+//    a table of exact window sets over all ranks of the p, both tables, all in shared memory.
 //
 //  * self-contained path (no workspace).  One thread per rank runs Algorithm 4 with the range
 //    search done by descending the homeranges; the send schedule is looked up in the rank-major
