@@ -27,6 +27,7 @@
 //    (Algorithm 5) where it is not.
 #include <cstddef>
 #include <mutex>
+#include <type_traits>
 
 #include "bcs_common.cuh"
 #include "paper_path.cuh"
@@ -581,10 +582,9 @@ struct QuadConsts {
     int32_t word[kQuadTableRounds][4][4];
     uint32_t len2[kRow];     // length of the second window of round i, or 0
     int table_rounds;        // rounds 0 .. table_rounds-1 are decided from the run table
-    // bit k of aligned[w]: the four window bounds that a quad loads at its first rank minus
-    // skips[k] (w = 0) or plus p minus skips[k] (w = 1: past the home round) start on a 16-byte
-    // boundary of the codes, so that they can be loaded as one 16-byte word
-    uint32_t aligned[2];
+    // bit k: the four window bounds that a quad loads at its first rank minus skips[k] start on a
+    // 16-byte boundary of the codes, so that they can be loaded as one 16-byte word
+    uint32_t aligned;
     // tiles that (may) hold a quad for the general code: those of the ranks skips[k], the first
     // and the last of the range; distinct, n_special <= 32 (missing one costs time, not correctness)
     uint32_t special[kRow];
@@ -650,8 +650,7 @@ inline QuadConsts make_quad_consts(const PTable &tab, uint64_t r_begin, uint64_t
     qc.table_rounds = quad_table_rounds(tab.s, tab.q);
     // quads start at ranks r_begin + multiples of 4, the codes at a 16-byte boundary
     for (int k = 0; k <= tab.q; ++k) {
-        if ((((uint32_t)r_begin - tab.s[k]) & 3u) == 0) qc.aligned[0] |= 1u << k;
-        if ((((uint32_t)r_begin + tab.p - tab.s[k]) & 3u) == 0) qc.aligned[1] |= 1u << k;
+        if ((((uint32_t)r_begin - tab.s[k]) & 3u) == 0) qc.aligned |= 1u << k;
     }
     for (int i = 0; i < qc.table_rounds; ++i)
         for (int w = 0; w < 4; ++w)
@@ -668,7 +667,6 @@ struct ParamEnv {
     __device__ __forceinline__ int word(int i, int w, int j) const { return qc.word[i][w][j]; }
     __device__ __forceinline__ uint32_t len2(int i) const { return qc.len2[i]; }
     __device__ __forceinline__ int table_rounds() const { return qc.table_rounds; }
-    __device__ __forceinline__ uint32_t aligned(int w) const { return qc.aligned[w]; }
 };
 // ... or shared memory (batch: the CTA computes them for the p of its tile).
 struct SharedEnv {
@@ -678,7 +676,6 @@ struct SharedEnv {
     __device__ __forceinline__ int word(int i, int w, int j) const { return qc->word[i][w][j]; }
     __device__ __forceinline__ uint32_t len2(int i) const { return qc->len2[i]; }
     __device__ __forceinline__ int table_rounds() const { return qc->table_rounds; }
-    __device__ __forceinline__ uint32_t aligned(int w) const { return qc->aligned[w]; }
 };
 
 // One tile: the n <= 512 ranks first .. first+n-1 of a p >= 64 (first may exceed p for the
@@ -883,13 +880,16 @@ __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh
         // group is the same for all quads of a launch (the ranks of quads are multiples of 4
         // apart); where they fill the group -- skips that are multiples of 4, e.g. the powers of
         // two of a p just below one -- they come as ONE 16-byte load, which touches a quarter of
-        // the L1 sectors of four one-word loads with the lanes 16 bytes apart.  The host says for
-        // which skips that holds (a test on the address would not be uniform for the compiler) and
-        // picks the instantiation with this test only for a p with many such skips: the test
-        // costs the other rounds a few percent.
-        auto load4 = [&](uint32_t (&dst)[4], uint32_t from, int k, uint32_t aligned_skips) {
+        // the L1 sectors of four one-word loads with the lanes 16 bytes apart.  kWideLoads: the
+        // host has checked that this holds for every round before the home round of any rank of
+        // the launch, and those rounds load 16 bytes unconditionally.  (A test per round, for a p
+        // with only some such skips, was compiled into both kinds of loads under a predicate: the
+        // four one-word loads were issued, switched off, in every round -- 4 % of the kernel's
+        // issue slots.)  The rounds past the home round load word by word: p is rarely a multiple
+        // of 4 further on.
+        auto load4 = [&](uint32_t (&dst)[4], uint32_t from, int k, auto wide) {
             const uint32_t *src = codes + (from - env.skip(k));
-            if (kWideLoads && ((aligned_skips >> k) & 1u)) {
+            if (decltype(wide)::value) {
                 const uint4 v = *reinterpret_cast<const uint4 *>(src);
                 dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
             } else {
@@ -925,7 +925,7 @@ __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh
             }
         };
         // rounds i .. end-1 with the window bounds at from - skip (from = r[0] or r[0] + p)
-        auto rounds_until = [&](int end, uint32_t from, const uint32_t aligned_skips) {
+        auto rounds_until = [&](int end, uint32_t from, auto aligned_skips) {
             if (i >= end) return;
             uint32_t ahead[4];
             load4(ahead, from, i + 1, aligned_skips);
@@ -981,17 +981,17 @@ __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh
                 store_round(entry);
             }
         };
-        load4(upper, r[0], i, env.aligned(0));                   // i <= h0: skips[i] <= r[0]
-        rounds_until(h0, r[0], env.aligned(0));
+        load4(upper, r[0], i, std::integral_constant<bool, kWideLoads>());   // i <= h0: skips[i] <= r[0]
+        rounds_until(h0, r[0], std::integral_constant<bool, kWideLoads>());
         {                                                      // home round: the baseblocks themselves
             int entry[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) entry[j] = __ffs(c[j]) - 1;
             store_round(entry);
-            load4(upper, r[0] + p, h0 + 1, env.aligned(1));       // r[3] < skips[h0+1]
+            load4(upper, r[0] + p, h0 + 1, std::false_type());    // r[3] < skips[h0+1]
             i = h0 + 1;
         }
-        rounds_until(q, r[0] + p, env.aligned(1));
+        rounds_until(q, r[0] + p, std::false_type());
     }
 }
 
@@ -1558,10 +1558,10 @@ send_batch_kernel(BatchArgs ba, const int8_t *__restrict__ recv_t, int8_t *send_
 }
 
 // Launches the quad receive kernel of one p >= 64 for a range, as a dependent of the kernel
-// before it on the stream.  The instantiation that loads aligned window bounds as 16-byte words
-// is taken when the bounds of at least four fifths of the rounds before the home round are
-// aligned (a p just below a power of two: its skips are powers of two); measured, it gains
-// 2-5 % there and loses as much where only few rounds, or only those past the home round, are.
+// before it on the stream.  The instantiation that loads the window bounds of the rounds before
+// the home round as 16-byte words is taken when all of them are aligned (a p in the top 32nd of
+// its octave, whose skips from 32 on are powers of two, and a range that starts at a multiple of
+// 4): 10 % fewer L1 wavefronts and 5 % fewer issue slots than the one-word loads.
 template <bool kRowOut, bool kColOut>
 inline void launch_recv_quad(const PTable &tab, const QuadConsts &qc, uint64_t r_begin, uint64_t r_end,
                              const uint32_t *codes, int8_t *recv_out, int8_t *recv_t, uint64_t t_stride,
@@ -1569,18 +1569,16 @@ inline void launch_recv_quad(const PTable &tab, const QuadConsts &qc, uint64_t r
 {
     const uint64_t count = r_end - r_begin;
     const unsigned grid = (unsigned)((count + kQuadTile - 1) / kQuadTile) + (unsigned)qc.n_special;
-    int wide = 0, rounds = 0;
-    for (int k = qc.table_rounds + 1; k <= tab.q; ++k) {
-        wide += (int)((qc.aligned[0] >> k) & 1u);
-        rounds += 1;
-    }
+    // bounds of every round from the first per-lane round to the last possible home round
+    bool all_wide = true;
+    for (int k = qc.table_rounds; k < tab.q; ++k) all_wide = all_wide && ((qc.aligned >> k) & 1u);
     // rows of a q that is a multiple of 4 are stored word by word (see put_rows)
     const bool word_rows = kRowOut && (tab.q & 3) == 0;
     auto go = [&](auto kernel) {
         launch_dependent(true, kernel, grid, kQuadThreads, stream, tab, qc, r_begin, r_end, codes, recv_out, recv_t,
                          t_stride);
     };
-    if (5 * wide >= 4 * rounds) {
+    if (all_wide) {
         if (word_rows) go(recv_codes_quad_kernel<kRowOut, kColOut, true, kRowOut>);
         else go(recv_codes_quad_kernel<kRowOut, kColOut, true, false>);
     } else {
