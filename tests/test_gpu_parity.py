@@ -168,6 +168,33 @@ def test_batch_of_large_and_tiny_p_mixed(bcs):
         assert np.array_equal(send[eo[j]:eo[j + 1]].cpu().numpy().reshape(p, -1), want_s), (j, p)
 
 
+def test_batch_output_is_complete_for_the_next_operation_on_the_stream(bcs):
+    """The kernels of a batch are launched as dependents of one another and the last one (the
+    CTAs of the small p) does not wait for the tiled kernels of the large p before it starts.
+    Whatever follows on the stream must still see both tables complete: a copy enqueued right
+    after the call, without a synchronisation in between, is compared with the oracle."""
+    plist = [5, 2**20 + 1, 300, 1000, 77]
+    plan = bcs.bcs_batch_plan(plist)
+    dev = plan.to("cuda")
+    want = {p: oracle.full_table(p) for p in set(plist)}
+    ws = torch.empty(plan.workspace_bytes(), dtype=torch.int8, device="cuda")
+    side = torch.cuda.Stream()
+    for stream in (None, side):
+        for _ in range(3):
+            recv = torch.full((plan.total_entries,), 99, dtype=torch.int8, device="cuda")
+            send = torch.full((plan.total_entries,), 99, dtype=torch.int8, device="cuda")
+            torch.cuda.synchronize()
+            with torch.cuda.stream(stream if stream is not None else torch.cuda.current_stream()):
+                bcs.bcs_build_batch(dev, recv, send, ws)
+                snap_r, snap_s = recv.clone(), send.clone()      # same stream, no synchronisation
+            torch.cuda.synchronize()
+            eo = plan.entry_off.tolist()
+            for j, p in enumerate(plist):
+                q = oracle.q_of(p)
+                assert np.array_equal(snap_r[eo[j]:eo[j + 1]].cpu().numpy().reshape(p, q), want[p][0]), (j, p)
+                assert np.array_equal(snap_s[eo[j]:eo[j + 1]].cpu().numpy().reshape(p, q), want[p][1]), (j, p)
+
+
 # ---------------------------------------------------------------- ranges, tails, degenerate
 @pytest.mark.parametrize("fast", [True, False])
 def test_sub_ranges_ragged_tails_and_single_outputs(bcs, fast):
