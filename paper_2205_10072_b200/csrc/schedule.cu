@@ -539,8 +539,8 @@ struct SharedSkips {
 // address, their four entries one aligned 32-bit word of the copy.  A thread whose four ranks
 // lie in the same homerange past the table rounds (all but a few dozen quads of a p) runs the
 // rounds for the four together, with the wrap decided per quad: before the home round h every
-// window bound is r - skip, after it r + p - skip.  A tile that holds any other quad (around a
-// skip, next to the root, at the end of the range: a few dozen tiles of a p) runs the general
+// window bound is r - skip, after it r + p - skip.  A warp that holds any other quad (around a
+// skip, next to the root, at the end of the range: a few dozen warps of a p) runs the general
 // code, home round and wrap tested per rank, for all its quads.
 //
 // The run table of the tile is kept as four sub-tables by position mod 4:
@@ -759,10 +759,11 @@ __device__ __forceinline__ void quad_tile(const Env env, const uint32_t *full_sh
     const int h0 = 31 - __clz(c[0]);                           // -1 for the root
     const bool together = 4u * t + 4u <= n && r[0] != 0u && r[3] == r[0] + 3u &&
                           h0 == 31 - __clz(c[3]) && h0 >= first_lane_round;
-    // One path for the whole tile (no divergence inside a warp): the general one if any of its
-    // quads needs it -- the first tile, the last, and the tiles in which a homerange starts.
+    // One path for a whole warp (no divergence inside it): the general one if any of its quads
+    // needs it -- in the first tile, the last, and the tiles in which a homerange starts.  Neither
+    // path has a barrier, so the other warps of such a tile keep the fast one.
     const bool empty = 4u * t >= n;
-    if (__syncthreads_or(!empty && !together)) {
+    if (__any_sync(0xffffffffu, !empty && !together)) {
         // Four ranks, each with its own homerange, wrap and validity: the table rounds with the
         // home round tested per rank, then recv_round for every rank and round.
         int h[4], bb[4];
