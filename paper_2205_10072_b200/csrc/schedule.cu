@@ -101,35 +101,41 @@ constexpr int kCodesThreads = 256;
 constexpr int kCodesSub = 32;                                   // consecutive ranks scanned as one
 constexpr int kCodesCta = kCodesThreads * kCodesSub;            // ranks per CTA
 constexpr int kCodesLow = 8;
+// Ranks per scan in the kernel of one p: 32 where the kernel streams (4 million ranks and more:
+// fewest instructions per rank), 16 for a smaller p, where its latency counts: twice the threads,
+// each with half the quads to write (p = 2^20+1: 1.1 us less).
+__host__ __device__ constexpr int codes_sub(int q) { return q <= 22 ? 16 : 32; }
 
 struct BlockScan {
-    uint32_t biased;   // remainder of the block's first rank, plus 31
+    uint32_t biased;   // remainder of the block's first rank, plus (ranks per block - 1)
     uint32_t code;     // its code so far
-    uint32_t stay;     // ranks g .. g+stay-1 decide like g; 32 while no level has split the block
+    uint32_t stay;     // ranks g .. g+stay-1 decide like g; the whole block while no level has split it
     uint32_t left;     // code, down to the splitting level, of the ranks that left there
     uint32_t plain;    // a second splitting level was met
 };
 
+template <int kSub = kCodesSub>
 __device__ __forceinline__ void scan_level(BlockScan &b, uint32_t skip, int k)
 {
     const uint32_t u = b.biased - skip;
-    if (u < (uint32_t)(kCodesSub - 1)) {              // skip - 31 <= remainder < skip: rare
-        if (b.stay == kCodesSub) {
-            b.stay = (kCodesSub - 1) - u;             // = skip - remainder
+    if (u < (uint32_t)(kSub - 1)) {                   // skip - (kSub - 1) <= remainder < skip: rare
+        if (b.stay == kSub) {
+            b.stay = (kSub - 1) - u;                  // = skip - remainder
             b.left = b.code | (1u << k);
         } else {
             b.plain = 1;
         }
     }
-    if ((int32_t)u >= kCodesSub - 1) {
+    if ((int32_t)u >= kSub - 1) {
         b.biased = u;
         b.code |= 1u << k;
     }
 }
 
+template <int kSub = kCodesSub>
 __device__ __forceinline__ uint4 pack_scan(const BlockScan &b)
 {
-    return make_uint4(b.biased - (kCodesSub - 1), b.code, b.stay | (b.plain << 8), b.left);
+    return make_uint4(b.biased - (kSub - 1), b.code, b.stay | (b.plain << 8), b.left);
 }
 
 // Codes of the four ranks at offset e0 .. e0+3 of a block whose scan is sb (no second split).
@@ -177,23 +183,25 @@ codes_single_kernel(const __grid_constant__ PTable tab, uint32_t *__restrict__ c
         low[threadIdx.x] = (uint16_t)c;
     }
     const uint32_t lane = threadIdx.x & 31u;
-    const uint32_t first = (blockIdx.x * kCodesThreads + (threadIdx.x & ~31u)) * (uint32_t)kCodesSub;
+    constexpr int kSub = codes_sub(kQ);
+    constexpr uint32_t kSubQuads = kSub / 4;                       // quads per block: 4 or 8
+    const uint32_t first = (blockIdx.x * kCodesThreads + (threadIdx.x & ~31u)) * (uint32_t)kSub;
     {
-        const uint32_t g = first + kCodesSub * lane;
-        BlockScan b = {g + (kCodesSub - 1), 0, kCodesSub, 0, 0};
+        const uint32_t g = first + kSub * lane;
+        BlockScan b = {g + (kSub - 1), 0, kSub, 0, 0};
         if (g < tab.p) {
 #pragma unroll
-            for (int k = kQ - 1; k >= kLow; --k) scan_level(b, tab.s[k], k);
+            for (int k = kQ - 1; k >= kLow; --k) scan_level<kSub>(b, tab.s[k], k);
         }
-        sub[threadIdx.x] = pack_scan(b);
+        sub[threadIdx.x] = pack_scan<kSub>(b);
     }
     __syncthreads();
-    const uint32_t e0 = 4u * (lane & 7u);
+    const uint32_t e0 = 4u * (lane % kSubQuads);
 #pragma unroll 2
-    for (uint32_t i = 0; i < 8; ++i) {
+    for (uint32_t i = 0; i < kSubQuads; ++i) {
         const uint32_t g = first + 4u * (i * 32u + lane);
         if (g >= tab.p) break;
-        const uint4 sb = sub[(threadIdx.x & ~31u) + i * 4u + (lane >> 3)];
+        const uint4 sb = sub[(threadIdx.x & ~31u) + i * (32u / kSubQuads) + lane / kSubQuads];
         if (sb.z < 256u && g + 4u <= tab.p) {
             *reinterpret_cast<uint4 *>(codes + g) = quad_codes(sb, low, e0);
         } else {
@@ -204,22 +212,23 @@ codes_single_kernel(const __grid_constant__ PTable tab, uint32_t *__restrict__ c
 
 template <int kQ>
 struct CodesLauncher {
-    static void launch(int q, const PTable &tab, uint32_t *codes, unsigned blocks, cudaStream_t stream)
+    static void launch(int q, const PTable &tab, uint32_t *codes, cudaStream_t stream)
     {
+        constexpr unsigned per_cta = kCodesThreads * codes_sub(kQ);
         if (q == kQ)
-            codes_single_kernel<kQ><<<blocks, kCodesThreads, 0, stream>>>(tab, codes);
+            codes_single_kernel<kQ><<<(tab.p + per_cta - 1) / per_cta, kCodesThreads, 0, stream>>>(tab, codes);
         else
-            CodesLauncher<kQ - 1>::launch(q, tab, codes, blocks, stream);
+            CodesLauncher<kQ - 1>::launch(q, tab, codes, stream);
     }
 };
 template <>
 struct CodesLauncher<0> {
-    static void launch(int, const PTable &, uint32_t *, unsigned, cudaStream_t) {}
+    static void launch(int, const PTable &, uint32_t *, cudaStream_t) {}
 };
 
 inline void launch_codes(const PTable &tab, uint32_t *codes, cudaStream_t stream)
 {
-    CodesLauncher<BCS_MAX_Q>::launch(tab.q, tab, codes, (unsigned)((tab.p + kCodesCta - 1) / kCodesCta), stream);
+    CodesLauncher<BCS_MAX_Q>::launch(tab.q, tab, codes, stream);
 }
 
 // Batch: codes[g] for the flattened rank g, 8192 flattened ranks per CTA, scanned in blocks of
