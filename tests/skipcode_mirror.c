@@ -236,7 +236,7 @@ static void recv_row(const skm_ctx *c, uint32_t r, int last, int8_t *row, uint64
 }
 
 /* ------------------------------------------------------------------ codes, 32 ranks per scan
- * The codes of the 32 consecutive ranks g .. g+31 from one greedy scan.  Rank g+e decides like g
+ * The codes of 32 consecutive ranks g .. g+31 (16 for q <= 22) from one greedy scan.  Rank g+e decides like g
  * at every level until the one where the remainder R of g has R < skips[k] <= R + e: there g+e
  * takes skips[k] and keeps R + e - skips[k] < 31, and g does not take it.  The levels below LOW
  * come from a table, low[v] = code of v over those levels (v < skips[LOW]), which also serves
@@ -245,10 +245,13 @@ static void recv_row(const skm_ctx *c, uint32_t r, int last, int8_t *row, uint64
  * Operations charged (whole operations, to ops[0]): per level of the scan 5 (subtract, the two
  * tests, select, or), 3 more at a splitting level; per four ranks 3 for the side of the split and
  * the table address, 4 table loads, 4 or, 1 vector store, and 8 more where the split falls
- * inside the four; the table's 3 per level and entry once per 8192 ranks; a plain scan 3 per
+ * inside the four; the table's 3 per level and entry once per 256 blocks; a plain scan 3 per
  * level and rank.  ops[1] = blocks, ops[2] = blocks with a splitting level, ops[3] = plain. */
 #define SKM_LOW 8
-#define SKM_BLOCK 32
+#define SKM_BLOCK 32          /* ranks per scan for q > 22; 16 for a smaller p */
+static int g_batch = 0;       /* the batch kernel scans 32 ranks at a time for every q */
+void skm_set_batch(int on) { g_batch = on; }
+static uint32_t block_of(int q) { return (q <= 22 && !g_batch) ? 16u : SKM_BLOCK; }
 #define SKM_BLOCKS_FROM 8192   /* smaller p are charged the plain scan, 3 per level and rank (the
                                   GPU scans them rank by rank: most blocks would cross p) */
 
@@ -256,22 +259,23 @@ static void codes_block(const skm_ctx *c, const uint16_t *low, int low_levels, u
                         uint32_t *out /* 32, or NULL */, uint64_t *ops)
 {
     const uint32_t p = c->p;
-    uint32_t rem = g, code = 0, stay = SKM_BLOCK, left = 0;
+    const uint32_t block = block_of(c->q);
+    uint32_t rem = g, code = 0, stay = block, left = 0;
     int plain = 0;
     for (int k = c->q - 1; k >= low_levels; --k) {
         const uint32_t skip = c->s[k];
         ops[0] += 5;
-        if (rem < skip && skip <= rem + (SKM_BLOCK - 1)) {
+        if (rem < skip && skip <= rem + (block - 1)) {
             ops[0] += 3;
-            if (stay == SKM_BLOCK) { stay = skip - rem; left = code | (1u << k); }
+            if (stay == block) { stay = skip - rem; left = code | (1u << k); }
             else plain = 1;
         }
         if (rem >= skip) { rem -= skip; code |= 1u << k; }
     }
     ops[1] += 1;
-    if (stay != SKM_BLOCK) ops[2] += 1;
+    if (stay != block) ops[2] += 1;
     if (plain) ops[3] += 1;
-    for (uint32_t e0 = 0; e0 < SKM_BLOCK && g + e0 < p; e0 += 4) {
+    for (uint32_t e0 = 0; e0 < block && g + e0 < p; e0 += 4) {
         if (plain) ops[0] += 4ull * 3 * (uint64_t)c->q;
         else ops[0] += 12 + ((stay > e0 && stay < e0 + 4) ? 8 : 0);
         for (uint32_t e = e0; e < e0 + 4 && g + e < p; ++e) {
@@ -314,11 +318,12 @@ int skm_codes_blocks(uint32_t p, uint64_t g_begin, uint64_t g_end, uint32_t *cod
     uint16_t low[1 << SKM_LOW];
     const int levels = build_low(&c, low);
     uint32_t tmp[SKM_BLOCK];
-    for (uint64_t g = g_begin; g < g_end; g += SKM_BLOCK) {
-        if ((g - g_begin) % 8192 == 0) ops[0] += (3ull * levels) << levels;
+    const uint32_t block = block_of(c.q);
+    for (uint64_t g = g_begin; g < g_end; g += block) {
+        if ((g - g_begin) % (256u * block) == 0) ops[0] += (3ull * levels) << levels;
         codes_block(&c, low, levels, (uint32_t)g, tmp, ops);
         if (codes)
-            for (uint32_t e = 0; e < SKM_BLOCK && g + e < g_end; ++e) codes[g - g_begin + e] = tmp[e];
+            for (uint32_t e = 0; e < block && g + e < g_end; ++e) codes[g - g_begin + e] = tmp[e];
     }
     return 0;
 }
@@ -452,7 +457,7 @@ int skm_rows(uint32_t p, const uint64_t *ranks, uint64_t n, int8_t *recv, int8_t
     for (uint64_t m = 0; m < n; ++m) {
         const uint32_t r = (uint32_t)ranks[m];
         if (r >= p) return -2;
-        if (p >= SKM_BLOCKS_FROM) codes_block(&c, low, levels, r & ~(uint32_t)(SKM_BLOCK - 1), NULL, block_ops);
+        if (p >= SKM_BLOCKS_FROM) codes_block(&c, low, levels, r & ~(block_of(q) - 1u), NULL, block_ops);
         if (recv) recv_row(&c, r, q - 1, recv + m * (uint64_t)q, counters);
         else recv_row(&c, r, q - 1, tmp, counters);
         if (send) {
@@ -466,7 +471,7 @@ int skm_rows(uint32_t p, const uint64_t *ranks, uint64_t n, int8_t *recv, int8_t
     }
     /* every listed rank pays 1/32 of its block's scan and of the table's share of 32 ranks */
     if (counters && p >= SKM_BLOCKS_FROM)
-        counters[SKM_CODE_OPS] += Q4(block_ops[0]) / SKM_BLOCK + Q4(n * ((3ull * levels) << levels)) / 8192;
+        counters[SKM_CODE_OPS] += Q4(block_ops[0]) / block_of(q) + Q4(n * ((3ull * levels) << levels)) / (256u * block_of(q));
     else if (counters)
         counters[SKM_CODE_OPS] += Q4(n * 3ull * (uint64_t)q);
     return 0;

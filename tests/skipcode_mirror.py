@@ -47,6 +47,8 @@ def _load():
         L.skm_small.argtypes = [c.c_uint32, c.c_void_p, c.c_void_p, c.c_void_p]
         L.skm_set_table_mode.argtypes = [c.c_int]
         L.skm_set_table_mode.restype = None
+        L.skm_set_batch.argtypes = [c.c_int]
+        L.skm_set_batch.restype = None
         assert L.skm_ncount() == len(COUNTERS)
         _lib = L
     return _lib
@@ -55,6 +57,12 @@ def _load():
 def set_table_mode(mode: int) -> None:
     """0: short windows from exact sets when p >= 64 (as the GPU); 1: never; 2: for every p."""
     _load().skm_set_table_mode(mode)
+
+
+def set_batch(on: bool) -> None:
+    """Codes as the batch kernel scans them (32 ranks per scan for every q) or as the kernel of
+    one p does (16 for q <= 22)."""
+    _load().skm_set_batch(1 if on else 0)
 
 
 def _counts(raw) -> dict:
@@ -160,6 +168,7 @@ def model_table() -> dict:
     table["q30_p1073741823"] = dict(per_rank(c), p=p, q=skm_q(p),
                                     sample="200000 ranks next() %% p, splitmix64 seed %d" % workloads.SEED_SPOT)
     # batched mix: 512 seeded ranks of each of the 4096 p, weighted by p
+    set_batch(True)
     g = workloads.SplitMix64(workloads.SEED_SPOT)
     tot = {}
     weight = 0
@@ -170,6 +179,7 @@ def model_table() -> dict:
         for k, v in c.items():
             tot[k] = tot.get(k, 0.0) + v * (pj / c["ranks"])
         weight += pj
+    set_batch(False)
     table["batch_4096p"] = dict(per_rank(tot), sample="512 seeded ranks of each p, weighted by p",
                                 total_ranks=weight)
     # every p in 2..1024, as one batch: each p by the run table over all its ranks
